@@ -1,0 +1,23 @@
+import os
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+
+def pytest_configure(config):
+    config.addinivalue_line("markers", "gpu: needs a CUDA device (runs on the B200 box only)")
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _host_builds():
+    """Compile the host-only helpers (generator, oracle) once per session."""
+    import datagen
+    import oracle
+
+    datagen.build_host()
+    oracle.build()
+    yield
