@@ -1,0 +1,281 @@
+/*
+ * sjq -- fused star-join query pipeline for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the library.  The operation is the fused per-row pipeline of the
+ * paper (Section 3.1 "Kernel Composition", Section 3.2 Listing 2, Section 3.3
+ * "Workload-Specific Optimizations", Section 4.2.2 "Fusion in SYCLDB"): one
+ * pass over a columnar fact table that evaluates the fact predicates, probes
+ * one dimension table per join (a miss drops the row, a hit gathers the
+ * dimension's payload), and aggregates the survivors (scalar sum, dense
+ * group array, or hashed groups); the dimension tables are produced
+ * beforehand by a separate build kernel from the filtered dimension columns.
+ *
+ * Conventions
+ *   - Every `data`, `*_dev`, `table_mem`, result and workspace pointer is a
+ *     DEVICE pointer owned by the caller, 16-byte aligned, and must stay
+ *     valid and unmodified until the work enqueued on `stream` has finished.
+ *     Descriptor structs (columns, predicates, expressions, options) are HOST
+ *     memory and are copied during the call.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *   - The library allocates no device memory.  All kernels are enqueued on
+ *     the given stream; calls return after enqueueing unless stated otherwise.
+ *   - Functions return 0 (SJQ_OK) or a host-detected error code.  Errors only
+ *     the device can see are written to the caller's int32 status word (first
+ *     error wins); kernels never trap and never spin without a bound.  Results
+ *     are undefined when the status word is non-zero after the stream syncs.
+ *   - Columns are int32 or int64, contiguous, little-endian.  All arithmetic
+ *     on values is done after sign-extension to 64 bits and wraps modulo 2^64
+ *     (the 64-bit product of Listing 2); `%` truncates toward zero as in C.
+ *   - No CPU fallback exists: without a CUDA device every compute call fails
+ *     with SJQ_ERR_CUDA.
+ */
+#ifndef SJQ_H
+#define SJQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t sjq_status;
+
+enum {
+    SJQ_OK = 0,
+    /* host-detected (returned) */
+    SJQ_ERR_INVALID_ARG = 1,
+    SJQ_ERR_UNSUPPORTED = 2,
+    SJQ_ERR_ALIGN = 3,        /* a device pointer is not 16-byte aligned */
+    SJQ_ERR_CUDA = 4,         /* a CUDA runtime call failed (no device, launch error) */
+    SJQ_ERR_BUFFER_SMALL = 5, /* caller-provided table / workspace memory too small */
+    /* device-detected (written to the status word) */
+    SJQ_ERR_DUP_KEY = 16,        /* two dimension rows passing the filter share a key */
+    SJQ_ERR_TABLE_FULL = 17,     /* open-addressing insert found no free slot */
+    SJQ_ERR_GROUP_RANGE = 18,    /* dense mode: a group key fell outside [0, num_groups) */
+    SJQ_ERR_GROUP_OVERFLOW = 19, /* hashed mode: more distinct groups than the capacity */
+    SJQ_ERR_RESERVED_KEY = 20,   /* a dimension key equals the reserved empty marker (minimum of its type) */
+    SJQ_ERR_LAYOUT_MISMATCH = 21 /* build saw a key or payload outside the planned layout */
+};
+
+enum { SJQ_I32 = 0, SJQ_I64 = 1 };
+
+/* One column: n values of `dtype` at device address `data`. */
+typedef struct sjq_col {
+    const void *data;
+    int32_t dtype;
+    int64_t n;
+} sjq_col;
+
+/* Predicate on one column; a query carries a conjunction of these
+ * (Section 4.2.2: a BETWEEN is the AND of its two inclusive bounds; the
+ * disjunction on one column in the Q4.1 text of Section 3.3 is an IN set). */
+enum { SJQ_EQ = 0, SJQ_NE, SJQ_LT, SJQ_LE, SJQ_GT, SJQ_GE, SJQ_BETWEEN, SJQ_IN };
+#define SJQ_MAX_IN_SET 16
+typedef struct sjq_pred {
+    int32_t col;        /* index into the column array it is applied to */
+    int32_t op;         /* SJQ_EQ ... SJQ_IN; one-sided ops compare with `lo` */
+    int64_t lo, hi;     /* BETWEEN: lo <= v <= hi */
+    const int64_t *set; /* IN: host array of nset values (nset <= SJQ_MAX_IN_SET) */
+    int32_t nset;
+} sjq_pred;
+
+/* A value available to the group key and the aggregate: a fact column
+ * (a = fact column index) or a payload gathered by a join (a = join index,
+ * b = payload index of that join's table), scaled by `mult`. */
+enum { SJQ_SRC_FACT = 0, SJQ_SRC_PAYLOAD = 1 };
+typedef struct sjq_term {
+    int32_t src, a, b;
+    int64_t mult;
+} sjq_term;
+
+/* key = (offset + sum_t mult_t * value_t) [% modulo]; modulo 0 = none. */
+#define SJQ_MAX_KEY_TERMS 4
+typedef struct sjq_key_expr {
+    sjq_term t[SJQ_MAX_KEY_TERMS];
+    int32_t nterms;
+    int64_t offset, modulo;
+} sjq_key_expr;
+
+/* Aggregated value per surviving row: COL: x; MUL: x*y; SUB: x-y; ADD: x+y
+ * (each of x, y already scaled by its `mult`); summed per group in int64. */
+enum { SJQ_AGG_COL = 0, SJQ_AGG_MUL, SJQ_AGG_SUB, SJQ_AGG_ADD };
+typedef struct sjq_agg_expr {
+    int32_t op;
+    sjq_term x, y;
+    int32_t want_count; /* non-zero: also count the rows per group */
+} sjq_agg_expr;
+
+/* ------------------------------------------------------------------ */
+/* Dimension tables (Section 3.3: direct-mapped and byte-packed maps for
+ * dense keys, an open-addressing table otherwise; Section 4.3.1: the key
+ * range is verified at run time and the packed or the unpacked form chosen). */
+
+enum {
+    SJQ_TABLE_AUTO = 0,
+    SJQ_TABLE_DIRECT_BITMAP = 1, /* 1 bit per key in [kmin, kmax]: filter only, no payload */
+    SJQ_TABLE_DIRECT_U8 = 2,     /* 1 byte per key: packed payload code, 0xFF = miss */
+    SJQ_TABLE_DIRECT_U16 = 3,
+    SJQ_TABLE_DIRECT_U32 = 4,
+    SJQ_TABLE_DIRECT_U64 = 5,
+    SJQ_TABLE_HASH_I32 = 6, /* open addressing, linear probing, int32 keys */
+    SJQ_TABLE_HASH_I64 = 7,
+    SJQ_TABLE_FORCE_DIRECT = 100, /* build option only */
+    SJQ_TABLE_FORCE_HASH = 101    /* build option only */
+};
+
+#define SJQ_MAX_PAYLOADS 2
+#define SJQ_PLAN_SCRATCH_BYTES 256
+
+typedef struct sjq_build_opts {
+    int32_t force_kind;       /* SJQ_TABLE_AUTO, SJQ_TABLE_FORCE_DIRECT or SJQ_TABLE_FORCE_HASH */
+    int32_t hash_load_pct;    /* 0 = default 50: slots >= entries * 100 / pct, power of two */
+    int64_t max_direct_bytes; /* 0 = default 64 MiB: larger direct tables fall back to hashing */
+} sjq_build_opts;
+
+/* Shape of a table, decided from the data by sjq_dim_plan. Plain host data. */
+typedef struct sjq_dim_layout {
+    int32_t kind;      /* one of SJQ_TABLE_DIRECT_* / SJQ_TABLE_HASH_* */
+    int32_t key_dtype; /* SJQ_I32 / SJQ_I64 */
+    int32_t npayload;
+    int32_t code_bits;                 /* width of the packed payload code stored per key (0, 8, 16, 32, 64) */
+    int64_t dim_rows;                  /* rows of the dimension */
+    int64_t entries;                   /* rows passing the filter */
+    int64_t kmin, kmax;                /* key range among the passing rows (0,0 if none) */
+    int64_t pay_min[SJQ_MAX_PAYLOADS]; /* payload i is stored as (value - pay_min[i]) in pay_bits[i] bits */
+    int64_t pay_max[SJQ_MAX_PAYLOADS];
+    int32_t pay_bits[SJQ_MAX_PAYLOADS];
+    int64_t slots;      /* direct: kmax-kmin+1; hash: power-of-two slot count */
+    size_t table_bytes; /* device bytes sjq_build_dim needs at table_mem */
+} sjq_dim_layout;
+
+typedef struct sjq_table sjq_table; /* opaque host handle */
+
+/*
+ * Scan the filtered dimension once (key range, passing-row count, payload
+ * ranges) and choose the table shape.  Enqueues one kernel on `stream`, copies
+ * 64 bytes back and SYNCHRONISES the stream before returning.
+ *   cols/ncols      dimension columns (device), all of equal length
+ *   preds/npreds    conjunction over those columns (npreds <= 16)
+ *   key_col         index of the key column
+ *   payload_cols    indices of up to SJQ_MAX_PAYLOADS payload columns
+ *   scratch_dev     device scratch of SJQ_PLAN_SCRATCH_BYTES bytes
+ * Errors: INVALID_ARG, ALIGN, UNSUPPORTED (payload ranges too wide to pack
+ * into 64 bits), CUDA.
+ */
+sjq_status sjq_dim_plan(const sjq_col *cols, int ncols, const sjq_pred *preds, int npreds, int key_col,
+                        const int *payload_cols, int npayload, const sjq_build_opts *opts, void *scratch_dev,
+                        void *stream, sjq_dim_layout *layout);
+
+/*
+ * Build the table described by `layout` into caller memory `table_mem`
+ * (>= layout->table_bytes, else BUFFER_SMALL) and return a handle.  Enqueues
+ * a fill, the build kernel and a verification kernel; does not synchronise.
+ * Direct tables are written by race-free direct stores indexed by key
+ * (Section 3.3); hash tables by atomicCAS on the key word with a bounded
+ * linear probe.  Keys must be unique among the passing rows: a repeated key
+ * sets SJQ_ERR_DUP_KEY in *status_dev.  Zero passing rows is valid (every
+ * probe then misses).  *status_dev is NOT cleared by this call.
+ */
+sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pred *preds, int npreds, int key_col,
+                         const int *payload_cols, int npayload, const sjq_dim_layout *layout, void *table_mem,
+                         size_t table_bytes, int32_t *status_dev, void *stream, sjq_table **table);
+
+/* Copy of the layout the table was built with. */
+sjq_status sjq_table_info(const sjq_table *table, sjq_dim_layout *layout);
+
+/* Frees the host handle only (the device memory belongs to the caller). */
+void sjq_table_destroy(sjq_table *table);
+
+/* ------------------------------------------------------------------ */
+/* The fused run. */
+
+typedef struct sjq_join {
+    int32_t fk_col;         /* fact column holding the foreign key (same dtype as the table's key) */
+    const sjq_table *table; /* table probed with it */
+} sjq_join;
+
+enum { SJQ_SCALAR = 0, SJQ_DENSE = 1, SJQ_HASHED = 2 };
+
+typedef struct sjq_result_spec {
+    int32_t mode;
+    int64_t num_groups; /* DENSE: keys must lie in [0, num_groups) */
+    int64_t capacity;   /* HASHED: maximum number of distinct groups */
+} sjq_result_spec;
+
+/* Device buffers receiving the result.
+ *   SCALAR: sums[0], counts[0].
+ *   DENSE : sums[num_groups], counts[num_groups] (absent groups are zero).
+ *   HASHED: keys/sums/counts[capacity] hold *n_groups entries in no particular
+ *           order; `workspace` is the group hash table (scratch).
+ * `counts` may be NULL when want_count is 0 (SCALAR and DENSE only).
+ * `n_groups` is required for HASHED.  `status` is always required. */
+typedef struct sjq_result {
+    int64_t *sums;
+    int64_t *counts;
+    int64_t *keys;
+    int64_t *n_groups;
+    int32_t *status;
+    void *workspace;
+    size_t workspace_bytes;
+} sjq_result;
+
+#define SJQ_MAX_PREDS 16
+#define SJQ_MAX_JOINS 8
+
+/* Tuning and ablation switches; a zeroed struct (or NULL) means defaults. */
+typedef struct sjq_run_opts {
+    int32_t block_threads; /* 0 = default; else 128..1024, multiple of 32 */
+    int32_t ctas_per_sm;   /* 0 = as many as fit */
+    int32_t eager_loads;   /* 1 = load every column for every row (ablation of lazy loading) */
+    int32_t agg_path;      /* 0 auto, 1 shared-memory privatised table, 2 global atomics (DENSE) */
+    int32_t smem_tables;   /* 0 auto, 1 never copy small direct tables into shared memory */
+    int32_t compaction;    /* 0 auto, 1 never, 2 always compact survivors before the sparse tail */
+    int32_t accumulate;    /* 1 = add into the result buffers instead of clearing them first */
+    int32_t norder;        /* 0 = library chooses the evaluation order */
+    int32_t order[SJQ_MAX_PREDS + SJQ_MAX_JOINS]; /* entry < npreds: predicate index; else npreds + join index */
+    int32_t reserved[8];
+} sjq_run_opts;
+
+/* What the planner decided for a run (for reports and tests). */
+typedef struct sjq_run_info {
+    int32_t nstages;
+    int32_t order[SJQ_MAX_PREDS + SJQ_MAX_JOINS + 8]; /* as in sjq_run_opts.order; -1 = plain column load */
+    int32_t stage_in_smem[SJQ_MAX_PREDS + SJQ_MAX_JOINS + 8];
+    int32_t first_sparse_stage; /* stages >= this run on compacted survivors; nstages = none */
+    int32_t agg_path;           /* 0 scalar registers, 1 shared-memory table, 2 global atomics, 3 global hash */
+    int32_t grid, block;
+    int32_t smem_bytes;
+    int32_t kernel_launches; /* kernels enqueued by the call */
+} sjq_run_info;
+
+/* Device bytes needed at sjq_result.workspace for `spec` (0 unless HASHED). */
+sjq_status sjq_run_workspace_bytes(const sjq_result_spec *spec, size_t *bytes);
+
+/*
+ * One fused pass over the fact table.
+ *   fact/nfact   fact columns (device), equal length N >= 0 (N need not be a
+ *                multiple of anything)
+ *   preds        conjunction over fact columns (npreds <= SJQ_MAX_PREDS)
+ *   joins        inner equi-joins (njoins <= SJQ_MAX_JOINS): a row survives
+ *                iff every fk finds its key; a key outside a direct table's
+ *                range is a miss, never an out-of-bounds access
+ *   key          group key expression (NULL iff spec->mode == SJQ_SCALAR)
+ *   agg          value summed per group
+ *   out          result buffers; cleared by this call unless opts->accumulate
+ *   info         optional: receives the plan that was used
+ * Enqueues a clear kernel, the fused kernel and (HASHED) a compaction kernel
+ * on `stream`; does not synchronise.  Host-detected errors are returned;
+ * device-detected errors (GROUP_RANGE, GROUP_OVERFLOW) go to *out->status.
+ */
+sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *preds, int npreds, const sjq_join *joins,
+                   int njoins, const sjq_key_expr *key, const sjq_agg_expr *agg, const sjq_result_spec *spec,
+                   const sjq_result *out, const sjq_run_opts *opts, void *stream, sjq_run_info *info);
+
+const char *sjq_strerror(sjq_status status);
+const char *sjq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SJQ_H */

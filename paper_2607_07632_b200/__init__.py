@@ -1,0 +1,3 @@
+"""sjq: fused star-join query pipeline for B200 (thin binding over libsjq.so)."""
+from .sjq import (Result, SjqError, Table, build_dim, lib, run, run_workload, build_workload_tables,  # noqa: F401
+                  strerror, version, RunOpts)

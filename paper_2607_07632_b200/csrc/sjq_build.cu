@@ -1,0 +1,598 @@
+// Dimension-table planning and build kernels.
+//
+// Section 3.3 of the paper: dense primary keys allow a directly indexed map
+// whose build is a race-free direct store and whose probe is one load; the
+// filter and the gathered attribute are fused into one narrow code per key
+// with a reserved all-ones sentinel for "filtered out".  Sparse keys fall back
+// to an open-addressing table populated with atomicCAS.  Section 4.3.1: the
+// key range is verified at run time and the packed or unpacked form chosen.
+#include <new>
+
+#include "sjq_internal.h"
+
+namespace sjq {
+
+namespace {
+
+constexpr int kMaxDimCols = 32;
+
+struct DimParams {
+    const void *col[kMaxDimCols];
+    uint8_t is64[kMaxDimCols];
+    DPred preds[SJQ_MAX_PREDS];
+    int32_t npreds;
+    int32_t key_col;
+    int32_t pay_col[SJQ_MAX_PAYLOADS];
+    int32_t npayload;
+    int64_t n;
+};
+
+__device__ inline bool dim_row_passes(const DimParams &P, int64_t r)
+{
+    bool ok = true;
+    for (int k = 0; k < P.npreds && ok; ++k) {
+        const DPred &d = P.preds[k];
+        if (d.is64) ok = pred_eval<int64_t>(d, static_cast<const int64_t *>(P.col[d.col])[r]);
+        else ok = pred_eval<int32_t>(d, static_cast<const int32_t *>(P.col[d.col])[r]);
+    }
+    return ok;
+}
+
+__device__ inline int64_t warp_min(int64_t v)
+{
+    for (int o = 16; o > 0; o >>= 1) {
+        int64_t t = __shfl_xor_sync(0xffffffffu, v, o);
+        v = t < v ? t : v;
+    }
+    return v;
+}
+__device__ inline int64_t warp_max(int64_t v)
+{
+    for (int o = 16; o > 0; o >>= 1) {
+        int64_t t = __shfl_xor_sync(0xffffffffu, v, o);
+        v = t > v ? t : v;
+    }
+    return v;
+}
+__device__ inline int64_t warp_sum(int64_t v)
+{
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// scratch: [0] kmin [1] kmax [2] count [3] p0min [4] p0max [5] p1min [6] p1max
+__global__ void plan_init_kernel(int64_t *s)
+{
+    if (threadIdx.x < 8) {
+        int64_t v = 0;
+        if (threadIdx.x == 0 || threadIdx.x == 3 || threadIdx.x == 5) v = INT64_MAX;
+        if (threadIdx.x == 1 || threadIdx.x == 4 || threadIdx.x == 6) v = INT64_MIN;
+        s[threadIdx.x] = v;
+    }
+}
+
+__global__ void __launch_bounds__(256) plan_scan_kernel(const __grid_constant__ DimParams P, int64_t *scratch)
+{
+    int64_t kmin = INT64_MAX, kmax = INT64_MIN, cnt = 0;
+    int64_t pmin[SJQ_MAX_PAYLOADS] = {INT64_MAX, INT64_MAX}, pmax[SJQ_MAX_PAYLOADS] = {INT64_MIN, INT64_MIN};
+    const int64_t stride = (int64_t)blockDim.x * gridDim.x;
+    for (int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; r < P.n; r += stride) {
+        if (!dim_row_passes(P, r)) continue;
+        int64_t k = load_cell(P.col[P.key_col], P.is64[P.key_col], r);
+        kmin = k < kmin ? k : kmin;
+        kmax = k > kmax ? k : kmax;
+        ++cnt;
+        for (int i = 0; i < P.npayload; ++i) {
+            int64_t v = load_cell(P.col[P.pay_col[i]], P.is64[P.pay_col[i]], r);
+            pmin[i] = v < pmin[i] ? v : pmin[i];
+            pmax[i] = v > pmax[i] ? v : pmax[i];
+        }
+    }
+    kmin = warp_min(kmin);
+    kmax = warp_max(kmax);
+    cnt = warp_sum(cnt);
+    for (int i = 0; i < SJQ_MAX_PAYLOADS; ++i) {
+        pmin[i] = warp_min(pmin[i]);
+        pmax[i] = warp_max(pmax[i]);
+    }
+    if ((threadIdx.x & 31) == 0 && cnt > 0) {
+        atomicMin((long long *)&scratch[0], (long long)kmin);
+        atomicMax((long long *)&scratch[1], (long long)kmax);
+        atomicAdd((unsigned long long *)&scratch[2], (unsigned long long)cnt);
+        for (int i = 0; i < P.npayload; ++i) {
+            atomicMin((long long *)&scratch[3 + 2 * i], (long long)pmin[i]);
+            atomicMax((long long *)&scratch[4 + 2 * i], (long long)pmax[i]);
+        }
+    }
+}
+
+struct BuildParams {
+    DimParams dim;
+    int32_t kind;
+    int32_t code_bits;
+    int64_t kmin;
+    uint64_t span;  // direct
+    uint64_t hmask; // hash: slots - 1
+    int64_t pay_min[SJQ_MAX_PAYLOADS], pay_max[SJQ_MAX_PAYLOADS];
+    int32_t pay_bits[SJQ_MAX_PAYLOADS];
+    void *slots;
+    void *codes;
+    unsigned long long *header; // [0] rows inserted, [1] slots occupied
+    int32_t *status;
+};
+
+template <typename W>
+__global__ void fill_kernel(W *p, W v, size_t n)
+{
+    const size_t stride = (size_t)blockDim.x * gridDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) p[i] = v;
+}
+
+__device__ inline bool pack_code(const BuildParams &B, int64_t r, uint64_t *code)
+{
+    uint64_t c = 0;
+    int shift = 0;
+    for (int i = 0; i < B.dim.npayload; ++i) {
+        int64_t v = load_cell(B.dim.col[B.dim.pay_col[i]], B.dim.is64[B.dim.pay_col[i]], r);
+        if (v < B.pay_min[i] || v > B.pay_max[i]) return false;
+        c |= ((uint64_t)v - (uint64_t)B.pay_min[i]) << shift;
+        shift += B.pay_bits[i];
+    }
+    *code = c;
+    return true;
+}
+
+__device__ inline void store_code(void *codes, int bits, uint64_t idx, uint64_t c)
+{
+    switch (bits) {
+    case 8: static_cast<uint8_t *>(codes)[idx] = (uint8_t)c; break;
+    case 16: static_cast<uint16_t *>(codes)[idx] = (uint16_t)c; break;
+    case 32: static_cast<uint32_t *>(codes)[idx] = (uint32_t)c; break;
+    case 64: static_cast<uint64_t *>(codes)[idx] = c; break;
+    default: break;
+    }
+}
+
+__global__ void __launch_bounds__(256) build_kernel(const __grid_constant__ BuildParams B)
+{
+    const DimParams &P = B.dim;
+    const int64_t stride = (int64_t)blockDim.x * gridDim.x;
+    unsigned long long inserted = 0;
+    for (int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; r < P.n; r += stride) {
+        if (!dim_row_passes(P, r)) continue;
+        const int64_t k = load_cell(P.col[P.key_col], P.is64[P.key_col], r);
+        uint64_t code = 0;
+        if (!pack_code(B, r, &code)) {
+            set_status(B.status, SJQ_ERR_LAYOUT_MISMATCH);
+            continue;
+        }
+        ++inserted;
+        if (B.kind <= SJQ_TABLE_DIRECT_U64) {
+            const uint64_t idx = (uint64_t)k - (uint64_t)B.kmin;
+            if (idx >= B.span) {
+                set_status(B.status, SJQ_ERR_LAYOUT_MISMATCH);
+                continue;
+            }
+            if (B.kind == SJQ_TABLE_DIRECT_BITMAP)
+                atomicOr(static_cast<unsigned int *>(B.slots) + (idx >> 5), 1u << (idx & 31));
+            else store_code(B.slots, B.code_bits, idx, code); // race-free: keys are unique
+        } else if (B.kind == SJQ_TABLE_HASH_I64) {
+            if (k == kEmptyKey64) {
+                set_status(B.status, SJQ_ERR_RESERVED_KEY);
+                continue;
+            }
+            unsigned long long *keys = static_cast<unsigned long long *>(B.slots);
+            uint64_t slot = hash64((uint64_t)k) & B.hmask;
+            bool done = false;
+            for (uint64_t it = 0; it <= B.hmask; ++it) {
+                unsigned long long old = atomicCAS(&keys[slot], (unsigned long long)kEmptyKey64, (unsigned long long)k);
+                if (old == (unsigned long long)kEmptyKey64) {
+                    store_code(B.codes, B.code_bits, slot, code);
+                    done = true;
+                    break;
+                }
+                if (old == (unsigned long long)k) {
+                    set_status(B.status, SJQ_ERR_DUP_KEY);
+                    done = true;
+                    break;
+                }
+                slot = (slot + 1) & B.hmask;
+            }
+            if (!done) set_status(B.status, SJQ_ERR_TABLE_FULL);
+        } else { // HASH_I32
+            const int32_t k32 = (int32_t)k;
+            if (k32 == kEmptyKey32) {
+                set_status(B.status, SJQ_ERR_RESERVED_KEY);
+                continue;
+            }
+            int *keys = static_cast<int *>(B.slots);
+            uint64_t slot = hash64((uint64_t)(int64_t)k32) & B.hmask;
+            bool done = false;
+            for (uint64_t it = 0; it <= B.hmask; ++it) {
+                int old = atomicCAS(&keys[slot], kEmptyKey32, k32);
+                if (old == kEmptyKey32) {
+                    store_code(B.codes, B.code_bits, slot, code);
+                    done = true;
+                    break;
+                }
+                if (old == k32) {
+                    set_status(B.status, SJQ_ERR_DUP_KEY);
+                    done = true;
+                    break;
+                }
+                slot = (slot + 1) & B.hmask;
+            }
+            if (!done) set_status(B.status, SJQ_ERR_TABLE_FULL);
+        }
+    }
+    inserted = (unsigned long long)warp_sum((int64_t)inserted);
+    if ((threadIdx.x & 31) == 0 && inserted) atomicAdd(&B.header[0], inserted);
+}
+
+// Count occupied slots of a direct table; a repeated key leaves fewer
+// occupied slots than inserted rows.
+__global__ void __launch_bounds__(256) direct_count_kernel(const __grid_constant__ BuildParams B)
+{
+    const uint64_t stride = (uint64_t)blockDim.x * gridDim.x;
+    unsigned long long occ = 0;
+    if (B.kind == SJQ_TABLE_DIRECT_BITMAP) {
+        const uint64_t words = (B.span + 31) >> 5;
+        const unsigned int *w = static_cast<const unsigned int *>(B.slots);
+        for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < words; i += stride) occ += __popc(w[i]);
+    } else {
+        for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < B.span; i += stride) {
+            bool set;
+            switch (B.code_bits) {
+            case 8: set = static_cast<const uint8_t *>(B.slots)[i] != 0xFFu; break;
+            case 16: set = static_cast<const uint16_t *>(B.slots)[i] != 0xFFFFu; break;
+            case 32: set = static_cast<const uint32_t *>(B.slots)[i] != 0xFFFFFFFFu; break;
+            default: set = static_cast<const uint64_t *>(B.slots)[i] != ~0ULL; break;
+            }
+            occ += set;
+        }
+    }
+    occ = (unsigned long long)warp_sum((int64_t)occ);
+    if ((threadIdx.x & 31) == 0 && occ) atomicAdd(&B.header[1], occ);
+}
+
+__global__ void direct_verify_kernel(const unsigned long long *header, int32_t *status)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0 && header[0] != header[1]) set_status(status, SJQ_ERR_DUP_KEY);
+}
+
+int bits_for(uint64_t range)
+{
+    int b = 0;
+    while (b < 64 && (range >> b) != 0) ++b;
+    return b;
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+sjq_status fill_dim_params(const sjq_col *cols, int ncols, const sjq_pred *preds, int npreds, int key_col,
+                           const int *payload_cols, int npayload, DimParams *P)
+{
+    if (!cols || ncols <= 0 || ncols > kMaxDimCols || npreds < 0 || npreds > SJQ_MAX_PREDS || (npreds && !preds) ||
+        key_col < 0 || key_col >= ncols || npayload < 0 || npayload > SJQ_MAX_PAYLOADS || (npayload && !payload_cols))
+        return SJQ_ERR_INVALID_ARG;
+    const int64_t n = cols[key_col].n;
+    if (n < 0) return SJQ_ERR_INVALID_ARG;
+    for (int c = 0; c < ncols; ++c) {
+        if (cols[c].n != n || (cols[c].dtype != SJQ_I32 && cols[c].dtype != SJQ_I64)) return SJQ_ERR_INVALID_ARG;
+        if (n > 0 && !cols[c].data) return SJQ_ERR_INVALID_ARG;
+        if (!aligned16(cols[c].data)) return SJQ_ERR_ALIGN;
+        P->col[c] = cols[c].data;
+        P->is64[c] = (uint8_t)cols[c].dtype;
+    }
+    for (int k = 0; k < npreds; ++k) {
+        if (preds[k].col < 0 || preds[k].col >= ncols) return SJQ_ERR_INVALID_ARG;
+        if (!canon_pred(preds[k], cols[preds[k].col].dtype, &P->preds[k])) return SJQ_ERR_INVALID_ARG;
+    }
+    for (int i = 0; i < npayload; ++i) {
+        if (payload_cols[i] < 0 || payload_cols[i] >= ncols) return SJQ_ERR_INVALID_ARG;
+        P->pay_col[i] = payload_cols[i];
+    }
+    P->npreds = npreds;
+    P->key_col = key_col;
+    P->npayload = npayload;
+    P->n = n;
+    return SJQ_OK;
+}
+
+int grid_for(int64_t n, int sm_count)
+{
+    int64_t blocks = (n + 255) / 256;
+    int64_t cap = (int64_t)sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    return blocks < 1 ? 1 : (int)blocks;
+}
+
+} // namespace
+
+bool canon_pred(const sjq_pred &p, int dtype, DPred *d)
+{
+    *d = DPred{};
+    d->col = p.col;
+    d->is64 = (uint8_t)(dtype == SJQ_I64);
+    bool empty = false;
+    switch (p.op) {
+    case SJQ_EQ: d->lo = d->hi = p.lo; break;
+    case SJQ_NE: d->lo = d->hi = p.lo; d->neg = 1; break;
+    case SJQ_LT:
+        if (p.lo == INT64_MIN) empty = true;
+        else { d->lo = INT64_MIN; d->hi = p.lo - 1; }
+        break;
+    case SJQ_LE: d->lo = INT64_MIN; d->hi = p.lo; break;
+    case SJQ_GT:
+        if (p.lo == INT64_MAX) empty = true;
+        else { d->lo = p.lo + 1; d->hi = INT64_MAX; }
+        break;
+    case SJQ_GE: d->lo = p.lo; d->hi = INT64_MAX; break;
+    case SJQ_BETWEEN: d->lo = p.lo; d->hi = p.hi; break;
+    case SJQ_IN:
+        if (p.nset < 0 || p.nset > SJQ_MAX_IN_SET || (p.nset && !p.set)) return false;
+        if (p.nset == 0) empty = true;
+        for (int k = 0; k < p.nset; ++k) d->set[k] = p.set[k];
+        d->nset = (uint8_t)p.nset;
+        break;
+    default: return false;
+    }
+    if (empty || d->lo > d->hi) {
+        d->lo = 1;
+        d->hi = 0;
+    }
+    // int32 view of the range
+    if (d->lo > d->hi || d->lo > INT32_MAX || d->hi < INT32_MIN) {
+        d->never = 1;
+        d->lo32 = 1;
+        d->hi32 = 0;
+    } else {
+        d->lo32 = d->lo < INT32_MIN ? INT32_MIN : (int32_t)d->lo;
+        d->hi32 = d->hi > INT32_MAX ? INT32_MAX : (int32_t)d->hi;
+    }
+    return true;
+}
+
+sjq_status device_info(DeviceInfo *out)
+{
+    static thread_local DeviceInfo cache[64];
+    static thread_local bool have[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SJQ_ERR_CUDA;
+    }
+    if (dev >= 0 && dev < 64 && have[dev]) {
+        *out = cache[dev];
+        return SJQ_OK;
+    }
+    DeviceInfo d{};
+    d.device = dev;
+    if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&d.l2_bytes, cudaDevAttrL2CacheSize, dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SJQ_ERR_CUDA;
+    }
+    if (dev >= 0 && dev < 64) {
+        cache[dev] = d;
+        have[dev] = true;
+    }
+    *out = d;
+    return SJQ_OK;
+}
+
+} // namespace sjq
+
+using namespace sjq;
+
+extern "C" sjq_status sjq_dim_plan(const sjq_col *cols, int ncols, const sjq_pred *preds, int npreds, int key_col,
+                                   const int *payload_cols, int npayload, const sjq_build_opts *opts,
+                                   void *scratch_dev, void *stream_, sjq_dim_layout *layout)
+{
+    if (!layout || !scratch_dev) return SJQ_ERR_INVALID_ARG;
+    if (!aligned16(scratch_dev)) return SJQ_ERR_ALIGN;
+    DimParams P{};
+    sjq_status st = fill_dim_params(cols, ncols, preds, npreds, key_col, payload_cols, npayload, &P);
+    if (st != SJQ_OK) return st;
+    DeviceInfo dev;
+    if ((st = device_info(&dev)) != SJQ_OK) return st;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    int64_t *scratch = static_cast<int64_t *>(scratch_dev);
+    plan_init_kernel<<<1, 32, 0, stream>>>(scratch);
+    if (P.n > 0) plan_scan_kernel<<<grid_for(P.n, dev.sm_count), 256, 0, stream>>>(P, scratch);
+    int64_t h[8];
+    if (cudaGetLastError() != cudaSuccess ||
+        cudaMemcpyAsync(h, scratch, sizeof(h), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SJQ_ERR_CUDA;
+    }
+
+    sjq_dim_layout L{};
+    L.key_dtype = cols[key_col].dtype;
+    L.npayload = npayload;
+    L.dim_rows = P.n;
+    L.entries = h[2];
+    if (L.entries > 0) {
+        L.kmin = h[0];
+        L.kmax = h[1];
+    }
+    uint64_t maxcode = 0;
+    int total_bits = 0;
+    for (int i = 0; i < npayload; ++i) {
+        L.pay_min[i] = L.entries > 0 ? h[3 + 2 * i] : 0;
+        L.pay_max[i] = L.entries > 0 ? h[4 + 2 * i] : 0;
+        const uint64_t range = (uint64_t)L.pay_max[i] - (uint64_t)L.pay_min[i];
+        L.pay_bits[i] = bits_for(range);
+        if (total_bits + L.pay_bits[i] > 63) return SJQ_ERR_UNSUPPORTED;
+        maxcode |= range << total_bits;
+        total_bits += L.pay_bits[i];
+    }
+    int code_bits = 0;
+    if (npayload > 0) {
+        if (maxcode < 0xFFu) code_bits = 8;
+        else if (maxcode < 0xFFFFu) code_bits = 16;
+        else if (maxcode < 0xFFFFFFFFu) code_bits = 32;
+        else code_bits = 64;
+    }
+    const int force = opts ? opts->force_kind : SJQ_TABLE_AUTO;
+    if (force != SJQ_TABLE_AUTO && force != SJQ_TABLE_FORCE_DIRECT && force != SJQ_TABLE_FORCE_HASH)
+        return SJQ_ERR_INVALID_ARG;
+    const int64_t max_direct = (opts && opts->max_direct_bytes > 0) ? opts->max_direct_bytes : (int64_t)64 << 20;
+    const int load_pct = (opts && opts->hash_load_pct > 0) ? opts->hash_load_pct : 50;
+    if (load_pct > 90) return SJQ_ERR_INVALID_ARG;
+
+    const uint64_t span_m1 = (uint64_t)L.kmax - (uint64_t)L.kmin; // span - 1, no overflow
+    bool direct_ok = span_m1 < ((uint64_t)1 << 40);
+    size_t direct_bytes = 0;
+    if (direct_ok) {
+        const uint64_t span = span_m1 + 1;
+        direct_bytes = npayload == 0 ? (size_t)((span + 31) / 32 * 4) : (size_t)(span * (uint64_t)(code_bits / 8));
+        direct_bytes = align_up(direct_bytes, 16);
+    }
+    bool use_direct;
+    if (force == SJQ_TABLE_FORCE_DIRECT) {
+        if (!direct_ok || direct_bytes > ((size_t)1 << 36)) return SJQ_ERR_UNSUPPORTED;
+        use_direct = true;
+    } else if (force == SJQ_TABLE_FORCE_HASH) {
+        use_direct = false;
+    } else {
+        use_direct = direct_ok && (int64_t)direct_bytes <= max_direct;
+    }
+    if (use_direct) {
+        L.slots = (int64_t)(span_m1 + 1);
+        L.code_bits = code_bits;
+        L.kind = npayload == 0 ? SJQ_TABLE_DIRECT_BITMAP
+                 : code_bits == 8 ? SJQ_TABLE_DIRECT_U8
+                 : code_bits == 16 ? SJQ_TABLE_DIRECT_U16
+                 : code_bits == 32 ? SJQ_TABLE_DIRECT_U32
+                                   : SJQ_TABLE_DIRECT_U64;
+        L.table_bytes = kTableHeaderBytes + align_up(direct_bytes, 256);
+    } else {
+        uint64_t want = ((uint64_t)L.entries * 100u + (uint64_t)load_pct - 1) / (uint64_t)load_pct;
+        uint64_t slots = 16;
+        while (slots < want) slots <<= 1;
+        L.slots = (int64_t)slots;
+        L.kind = L.key_dtype == SJQ_I64 ? SJQ_TABLE_HASH_I64 : SJQ_TABLE_HASH_I32;
+        L.code_bits = npayload == 0 ? 0 : (code_bits <= 32 ? 32 : 64);
+        const size_t kb = (size_t)slots * (L.key_dtype == SJQ_I64 ? 8 : 4);
+        const size_t cb = (size_t)slots * (size_t)(L.code_bits / 8);
+        L.table_bytes = kTableHeaderBytes + align_up(kb, 256) + align_up(cb, 256);
+    }
+    *layout = L;
+    return SJQ_OK;
+}
+
+extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pred *preds, int npreds, int key_col,
+                                    const int *payload_cols, int npayload, const sjq_dim_layout *layout,
+                                    void *table_mem, size_t table_bytes, int32_t *status_dev, void *stream_,
+                                    sjq_table **table)
+{
+    if (!layout || !table_mem || !status_dev || !table) return SJQ_ERR_INVALID_ARG;
+    if (!aligned16(table_mem)) return SJQ_ERR_ALIGN;
+    BuildParams B{};
+    sjq_status st = fill_dim_params(cols, ncols, preds, npreds, key_col, payload_cols, npayload, &B.dim);
+    if (st != SJQ_OK) return st;
+    const sjq_dim_layout &L = *layout;
+    if (L.kind < SJQ_TABLE_DIRECT_BITMAP || L.kind > SJQ_TABLE_HASH_I64 || L.npayload != npayload ||
+        L.key_dtype != cols[key_col].dtype || L.slots <= 0 || L.dim_rows != B.dim.n)
+        return SJQ_ERR_INVALID_ARG;
+    if (table_bytes < L.table_bytes) return SJQ_ERR_BUFFER_SMALL;
+    DeviceInfo dev;
+    if ((st = device_info(&dev)) != SJQ_OK) return st;
+    cudaStream_t stream = (cudaStream_t)stream_;
+
+    sjq_table *T = new (std::nothrow) sjq_table();
+    if (!T) return SJQ_ERR_INVALID_ARG;
+    T->layout = L;
+    T->base = static_cast<char *>(table_mem);
+    T->slots = T->base + kTableHeaderBytes;
+    T->codes = nullptr;
+    T->magic = kTableMagic;
+
+    B.kind = L.kind;
+    B.code_bits = L.code_bits;
+    B.kmin = L.kmin;
+    B.span = (uint64_t)L.slots;
+    B.hmask = (uint64_t)L.slots - 1;
+    for (int i = 0; i < SJQ_MAX_PAYLOADS; ++i) {
+        B.pay_min[i] = L.pay_min[i];
+        B.pay_max[i] = L.pay_max[i];
+        B.pay_bits[i] = L.pay_bits[i];
+    }
+    B.header = reinterpret_cast<unsigned long long *>(T->base);
+    B.status = status_dev;
+    B.slots = T->slots;
+
+    bool ok = cudaMemsetAsync(T->base, 0, kTableHeaderBytes, stream) == cudaSuccess;
+    const bool direct = L.kind <= SJQ_TABLE_DIRECT_U64;
+    if (direct) {
+        const uint64_t span = (uint64_t)L.slots;
+        size_t bytes = L.kind == SJQ_TABLE_DIRECT_BITMAP ? (size_t)((span + 31) / 32 * 4)
+                                                         : (size_t)(span * (uint64_t)(L.code_bits / 8));
+        bytes = align_up(bytes, 16);
+        T->slots_bytes = bytes;
+        ok = ok && cudaMemsetAsync(T->slots, L.kind == SJQ_TABLE_DIRECT_BITMAP ? 0 : 0xFF, bytes, stream) == cudaSuccess;
+    } else {
+        const size_t kb = (size_t)L.slots * (L.key_dtype == SJQ_I64 ? 8 : 4);
+        T->slots_bytes = kb;
+        if (L.code_bits) T->codes = T->slots + align_up(kb, 256);
+        B.codes = T->codes;
+        const int g = grid_for(L.slots, dev.sm_count);
+        if (L.key_dtype == SJQ_I64)
+            fill_kernel<int64_t><<<g, 256, 0, stream>>>(reinterpret_cast<int64_t *>(T->slots), kEmptyKey64, (size_t)L.slots);
+        else
+            fill_kernel<int32_t><<<g, 256, 0, stream>>>(reinterpret_cast<int32_t *>(T->slots), kEmptyKey32, (size_t)L.slots);
+        if (L.code_bits)
+            ok = ok && cudaMemsetAsync(T->codes, 0, (size_t)L.slots * (size_t)(L.code_bits / 8), stream) == cudaSuccess;
+    }
+    if (ok && B.dim.n > 0) build_kernel<<<grid_for(B.dim.n, dev.sm_count), 256, 0, stream>>>(B);
+    if (ok && direct) {
+        direct_count_kernel<<<grid_for(L.slots, dev.sm_count), 256, 0, stream>>>(B);
+        direct_verify_kernel<<<1, 32, 0, stream>>>(B.header, status_dev);
+    }
+    if (!ok || cudaGetLastError() != cudaSuccess) {
+        (void)cudaGetLastError();
+        delete T;
+        return SJQ_ERR_CUDA;
+    }
+    *table = T;
+    return SJQ_OK;
+}
+
+extern "C" sjq_status sjq_table_info(const sjq_table *table, sjq_dim_layout *layout)
+{
+    if (!table || table->magic != kTableMagic || !layout) return SJQ_ERR_INVALID_ARG;
+    *layout = table->layout;
+    return SJQ_OK;
+}
+
+extern "C" void sjq_table_destroy(sjq_table *table)
+{
+    if (table && table->magic == kTableMagic) {
+        table->magic = 0;
+        delete table;
+    }
+}
+
+extern "C" const char *sjq_strerror(sjq_status s)
+{
+    switch (s) {
+    case SJQ_OK: return "ok";
+    case SJQ_ERR_INVALID_ARG: return "invalid argument";
+    case SJQ_ERR_UNSUPPORTED: return "unsupported query or table shape";
+    case SJQ_ERR_ALIGN: return "device pointer not 16-byte aligned";
+    case SJQ_ERR_CUDA: return "CUDA runtime error (no device or launch failure)";
+    case SJQ_ERR_BUFFER_SMALL: return "caller-provided buffer too small";
+    case SJQ_ERR_DUP_KEY: return "duplicate dimension key among rows passing the filter";
+    case SJQ_ERR_TABLE_FULL: return "hash table full";
+    case SJQ_ERR_GROUP_RANGE: return "group key outside [0, num_groups)";
+    case SJQ_ERR_GROUP_OVERFLOW: return "more distinct groups than the hashed capacity";
+    case SJQ_ERR_RESERVED_KEY: return "dimension key equals the reserved empty marker";
+    case SJQ_ERR_LAYOUT_MISMATCH: return "dimension data does not match the planned layout";
+    default: return "unknown status";
+    }
+}
+
+extern "C" const char *sjq_version(void) { return "sjq 0.1 (sm_100a)"; }

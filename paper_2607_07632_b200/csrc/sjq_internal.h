@@ -1,0 +1,94 @@
+// Internal structures shared by the translation units of libsjq.
+#ifndef SJQ_INTERNAL_H
+#define SJQ_INTERNAL_H
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sjq.h"
+
+namespace sjq {
+
+// ---------------------------------------------------------------- predicates
+// Canonical form of one predicate: an inclusive range [lo, hi], optionally
+// negated, or a small set.  An empty range is encoded as lo > hi.
+struct DPred {
+    int64_t lo, hi;
+    int64_t set[SJQ_MAX_IN_SET];
+    int32_t lo32, hi32; // the same range clamped to int32 (for int32 columns)
+    int32_t col;
+    uint8_t neg;   // pass iff NOT in range
+    uint8_t nset;  // > 0: pass iff value in set[0..nset)
+    uint8_t is64;  // dtype of the column
+    uint8_t never; // range empty for this dtype: nothing passes (before negation)
+};
+
+bool canon_pred(const sjq_pred &p, int dtype, DPred *out);
+
+// ---------------------------------------------------------------- tables
+constexpr int64_t kEmptyKey64 = INT64_MIN;
+constexpr int32_t kEmptyKey32 = INT32_MIN;
+constexpr size_t kTableHeaderBytes = 256; // device-side counters at the start of table_mem
+
+} // namespace sjq
+
+struct sjq_table {
+    sjq_dim_layout layout;
+    char *base;          // table_mem
+    char *slots;         // direct: code array / bitmap words; hash: key array
+    char *codes;         // hash: code array (NULL when no payload)
+    size_t slots_bytes;  // bytes of the direct array (for shared-memory staging)
+    uint32_t magic;
+};
+
+namespace sjq {
+
+constexpr uint32_t kTableMagic = 0x534a5154u; // "SJQT"
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// murmur3-style 64-bit finaliser used for both the dimension hash tables and
+// the group hash table.
+__host__ __device__ inline uint64_t hash64(uint64_t k)
+{
+    k ^= k >> 33;
+    k *= 0xff51afd7ed558ccdULL;
+    k ^= k >> 33;
+    k *= 0xc4ceb9fe1a85ec53ULL;
+    k ^= k >> 33;
+    return k;
+}
+
+// first-error-wins store into the status word
+__device__ inline void set_status(int32_t *status, int32_t code) { atomicCAS(status, 0, code); }
+
+template <typename T>
+__device__ inline bool pred_eval(const DPred &d, T v)
+{
+    if (d.nset) {
+        bool f = false;
+        for (int k = 0; k < d.nset; ++k) f |= ((int64_t)v == d.set[k]);
+        return f;
+    }
+    bool in;
+    if (sizeof(T) == 4) in = ((int32_t)v >= d.lo32) & ((int32_t)v <= d.hi32) & !d.never;
+    else in = ((int64_t)v >= d.lo) & ((int64_t)v <= d.hi);
+    return in != (bool)d.neg;
+}
+
+__device__ inline int64_t load_cell(const void *col, int is64, int64_t i)
+{
+    return is64 ? static_cast<const int64_t *>(col)[i] : (int64_t) static_cast<const int32_t *>(col)[i];
+}
+
+struct DeviceInfo {
+    int device;
+    int sm_count;
+    int max_smem_optin;
+    int l2_bytes;
+};
+sjq_status device_info(DeviceInfo *out);
+
+} // namespace sjq
+
+#endif

@@ -1,0 +1,395 @@
+// Host side of sjq_run: validation, the plan (evaluation order, which tables
+// are staged in shared memory, which aggregation path), and the launches.
+//
+// The order rule follows the paper's observation that bytes moved, not
+// arithmetic, decide the run time (Section 3.2): evaluate first what removes
+// the most rows per byte read, so that later columns are loaded for few rows.
+// The aggregation rule follows Section 3.3: privatise the group table in
+// shared memory only when it fits and many survivors contend on it; keep the
+// global table when few rows survive or the groups are many.  The rows-per-
+// thread choice of Section 4.3.1 ("asymmetric batching") is the fixed four
+// rows per 128-bit load here; occupancy supplies the memory-level parallelism.
+#include <algorithm>
+#include <cstring>
+#include <vector>
+
+#include "sjq_run.cuh"
+
+namespace sjq {
+
+sjq_status fused_occupancy(int agg, bool mul, int block, size_t smem, int *ctas_per_sm);
+sjq_status fused_launch(int agg, bool mul, int grid, int block, size_t smem, const RunParams &P, cudaStream_t stream);
+sjq_status clear_launch(int64_t *sums, int64_t *counts, int64_t cells, int64_t *gkeys, int64_t gslots,
+                        int64_t *n_groups, int32_t *status, int sm_count, cudaStream_t stream);
+sjq_status compact_launch(const int64_t *gkeys, const int64_t *gsums, const int64_t *gcounts, int64_t gslots,
+                          int64_t *keys, int64_t *sums, int64_t *counts, int64_t capacity, int64_t *n_groups,
+                          int32_t *status, int sm_count, cudaStream_t stream);
+
+namespace {
+
+struct StageSpec {
+    int kind;     // ST_PRED / ST_PROBE / ST_LOAD
+    int index;    // predicate or join index (-1 for loads)
+    int col;      // fact column
+    double sel;   // estimated fraction of rows passing
+    double cost;  // relative cost per row evaluated
+};
+
+double pred_selectivity(const sjq_pred &p)
+{
+    switch (p.op) {
+    case SJQ_EQ: return 0.1;
+    case SJQ_NE: return 0.9;
+    case SJQ_IN: return std::min(0.5, 0.1 * std::max(1, p.nset));
+    case SJQ_BETWEEN: return 0.25;
+    default: return 0.4;
+    }
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+uint64_t hashed_slots(int64_t capacity)
+{
+    uint64_t want = (uint64_t)std::max<int64_t>(capacity, 8) * 2;
+    uint64_t slots = 16;
+    while (slots < want) slots <<= 1;
+    return slots;
+}
+
+bool valid_term(const sjq_term &t, int nfact, const sjq_join *joins, int njoins)
+{
+    if (t.src == SJQ_SRC_FACT) return t.a >= 0 && t.a < nfact;
+    if (t.src == SJQ_SRC_PAYLOAD)
+        return t.a >= 0 && t.a < njoins && t.b >= 0 && t.b < joins[t.a].table->layout.npayload;
+    return false;
+}
+
+} // namespace
+} // namespace sjq
+
+using namespace sjq;
+
+extern "C" sjq_status sjq_run_workspace_bytes(const sjq_result_spec *spec, size_t *bytes)
+{
+    if (!spec || !bytes) return SJQ_ERR_INVALID_ARG;
+    *bytes = 0;
+    if (spec->mode == SJQ_HASHED) {
+        if (spec->capacity <= 0) return SJQ_ERR_INVALID_ARG;
+        *bytes = align_up((size_t)(hashed_slots(spec->capacity) + 1) * 8, 256) * 3;
+    } else if (spec->mode != SJQ_SCALAR && spec->mode != SJQ_DENSE) {
+        return SJQ_ERR_INVALID_ARG;
+    }
+    return SJQ_OK;
+}
+
+extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *preds, int npreds,
+                              const sjq_join *joins, int njoins, const sjq_key_expr *key, const sjq_agg_expr *agg,
+                              const sjq_result_spec *spec, const sjq_result *out, const sjq_run_opts *opts_,
+                              void *stream_, sjq_run_info *info)
+{
+    // ------------------------------------------------------------ validation
+    if (!fact || nfact <= 0 || nfact > 64 || npreds < 0 || npreds > SJQ_MAX_PREDS || (npreds && !preds) ||
+        njoins < 0 || njoins > SJQ_MAX_JOINS || (njoins && !joins) || !agg || !spec || !out || !out->status ||
+        !out->sums)
+        return SJQ_ERR_INVALID_ARG;
+    sjq_run_opts opts{};
+    if (opts_) opts = *opts_;
+    const int64_t n = fact[0].n;
+    if (n < 0) return SJQ_ERR_INVALID_ARG;
+    for (int c = 0; c < nfact; ++c) {
+        if (fact[c].n != n || (fact[c].dtype != SJQ_I32 && fact[c].dtype != SJQ_I64)) return SJQ_ERR_INVALID_ARG;
+        if (n > 0 && !fact[c].data) return SJQ_ERR_INVALID_ARG;
+        if (!aligned16(fact[c].data)) return SJQ_ERR_ALIGN;
+    }
+    if (spec->mode != SJQ_SCALAR && spec->mode != SJQ_DENSE && spec->mode != SJQ_HASHED) return SJQ_ERR_INVALID_ARG;
+    if ((spec->mode == SJQ_SCALAR) != (key == nullptr)) return SJQ_ERR_INVALID_ARG;
+    if (spec->mode == SJQ_DENSE && spec->num_groups <= 0) return SJQ_ERR_INVALID_ARG;
+    if (spec->mode == SJQ_HASHED &&
+        (spec->capacity <= 0 || !out->keys || !out->counts || !out->n_groups || !out->workspace))
+        return SJQ_ERR_INVALID_ARG;
+    if (agg->want_count && !out->counts) return SJQ_ERR_INVALID_ARG;
+    if (agg->op < SJQ_AGG_COL || agg->op > SJQ_AGG_ADD) return SJQ_ERR_INVALID_ARG;
+    if (!aligned16(out->sums) || !aligned16(out->counts) || !aligned16(out->keys) || !aligned16(out->workspace) ||
+        (reinterpret_cast<uintptr_t>(out->status) & 3u) || (reinterpret_cast<uintptr_t>(out->n_groups) & 7u))
+        return SJQ_ERR_ALIGN;
+    for (int j = 0; j < njoins; ++j) {
+        const sjq_table *T = joins[j].table;
+        if (!T || T->magic != kTableMagic || joins[j].fk_col < 0 || joins[j].fk_col >= nfact)
+            return SJQ_ERR_INVALID_ARG;
+        if (fact[joins[j].fk_col].dtype != T->layout.key_dtype) return SJQ_ERR_UNSUPPORTED;
+    }
+    for (int p = 0; p < npreds; ++p)
+        if (preds[p].col < 0 || preds[p].col >= nfact) return SJQ_ERR_INVALID_ARG;
+    if (key) {
+        if (key->nterms < 0 || key->nterms > SJQ_MAX_KEY_TERMS) return SJQ_ERR_INVALID_ARG;
+        for (int t = 0; t < key->nterms; ++t)
+            if (!valid_term(key->t[t], nfact, joins, njoins)) return SJQ_ERR_INVALID_ARG;
+    }
+    if (!valid_term(agg->x, nfact, joins, njoins)) return SJQ_ERR_INVALID_ARG;
+    if (agg->op != SJQ_AGG_COL && !valid_term(agg->y, nfact, joins, njoins)) return SJQ_ERR_INVALID_ARG;
+    if (opts.block_threads && (opts.block_threads < 128 || opts.block_threads > 1024 || opts.block_threads % 32))
+        return SJQ_ERR_INVALID_ARG;
+    if (opts.norder && opts.norder != npreds + njoins) return SJQ_ERR_INVALID_ARG;
+
+    DeviceInfo dev;
+    sjq_status st = device_info(&dev);
+    if (st != SJQ_OK) return st;
+    cudaStream_t stream = (cudaStream_t)stream_;
+
+    // ------------------------------------------------------------ stage list
+    std::vector<StageSpec> specs;
+    for (int p = 0; p < npreds; ++p) {
+        const double bytes = fact[preds[p].col].dtype == SJQ_I64 ? 2.0 : 1.0;
+        specs.push_back({ST_PRED, p, preds[p].col, pred_selectivity(preds[p]), bytes});
+    }
+    for (int j = 0; j < njoins; ++j) {
+        const sjq_table *T = joins[j].table;
+        const sjq_dim_layout &L = T->layout;
+        const double bytes = L.key_dtype == SJQ_I64 ? 2.0 : 1.0;
+        double sel = L.dim_rows > 0 ? (double)L.entries / (double)L.dim_rows : 0.0;
+        const size_t tb = L.table_bytes;
+        double probe = tb <= (size_t)200 << 10 ? 0.3 : tb <= (size_t)32 << 20 ? 1.5 : 4.0;
+        specs.push_back({ST_PROBE, j, joins[j].fk_col, std::min(1.0, sel), bytes + probe});
+    }
+    const int nfilter = (int)specs.size();
+    std::vector<int> order(nfilter);
+    if (opts.norder) {
+        std::vector<char> seen(nfilter, 0);
+        for (int i = 0; i < nfilter; ++i) {
+            const int o = opts.order[i];
+            if (o < 0 || o >= nfilter || seen[o]) return SJQ_ERR_INVALID_ARG;
+            seen[o] = 1;
+            order[i] = o;
+        }
+    } else {
+        for (int i = 0; i < nfilter; ++i) order[i] = i;
+        std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+            return (1.0 - specs[a].sel) / specs[a].cost > (1.0 - specs[b].sel) / specs[b].cost;
+        });
+    }
+
+    // ------------------------------------------------------------ accumulators
+    // Every term adds mult * value to one accumulator; fold the expressions
+    // into per-source multipliers: src_mult[source][dest].
+    struct Contribution { int src, a, b, dest; int64_t mult; };
+    std::vector<Contribution> contrib;
+    auto add_term = [&](const sjq_term &t, int dest, int64_t sign) {
+        contrib.push_back({t.src, t.a, t.b, dest, (int64_t)((uint64_t)t.mult * (uint64_t)sign)});
+    };
+    if (key)
+        for (int t = 0; t < key->nterms; ++t) add_term(key->t[t], kAccKey, 1);
+    const bool mul = agg->op == SJQ_AGG_MUL;
+    add_term(agg->x, kAccX, 1);
+    if (agg->op == SJQ_AGG_MUL) add_term(agg->y, kAccY, 1);
+    if (agg->op == SJQ_AGG_SUB) add_term(agg->y, kAccX, -1);
+    if (agg->op == SJQ_AGG_ADD) add_term(agg->y, kAccX, 1);
+
+    RunParams P;
+    std::memset(&P, 0, sizeof(P));
+    P.n = n;
+    int ns = 0;
+    std::vector<int> stage_of_join(njoins, -1);
+    std::vector<int> stage_of_col(nfact, -1);
+    std::vector<int> stage_label;
+    for (int i = 0; i < nfilter; ++i) {
+        const StageSpec &sp = specs[order[i]];
+        DStage &S = P.st[ns];
+        S.kind = (uint8_t)sp.kind;
+        S.col = fact[sp.col].data;
+        S.is64 = (uint8_t)(fact[sp.col].dtype == SJQ_I64);
+        if (sp.kind == ST_PRED) {
+            if (!canon_pred(preds[sp.index], fact[sp.col].dtype, &S.pred)) return SJQ_ERR_INVALID_ARG;
+        } else {
+            const sjq_table *T = joins[sp.index].table;
+            const sjq_dim_layout &L = T->layout;
+            S.tkind = (uint8_t)L.kind;
+            S.tab = T->slots;
+            S.codes = T->codes;
+            S.kmin = L.kmin;
+            S.span = (uint64_t)L.slots;
+            S.hmask = (uint64_t)L.slots - 1;
+            S.pmin0 = L.pay_min[0];
+            S.pmin1 = L.pay_min[1];
+            S.pbits0 = (uint8_t)L.pay_bits[0];
+            S.pmask0 = L.pay_bits[0] >= 64 ? ~0ULL : ((1ULL << L.pay_bits[0]) - 1ULL);
+            S.code_bits = (uint8_t)L.code_bits;
+            S.tab_bytes = (uint32_t)std::min<size_t>(T->slots_bytes, 0xFFFFFFF0u);
+            stage_of_join[sp.index] = ns;
+        }
+        if (stage_of_col[sp.col] < 0) stage_of_col[sp.col] = ns;
+        stage_label.push_back(order[i]);
+        ++ns;
+    }
+    for (const Contribution &c : contrib) {
+        int s, src;
+        if (c.src == SJQ_SRC_FACT) {
+            if (stage_of_col[c.a] < 0) { // a column nobody filters on: plain load stage at the end
+                if (ns >= kMaxStages) return SJQ_ERR_UNSUPPORTED;
+                DStage &S = P.st[ns];
+                S.kind = ST_LOAD;
+                S.col = fact[c.a].data;
+                S.is64 = (uint8_t)(fact[c.a].dtype == SJQ_I64);
+                stage_of_col[c.a] = ns;
+                stage_label.push_back(-1);
+                ++ns;
+            }
+            s = stage_of_col[c.a];
+            src = 0;
+        } else {
+            s = stage_of_join[c.a];
+            src = 1 + c.b;
+        }
+        DStage &S = P.st[s];
+        const int slot = 3 * src + c.dest;
+        S.mult[slot] = (int64_t)((uint64_t)S.mult[slot] + (uint64_t)c.mult);
+        S.acc |= (uint16_t)(1u << slot);
+    }
+    P.nstages = ns;
+    P.first_sparse = ns;
+    P.eager = opts.eager_loads ? 1 : 0;
+    P.want_count = agg->want_count ? 1 : 0;
+    P.status = out->status;
+    if (key) {
+        P.key_offset = key->offset;
+        P.modulo = key->modulo;
+        if (key->modulo > 0 && (key->modulo & (key->modulo - 1)) == 0) P.modmask = (uint64_t)key->modulo - 1;
+        P.mod32 = key->modulo > 0 && key->modulo <= 0xFFFFFFFFLL;
+    }
+
+    // ------------------------------------------------------------ survivors estimate
+    double cum = 1.0;
+    std::vector<double> reach(ns, 1.0); // fraction of rows reaching each stage
+    for (int s = 0; s < ns; ++s) {
+        reach[s] = cum;
+        if (s < nfilter) cum *= specs[order[s]].sel;
+    }
+    const double survivors = (double)n * cum;
+
+    // ------------------------------------------------------------ aggregation path
+    int aggp;
+    size_t group_bytes = 0;
+    const int approx_grid = dev.sm_count * 2;
+    if (spec->mode == SJQ_SCALAR) {
+        aggp = AGG_SCALAR;
+    } else if (spec->mode == SJQ_HASHED) {
+        aggp = AGG_HASH;
+    } else if (spec->num_groups == 1) {
+        aggp = AGG_SCALAR; // a single group: register accumulation, key only range-checked
+        P.has_key = 1;
+    } else {
+        const size_t gb = (size_t)spec->num_groups * 8 * (P.want_count ? 2 : 1);
+        const bool fits = gb <= (size_t)64 << 10;
+        bool contended = survivors / approx_grid >= 8.0 * (double)spec->num_groups;
+        if (opts.agg_path == 1) {
+            if (!fits) return SJQ_ERR_UNSUPPORTED;
+            aggp = AGG_SMEM;
+        } else if (opts.agg_path == 2) {
+            aggp = AGG_GLOBAL;
+        } else {
+            aggp = (fits && contended) ? AGG_SMEM : AGG_GLOBAL;
+        }
+        if (aggp == AGG_SMEM) group_bytes = gb;
+    }
+    P.num_groups = spec->mode == SJQ_DENSE ? spec->num_groups : 0;
+
+    // ------------------------------------------------------------ result buffers
+    int64_t *gkeys = nullptr, *gsums = nullptr, *gcounts = nullptr;
+    uint64_t gslots = 0;
+    if (spec->mode == SJQ_HASHED) {
+        size_t need = 0;
+        sjq_run_workspace_bytes(spec, &need);
+        if (out->workspace_bytes < need) return SJQ_ERR_BUFFER_SMALL;
+        gslots = hashed_slots(spec->capacity);
+        const size_t arr = align_up((size_t)(gslots + 1) * 8, 256);
+        gkeys = reinterpret_cast<int64_t *>(static_cast<char *>(out->workspace));
+        gsums = reinterpret_cast<int64_t *>(static_cast<char *>(out->workspace) + arr);
+        gcounts = reinterpret_cast<int64_t *>(static_cast<char *>(out->workspace) + 2 * arr);
+        P.gmask = gslots - 1;
+        P.gkeys = gkeys;
+        P.sums = gsums;
+        P.counts = gcounts;
+    } else {
+        P.sums = out->sums;
+        P.counts = agg->want_count ? out->counts : nullptr;
+    }
+
+    // ------------------------------------------------------------ shared-memory tables
+    size_t smem = 0;
+    const size_t smem_cap = (size_t)dev.max_smem_optin - 1024; // static reduce scratch + slack
+    const size_t table_budget = smem_cap > group_bytes ? smem_cap - group_bytes : 0;
+    if (opts.smem_tables != 1) {
+        std::vector<int> cand;
+        for (int s = 0; s < nfilter; ++s)
+            if (P.st[s].kind == ST_PROBE && P.st[s].tkind <= SJQ_TABLE_DIRECT_U64) cand.push_back(s);
+        // most probes per staged byte first
+        std::stable_sort(cand.begin(), cand.end(), [&](int a, int b) {
+            return reach[a] / (double)P.st[a].tab_bytes > reach[b] / (double)P.st[b].tab_bytes;
+        });
+        for (int s : cand) {
+            DStage &S = P.st[s];
+            const size_t tb = align_up(S.tab_bytes, 16);
+            if (smem + tb > table_budget) continue;
+            // worth it only if a CTA probes it more often than it costs to copy
+            const double probes_per_cta = (double)n * reach[s] / approx_grid;
+            if (probes_per_cta * 4.0 < (double)tb) continue;
+            S.in_smem = 1;
+            S.smem_off = (uint32_t)smem;
+            smem += tb;
+        }
+    }
+    P.smem_groups = (uint32_t)smem;
+    smem += group_bytes;
+    P.smem_queue = (uint32_t)smem;
+
+    // ------------------------------------------------------------ launch shape
+    int block = opts.block_threads ? opts.block_threads : 512;
+    int per_sm = 0;
+    if ((st = fused_occupancy(aggp, mul, block, smem, &per_sm)) != SJQ_OK) return st;
+    if (!opts.block_threads && per_sm <= 1) { // big shared-memory footprint: one large CTA per SM
+        block = 1024;
+        if ((st = fused_occupancy(aggp, mul, block, smem, &per_sm)) != SJQ_OK) return st;
+    }
+    if (per_sm < 1) return SJQ_ERR_UNSUPPORTED;
+    if (opts.ctas_per_sm > 0) per_sm = std::min(per_sm, opts.ctas_per_sm);
+    const int64_t tile_rows = (int64_t)block * 4;
+    const int64_t ntiles = (n + tile_rows - 1) / tile_rows;
+    int grid = (int)std::min<int64_t>((int64_t)dev.sm_count * per_sm, std::max<int64_t>(ntiles, 1));
+
+    // ------------------------------------------------------------ launches
+    int launches = 0;
+    if (!opts.accumulate) {
+        int64_t cells = spec->mode == SJQ_SCALAR ? 1 : spec->mode == SJQ_DENSE ? spec->num_groups : (int64_t)gslots + 1;
+        st = clear_launch(P.sums, spec->mode == SJQ_HASHED ? gcounts : out->counts, cells, gkeys,
+                          spec->mode == SJQ_HASHED ? (int64_t)gslots + 1 : 0, out->n_groups, out->status,
+                          dev.sm_count, stream);
+        if (st != SJQ_OK) return st;
+        ++launches;
+    } else if (spec->mode == SJQ_HASHED) {
+        if (cudaMemsetAsync(out->n_groups, 0, sizeof(int64_t), stream) != cudaSuccess) return SJQ_ERR_CUDA;
+    }
+    if (n > 0) {
+        if ((st = fused_launch(aggp, mul, grid, block, smem, P, stream)) != SJQ_OK) return st;
+        ++launches;
+    }
+    if (spec->mode == SJQ_HASHED) {
+        st = compact_launch(gkeys, gsums, gcounts, (int64_t)gslots, out->keys, out->sums, out->counts, spec->capacity,
+                            out->n_groups, out->status, dev.sm_count, stream);
+        if (st != SJQ_OK) return st;
+        ++launches;
+    }
+    if (info) {
+        std::memset(info, 0, sizeof(*info));
+        info->nstages = ns;
+        for (int s = 0; s < ns; ++s) {
+            info->order[s] = stage_label[s];
+            info->stage_in_smem[s] = P.st[s].in_smem;
+        }
+        info->first_sparse_stage = P.first_sparse;
+        info->agg_path = aggp;
+        info->grid = grid;
+        info->block = block;
+        info->smem_bytes = (int32_t)smem;
+        info->kernel_launches = launches;
+    }
+    return SJQ_OK;
+}

@@ -1,0 +1,351 @@
+"""ctypes binding of the C ABI declared in include/sjq.h.
+
+Only argument marshalling happens here: every step of the query runs in the
+CUDA kernels of libsjq.so.  PyTorch supplies device memory and the stream.
+There is no CPU fallback: if the library is missing, importing fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass, field
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsjq.so")
+
+MAX_PREDS, MAX_JOINS, MAX_PAYLOADS, MAX_KEY_TERMS = 16, 8, 2, 4
+PLAN_SCRATCH_BYTES = 256
+OPS = {"EQ": 0, "NE": 1, "LT": 2, "LE": 3, "GT": 4, "GE": 5, "BETWEEN": 6, "IN": 7}
+AGGS = {"COL": 0, "MUL": 1, "SUB": 2, "ADD": 3}
+MODES = {"SCALAR": 0, "DENSE": 1, "HASHED": 2}
+TABLE_KINDS = {1: "DIRECT_BITMAP", 2: "DIRECT_U8", 3: "DIRECT_U16", 4: "DIRECT_U32", 5: "DIRECT_U64", 6: "HASH_I32",
+               7: "HASH_I64"}
+FORCE_DIRECT, FORCE_HASH = 100, 101
+AGG_PATHS = {0: "registers", 1: "shared", 2: "global", 3: "hash"}
+
+
+class SjqError(RuntimeError):
+    def __init__(self, status: int, where: str = ""):
+        self.status = int(status)
+        super().__init__(f"{where}: {strerror(status)} ({status})")
+
+
+class _Col(ctypes.Structure):
+    _fields_ = [("data", ctypes.c_void_p), ("dtype", ctypes.c_int32), ("n", ctypes.c_int64)]
+
+
+class _Pred(ctypes.Structure):
+    _fields_ = [("col", ctypes.c_int32), ("op", ctypes.c_int32), ("lo", ctypes.c_int64), ("hi", ctypes.c_int64),
+                ("set", ctypes.POINTER(ctypes.c_int64)), ("nset", ctypes.c_int32)]
+
+
+class _Term(ctypes.Structure):
+    _fields_ = [("src", ctypes.c_int32), ("a", ctypes.c_int32), ("b", ctypes.c_int32), ("mult", ctypes.c_int64)]
+
+
+class _KeyExpr(ctypes.Structure):
+    _fields_ = [("t", _Term * MAX_KEY_TERMS), ("nterms", ctypes.c_int32), ("offset", ctypes.c_int64),
+                ("modulo", ctypes.c_int64)]
+
+
+class _AggExpr(ctypes.Structure):
+    _fields_ = [("op", ctypes.c_int32), ("x", _Term), ("y", _Term), ("want_count", ctypes.c_int32)]
+
+
+class _BuildOpts(ctypes.Structure):
+    _fields_ = [("force_kind", ctypes.c_int32), ("hash_load_pct", ctypes.c_int32),
+                ("max_direct_bytes", ctypes.c_int64)]
+
+
+class DimLayout(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int32), ("key_dtype", ctypes.c_int32), ("npayload", ctypes.c_int32),
+                ("code_bits", ctypes.c_int32), ("dim_rows", ctypes.c_int64), ("entries", ctypes.c_int64),
+                ("kmin", ctypes.c_int64), ("kmax", ctypes.c_int64), ("pay_min", ctypes.c_int64 * MAX_PAYLOADS),
+                ("pay_max", ctypes.c_int64 * MAX_PAYLOADS), ("pay_bits", ctypes.c_int32 * MAX_PAYLOADS),
+                ("slots", ctypes.c_int64), ("table_bytes", ctypes.c_size_t)]
+
+    @property
+    def kind_name(self) -> str:
+        return TABLE_KINDS.get(self.kind, str(self.kind))
+
+
+class _Join(ctypes.Structure):
+    _fields_ = [("fk_col", ctypes.c_int32), ("table", ctypes.c_void_p)]
+
+
+class _ResultSpec(ctypes.Structure):
+    _fields_ = [("mode", ctypes.c_int32), ("num_groups", ctypes.c_int64), ("capacity", ctypes.c_int64)]
+
+
+class _Result(ctypes.Structure):
+    _fields_ = [("sums", ctypes.c_void_p), ("counts", ctypes.c_void_p), ("keys", ctypes.c_void_p),
+                ("n_groups", ctypes.c_void_p), ("status", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
+                ("workspace_bytes", ctypes.c_size_t)]
+
+
+class _RunOpts(ctypes.Structure):
+    _fields_ = [("block_threads", ctypes.c_int32), ("ctas_per_sm", ctypes.c_int32), ("eager_loads", ctypes.c_int32),
+                ("agg_path", ctypes.c_int32), ("smem_tables", ctypes.c_int32), ("compaction", ctypes.c_int32),
+                ("accumulate", ctypes.c_int32), ("norder", ctypes.c_int32),
+                ("order", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS)), ("reserved", ctypes.c_int32 * 8)]
+
+
+class RunInfo(ctypes.Structure):
+    _fields_ = [("nstages", ctypes.c_int32), ("order", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS + 8)),
+                ("stage_in_smem", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS + 8)),
+                ("first_sparse_stage", ctypes.c_int32), ("agg_path", ctypes.c_int32), ("grid", ctypes.c_int32),
+                ("block", ctypes.c_int32), ("smem_bytes", ctypes.c_int32), ("kernel_launches", ctypes.c_int32)]
+
+    def describe(self) -> dict:
+        return {"order": list(self.order[: self.nstages]), "in_smem": list(self.stage_in_smem[: self.nstages]),
+                "first_sparse_stage": self.first_sparse_stage, "agg_path": AGG_PATHS.get(self.agg_path),
+                "grid": self.grid, "block": self.block, "smem_bytes": self.smem_bytes,
+                "kernel_launches": self.kernel_launches}
+
+
+@dataclass
+class RunOpts:
+    block_threads: int = 0
+    ctas_per_sm: int = 0
+    eager_loads: bool = False
+    agg_path: int = 0
+    smem_tables: int = 0
+    compaction: int = 0
+    accumulate: bool = False
+    order: Sequence[int] = ()
+
+    def to_c(self) -> _RunOpts:
+        o = _RunOpts()
+        o.block_threads, o.ctas_per_sm = self.block_threads, self.ctas_per_sm
+        o.eager_loads, o.agg_path, o.smem_tables = int(self.eager_loads), self.agg_path, self.smem_tables
+        o.compaction, o.accumulate = self.compaction, int(self.accumulate)
+        o.norder = len(self.order)
+        for i, v in enumerate(self.order):
+            o.order[i] = v
+        return o
+
+
+_lib = None
+
+
+def lib():
+    """Load libsjq.so; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with paper_2607_07632_b200/build.py "
+                              "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, ip = ctypes.c_void_p, ctypes.c_int
+        L.sjq_dim_plan.restype = ctypes.c_int32
+        L.sjq_dim_plan.argtypes = [ctypes.POINTER(_Col), ip, ctypes.POINTER(_Pred), ip, ip, ctypes.POINTER(ip), ip,
+                                   ctypes.POINTER(_BuildOpts), vp, vp, ctypes.POINTER(DimLayout)]
+        L.sjq_build_dim.restype = ctypes.c_int32
+        L.sjq_build_dim.argtypes = [ctypes.POINTER(_Col), ip, ctypes.POINTER(_Pred), ip, ip, ctypes.POINTER(ip), ip,
+                                    ctypes.POINTER(DimLayout), vp, ctypes.c_size_t, vp, vp, ctypes.POINTER(vp)]
+        L.sjq_table_info.restype = ctypes.c_int32
+        L.sjq_table_info.argtypes = [vp, ctypes.POINTER(DimLayout)]
+        L.sjq_table_destroy.restype = None
+        L.sjq_table_destroy.argtypes = [vp]
+        L.sjq_run_workspace_bytes.restype = ctypes.c_int32
+        L.sjq_run_workspace_bytes.argtypes = [ctypes.POINTER(_ResultSpec), ctypes.POINTER(ctypes.c_size_t)]
+        L.sjq_run.restype = ctypes.c_int32
+        L.sjq_run.argtypes = [ctypes.POINTER(_Col), ip, ctypes.POINTER(_Pred), ip, ctypes.POINTER(_Join), ip,
+                              ctypes.POINTER(_KeyExpr), ctypes.POINTER(_AggExpr), ctypes.POINTER(_ResultSpec),
+                              ctypes.POINTER(_Result), ctypes.POINTER(_RunOpts), vp, ctypes.POINTER(RunInfo)]
+        L.sjq_strerror.restype = ctypes.c_char_p
+        L.sjq_strerror.argtypes = [ctypes.c_int32]
+        L.sjq_version.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def strerror(status: int) -> str:
+    return lib().sjq_strerror(int(status)).decode()
+
+
+def version() -> str:
+    return lib().sjq_version().decode()
+
+
+def _stream_ptr(device) -> int:
+    return torch.cuda.current_stream(device).cuda_stream
+
+
+def _cols(tensors: Sequence[torch.Tensor]):
+    arr = (_Col * max(1, len(tensors)))()
+    for i, t in enumerate(tensors):
+        if t.dtype not in (torch.int32, torch.int64) or not t.is_cuda or not t.is_contiguous() or t.dim() != 1:
+            raise ValueError("columns must be contiguous 1-D int32/int64 CUDA tensors")
+        arr[i] = _Col(t.data_ptr(), 1 if t.dtype == torch.int64 else 0, t.numel())
+    return arr
+
+
+def _preds(preds, names: Sequence[str]):
+    keep = []
+    arr = (_Pred * max(1, len(preds)))()
+    for i, p in enumerate(preds):
+        vals = (ctypes.c_int64 * max(1, len(p.values)))(*p.values)
+        keep.append(vals)
+        arr[i] = _Pred(names.index(p.col), OPS[p.op], p.lo, p.hi, vals, len(p.values))
+    return arr, keep
+
+
+class Table:
+    """A built dimension table: host handle + the device memory it lives in."""
+
+    def __init__(self, handle: int, layout: DimLayout, mem: torch.Tensor, status: torch.Tensor):
+        self.handle, self.layout, self.mem, self.status_dev = handle, layout, mem, status
+
+    def status(self) -> int:
+        return int(self.status_dev.item())
+
+    def check(self) -> "Table":
+        st = self.status()
+        if st != 0:
+            raise SjqError(st, "sjq_build_dim")
+        return self
+
+    def __del__(self):
+        if getattr(self, "handle", None) and _lib is not None:
+            _lib.sjq_table_destroy(self.handle)
+            self.handle = None
+
+
+def build_dim(cols: dict, key: str, preds=(), payloads=(), force_kind: int = 0, hash_load_pct: int = 0,
+              max_direct_bytes: int = 0) -> Table:
+    """sjq_dim_plan + sjq_build_dim over a dict of CUDA tensors (dimension columns)."""
+    names = list(cols.keys())
+    tensors = [cols[n] for n in names]
+    device = tensors[0].device
+    with torch.cuda.device(device):
+        carr = _cols(tensors)
+        parr, keep = _preds(preds, names)
+        pay = (ctypes.c_int * max(1, len(payloads)))(*[names.index(p) for p in payloads])
+        opts = _BuildOpts(force_kind, hash_load_pct, max_direct_bytes)
+        scratch = torch.empty(PLAN_SCRATCH_BYTES, dtype=torch.uint8, device=device)
+        layout = DimLayout()
+        stream = _stream_ptr(device)
+        rc = lib().sjq_dim_plan(carr, len(names), parr, len(preds), names.index(key), pay, len(payloads),
+                                ctypes.byref(opts), scratch.data_ptr(), stream, ctypes.byref(layout))
+        if rc != 0:
+            raise SjqError(rc, "sjq_dim_plan")
+        mem = torch.empty(layout.table_bytes, dtype=torch.uint8, device=device)
+        status = torch.zeros(1, dtype=torch.int32, device=device)
+        handle = ctypes.c_void_p()
+        rc = lib().sjq_build_dim(carr, len(names), parr, len(preds), names.index(key), pay, len(payloads),
+                                 ctypes.byref(layout), mem.data_ptr(), mem.numel(), status.data_ptr(), stream,
+                                 ctypes.byref(handle))
+        if rc != 0:
+            raise SjqError(rc, "sjq_build_dim")
+    return Table(handle.value, layout, mem, status)
+
+
+@dataclass
+class Result:
+    mode: str
+    sums: torch.Tensor
+    counts: Optional[torch.Tensor]
+    keys: Optional[torch.Tensor]
+    n_groups: Optional[torch.Tensor]
+    status_dev: torch.Tensor
+    workspace: Optional[torch.Tensor]
+    info: RunInfo = field(default_factory=RunInfo)
+
+    def status(self) -> int:
+        return int(self.status_dev.item())
+
+    def check(self) -> "Result":
+        st = self.status()
+        if st != 0:
+            raise SjqError(st, "sjq_run")
+        return self
+
+    def hashed_sorted(self):
+        """(keys, sums, counts) of a HASHED result in ascending key order."""
+        n = int(self.n_groups.item())
+        k, idx = torch.sort(self.keys[:n])
+        return k, self.sums[:n][idx], self.counts[:n][idx]
+
+
+def _term(t, names) -> _Term:
+    if t is None:
+        return _Term(0, 0, 0, 0)
+    if t.src == "FACT":
+        return _Term(0, names.index(t.a), 0, t.mult)
+    return _Term(1, int(t.a), t.b, t.mult)
+
+
+def alloc_result(mode: str, num_groups: int, capacity: int, want_count: bool, device) -> Result:
+    spec = _ResultSpec(MODES[mode], num_groups, capacity)
+    n = 1 if mode == "SCALAR" else num_groups if mode == "DENSE" else capacity
+    sums = torch.empty(n, dtype=torch.int64, device=device)
+    counts = torch.empty(n, dtype=torch.int64, device=device) if (want_count or mode == "HASHED") else None
+    keys = n_groups = ws = None
+    if mode == "HASHED":
+        keys = torch.empty(n, dtype=torch.int64, device=device)
+        n_groups = torch.zeros(1, dtype=torch.int64, device=device)
+        nbytes = ctypes.c_size_t(0)
+        rc = lib().sjq_run_workspace_bytes(ctypes.byref(spec), ctypes.byref(nbytes))
+        if rc != 0:
+            raise SjqError(rc, "sjq_run_workspace_bytes")
+        ws = torch.empty(nbytes.value, dtype=torch.uint8, device=device)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    return Result(mode, sums, counts, keys, n_groups, status, ws)
+
+
+def run(fact: dict, preds=(), joins=(), key=None, agg=None, mode: str = "SCALAR", num_groups: int = 1,
+        capacity: int = 0, opts: Optional[RunOpts] = None, result: Optional[Result] = None) -> Result:
+    """sjq_run over a dict of CUDA tensors.  joins: sequence of (fk column name, Table)."""
+    names = list(fact.keys())
+    tensors = [fact[n] for n in names]
+    device = tensors[0].device
+    with torch.cuda.device(device):
+        carr = _cols(tensors)
+        parr, keep = _preds(preds, names)
+        jarr = (_Join * max(1, len(joins)))()
+        for j, (fk, table) in enumerate(joins):
+            jarr[j] = _Join(names.index(fk), table.handle)
+        kexpr = None
+        if key is not None:
+            kexpr = _KeyExpr()
+            if len(key.terms) > MAX_KEY_TERMS:
+                raise ValueError("too many key terms")
+            for i, t in enumerate(key.terms):
+                kexpr.t[i] = _term(t, names)
+            kexpr.nterms, kexpr.offset, kexpr.modulo = len(key.terms), key.offset, key.modulo
+        aexpr = _AggExpr(AGGS[agg.op], _term(agg.x, names), _term(agg.y, names), int(agg.want_count))
+        spec = _ResultSpec(MODES[mode], num_groups, capacity)
+        res = result if result is not None else alloc_result(mode, num_groups, capacity, agg.want_count, device)
+        cres = _Result(res.sums.data_ptr(), res.counts.data_ptr() if res.counts is not None else None,
+                       res.keys.data_ptr() if res.keys is not None else None,
+                       res.n_groups.data_ptr() if res.n_groups is not None else None, res.status_dev.data_ptr(),
+                       res.workspace.data_ptr() if res.workspace is not None else None,
+                       res.workspace.numel() if res.workspace is not None else 0)
+        copts = (opts or RunOpts()).to_c()
+        rc = lib().sjq_run(carr, len(names), parr, len(preds), jarr, len(joins),
+                           ctypes.byref(kexpr) if kexpr is not None else None, ctypes.byref(aexpr),
+                           ctypes.byref(spec), ctypes.byref(cres), ctypes.byref(copts), _stream_ptr(device),
+                           ctypes.byref(res.info))
+        if rc != 0:
+            raise SjqError(rc, "sjq_run")
+    return res
+
+
+def build_workload_tables(w, dims: dict) -> dict:
+    """dims: dimension name -> dict of CUDA column tensors (a workload description's dims)."""
+    out = {}
+    for d in w.dims:
+        out[d.name] = build_dim(dims[d.name], d.key, d.preds, d.payloads,
+                                force_kind=FORCE_HASH if d.force_hash else 0)
+    return out
+
+
+def run_workload(w, fact: dict, tables: dict, opts: Optional[RunOpts] = None,
+                 result: Optional[Result] = None) -> Result:
+    fact = {c.name: fact[c.name] for c in w.fact_cols}
+    return run(fact, w.preds, [(fk, tables[dn]) for fk, dn in w.joins], w.key, w.agg, w.mode, w.num_groups,
+               w.capacity, opts, result)

@@ -1,0 +1,213 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle: bit-exact
+on every output element, on the same seeded inputs."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from datagen import workloads as W
+from datagen.workloads import AggExpr, KeyExpr, Pred, Term
+
+pytestmark = pytest.mark.gpu
+
+sjq = pytest.importorskip("paper_2607_07632_b200") if torch.cuda.is_available() else None
+
+from gpuhelpers import compare, run_both, to_dev  # noqa: E402
+from qhelpers import adhoc, ex1, ex2, ex3, random_query  # noqa: E402
+from bruteforce import dup_keys_among_passing  # noqa: E402
+
+RAGGED = [0, 1, 3, 4, 5, 255, 256, 257, 2047, 2048, 2049, 4097, 100003]
+
+
+def test_hand_examples():
+    for mk in (ex1, ex2, ex3):
+        w, fact, hd, _ = mk()
+        res, exp, _ = run_both(w, fact, hd)
+        assert res.status() == 0
+        compare(w, res, exp)
+
+
+@pytest.mark.parametrize("seed", range(200))
+def test_random_small_queries(seed):
+    w, fact, hd = random_query(seed, allow_dup=False, wide_keys=True)
+    res, exp, _ = run_both(w, fact, hd, check=False)
+    if exp["status"] == oracle.GROUP_RANGE:
+        assert res.status() == 18
+        # rows with an in-range key still land where the oracle puts them
+        compare(w, res, exp)
+    else:
+        assert res.status() == 0
+        compare(w, res, exp)
+
+
+@pytest.mark.parametrize("seed", range(200, 240))
+def test_random_queries_option_matrix(seed):
+    w, fact, hd = random_query(seed, n_fact=700, allow_dup=False, wide_keys=True)
+    dev_fact = to_dev(fact)
+    tables = None
+    for opts in (sjq.RunOpts(), sjq.RunOpts(eager_loads=True), sjq.RunOpts(smem_tables=1),
+                 sjq.RunOpts(block_threads=128, ctas_per_sm=1), sjq.RunOpts(agg_path=2),
+                 sjq.RunOpts(compaction=2), sjq.RunOpts(compaction=1),
+                 sjq.RunOpts(order=tuple(reversed(range(len(w.preds) + len(w.joins)))))):
+        res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)
+        assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)
+        compare(w, res, exp)
+
+
+@pytest.mark.parametrize("n", RAGGED)
+@pytest.mark.parametrize("cfg", ["c1", "c2", "c3", "c4d", "c4h", "c5"])
+def test_configs_ragged_sizes(cfg, n):
+    w = {"c1": lambda: W.config1(n), "c2": lambda: W.config2(n), "c3": lambda: W.config3(n),
+         "c4d": lambda: W.config4(n, 0.5, 1000, dim_rows=50000),
+         "c4h": lambda: W.config4(n, 0.5, 100000, dim_rows=50000),
+         "c5": lambda: W.config5(n, 20000)}[cfg]()
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    res, exp, _ = run_both(w, fact, hd)
+    assert res.status() == 0
+    compare(w, res, exp)
+
+
+@pytest.mark.parametrize("mk", [lambda: W.config1(1_500_007), lambda: W.config2(2_000_003),
+                                lambda: W.config3(2_500_001), lambda: W.config5(1_200_005, 300000)] +
+                         [lambda s=s, g=g: W.config4(1_000_003, s, g) for s in (0.0001, 0.1, 1.0)
+                          for g in (1, 1000, 100000, 1000000)])
+def test_configs_multi_tile(mk):
+    w = mk()
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    res, exp, tables = run_both(w, fact, hd)
+    assert res.status() == 0
+    compare(w, res, exp)
+    # the same query with every switch flipped gives the same bits
+    dev_fact = to_dev(fact)
+    for opts in (sjq.RunOpts(eager_loads=True, smem_tables=1, compaction=1),
+                 sjq.RunOpts(agg_path=2 if w.mode == "DENSE" else 0, block_threads=256, compaction=2)):
+        res2, _, _ = run_both(w, fact, hd, opts=opts, dev_fact=dev_fact, tables=tables)
+        compare(w, res2, exp)
+
+
+def test_device_generator_matches_host():
+    for w in (W.config1(100_003), W.config3(100_003), W.config5(100_003, 50000)):
+        host = W.host_fact(w)
+        dev = W.device_fact(w)
+        for k in host:
+            assert np.array_equal(dev[k].cpu().numpy(), host[k]), (w.name, k)
+        # a window in the middle of a large table is the same function of the row
+        dev2 = W.device_fact(w, 50_000, 1000)
+        for k in host:
+            assert np.array_equal(dev2[k].cpu().numpy(), host[k][50_000:51_000])
+        for d in w.dims:
+            hd, dd = W.host_dim(w, d), W.device_dim(w, d)
+            for k in hd:
+                assert np.array_equal(dd[k].cpu().numpy(), hd[k])
+
+
+def test_table_kinds_and_sizes():
+    # Section 3.3 sizes: 3M keys -> 3 MB byte-packed map (12 MB as int32)
+    w = W.config3(10)
+    dims = {d.name: W.device_dim(w, d) for d in w.dims}
+    tabs = sjq.build_workload_tables(w, dims)
+    L = tabs["customer"].layout
+    assert L.kind_name == "DIRECT_U8" and L.slots == 3_000_000 and L.code_bits == 8
+    assert 3_000_000 <= L.table_bytes <= 3_000_000 + 1024
+    assert tabs["supplier"].layout.kind_name == "DIRECT_BITMAP" and tabs["supplier"].layout.slots == 200_000
+    assert tabs["part"].layout.kind_name == "DIRECT_BITMAP"
+    d = tabs["date"].layout
+    assert d.kind_name == "DIRECT_U8" and d.entries == 729 and d.kmin == 19970101 and d.kmax == 19981230
+    # forcing the unpacked form: open addressing at load <= 0.5
+    t = sjq.build_dim(dims["customer"], "custkey", w.dim("customer").preds, ("nation",), force_kind=sjq.sjq.FORCE_HASH)
+    assert t.layout.kind_name == "HASH_I32" and t.layout.slots >= 2 * t.layout.entries
+    assert t.check().status() == 0
+    # wide payloads choose wider codes
+    cols = {"k": torch.arange(1, 1001, dtype=torch.int32, device="cuda"),
+            "a": torch.arange(0, 1000, dtype=torch.int32, device="cuda") * 70,
+            "b": torch.arange(0, 1000, dtype=torch.int32, device="cuda") - 500}
+    assert sjq.build_dim(cols, "k", (), ("a",)).layout.kind_name == "DIRECT_U32"
+    assert sjq.build_dim(cols, "k", (), ("b",)).layout.kind_name == "DIRECT_U16"
+    t2 = sjq.build_dim(cols, "k", (), ("a", "b"))
+    assert t2.layout.kind_name == "DIRECT_U32" and t2.layout.pay_bits[0] == 17 and t2.layout.pay_bits[1] == 10
+
+
+def test_duplicate_key_is_reported():
+    for force in (0, sjq.sjq.FORCE_HASH):
+        for npay in (0, 1):
+            cols = {"k": torch.tensor([5, 9, 7, 9], dtype=torch.int32, device="cuda"),
+                    "p": torch.tensor([1, 2, 3, 4], dtype=torch.int32, device="cuda")}
+            t = sjq.build_dim(cols, "k", (), ("p",)[:npay], force_kind=force)
+            assert t.status() == 16
+            # the duplicate filtered away -> fine
+            t = sjq.build_dim(cols, "k", (Pred("p", "NE", 4),), ("p",)[:npay], force_kind=force)
+            assert t.status() == 0
+
+
+def test_reserved_key_and_empty_dimension():
+    cols = {"k": torch.tensor([-(2 ** 63), 4], dtype=torch.int64, device="cuda")}
+    assert sjq.build_dim(cols, "k", force_kind=sjq.sjq.FORCE_HASH).status() == 20
+    fact = {"fk": np.array([4, 5, -(2 ** 63)], np.int64), "v": np.array([1, 2, 3], np.int32)}
+    dim = {"k": np.array([4, 5], np.int64), "f": np.array([0, 0], np.int32)}
+    w = adhoc("empty", fact, [("d", dim, "k", [Pred("f", "EQ", 1)], [], True)], [("fk", "d")], [], None,
+              AggExpr("COL", Term("FACT", "v")), "SCALAR")
+    res, exp, tabs = run_both(w, fact, {"d": dim})
+    assert tabs["d"].layout.entries == 0
+    compare(w, res, exp)
+    assert int(res.counts[0].item()) == 0
+
+
+def test_fk_outside_key_range_is_a_miss():
+    fact = {"fk": np.array([-7, 0, 1, 5, 6, 2 ** 31 - 1, -2 ** 31], np.int32), "v": np.arange(7, dtype=np.int32) + 1}
+    dim = {"k": np.array([1, 5], np.int32), "p": np.array([3, 4], np.int32)}
+    for force in (False, True):
+        w = adhoc("miss", fact, [("d", dim, "k", [], ["p"], force)], [("fk", "d")], [], None,
+                  AggExpr("MUL", Term("FACT", "v"), Term("PAYLOAD", 0, 0)), "SCALAR")
+        res, exp, _ = run_both(w, fact, {"d": dim})
+        compare(w, res, exp)
+        assert int(res.sums[0].item()) == 25
+
+
+def test_hashed_overflow_and_group_range_status():
+    n = 5000
+    fact = {"g": np.arange(n, dtype=np.int32)}
+    w = adhoc("ovf", fact, [], [], [], KeyExpr((Term("FACT", "g"),)), AggExpr("COL", Term("FACT", "g")), "HASHED",
+              capacity=64)
+    res = sjq.run_workload(w, to_dev(fact), {})
+    assert res.status() == 19
+    w = adhoc("rng", fact, [], [], [], KeyExpr((Term("FACT", "g"),)), AggExpr("COL", Term("FACT", "g")), "DENSE",
+              num_groups=100)
+    res = sjq.run_workload(w, to_dev(fact), {})
+    assert res.status() == 18
+    assert int(res.counts.sum().item()) == 100
+
+
+def test_accumulate_equals_whole():
+    w = W.config3(300_001)
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    res, exp, tables = run_both(w, fact, hd)
+    k = 123_457
+    a = to_dev({c: v[:k] for c, v in fact.items()})
+    b = to_dev({c: v[k:].copy() for c, v in fact.items()})
+    r = sjq.run_workload(replace(w, n_rows=k), a, tables)
+    r = sjq.run_workload(replace(w, n_rows=w.n_rows - k), b, tables, sjq.RunOpts(accumulate=True), result=r)
+    torch.cuda.synchronize()
+    compare(w, r, exp)
+
+
+def test_invalid_arguments_are_rejected():
+    fact = {"a": torch.zeros(8, dtype=torch.int32, device="cuda"), "b": torch.zeros(9, dtype=torch.int32, device="cuda")}
+    with pytest.raises(sjq.SjqError) as e:
+        sjq.run(fact, agg=AggExpr("COL", Term("FACT", "a")))
+    assert e.value.status == 1
+    ok = {"a": torch.zeros(64, dtype=torch.int32, device="cuda")}
+    with pytest.raises(sjq.SjqError) as e:  # misaligned column
+        sjq.run({"a": ok["a"][1:9]}, agg=AggExpr("COL", Term("FACT", "a")))
+    assert e.value.status == 3
+    with pytest.raises(sjq.SjqError) as e:  # grouped mode without a key
+        sjq.run(ok, agg=AggExpr("COL", Term("FACT", "a")), mode="DENSE", num_groups=4)
+    assert e.value.status == 1
+    dim = sjq.build_dim({"k": torch.arange(4, dtype=torch.int64, device="cuda")}, "k")
+    with pytest.raises(sjq.SjqError) as e:  # int32 fk into an int64-keyed table
+        sjq.run(ok, joins=[("a", dim)], agg=AggExpr("COL", Term("FACT", "a")))
+    assert e.value.status == 2

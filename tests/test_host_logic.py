@@ -1,0 +1,67 @@
+"""CPU-only checks of the boundary: the C-ABI library loads and exports every
+symbol the public header declares, and host-side argument validation answers
+without a GPU (no compute is attempted)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def libsjq():
+    from paper_2607_07632_b200 import build
+
+    return ctypes.CDLL(build.build())
+
+
+def _declared_symbols():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        text = open(os.path.join(ROOT, "include", fn)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names |= set(re.findall(r"\b(sjq_[a-z0-9_]+)\s*\(", text))
+    return names
+
+
+def test_library_exports_every_declared_symbol(libsjq):
+    names = _declared_symbols()
+    assert {"sjq_dim_plan", "sjq_build_dim", "sjq_run", "sjq_table_info", "sjq_table_destroy",
+            "sjq_run_workspace_bytes", "sjq_strerror", "sjq_version"} <= names
+    for n in names:
+        assert hasattr(libsjq, n), n
+
+
+def test_strerror_and_workspace_size(libsjq):
+    import paper_2607_07632_b200.sjq as b
+
+    assert b.strerror(0) == "ok" and "duplicate" in b.strerror(16)
+    spec = b._ResultSpec(b.MODES["HASHED"], 0, 1000)
+    n = ctypes.c_size_t(0)
+    assert b.lib().sjq_run_workspace_bytes(ctypes.byref(spec), ctypes.byref(n)) == 0
+    # 2048 slots + the side slot, three int64 arrays
+    assert 3 * 2049 * 8 <= n.value <= 3 * 2049 * 8 + 3 * 256
+    spec = b._ResultSpec(b.MODES["DENSE"], 7000, 0)
+    assert b.lib().sjq_run_workspace_bytes(ctypes.byref(spec), ctypes.byref(n)) == 0 and n.value == 0
+    spec = b._ResultSpec(b.MODES["HASHED"], 0, 0)
+    assert b.lib().sjq_run_workspace_bytes(ctypes.byref(spec), ctypes.byref(n)) == 1
+
+
+def test_null_arguments_rejected_without_gpu(libsjq):
+    import paper_2607_07632_b200.sjq as b
+
+    assert b.lib().sjq_run(None, 0, None, 0, None, 0, None, None, None, None, None, None, None) == 1
+    assert b.lib().sjq_dim_plan(None, 0, None, 0, 0, None, 0, None, None, None, None) == 1
+    assert b.lib().sjq_table_info(None, None) == 1
+    b.lib().sjq_table_destroy(None)
+
+
+def test_product_never_imports_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2607_07632_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower(), f
