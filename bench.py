@@ -1,0 +1,422 @@
+#!/usr/bin/env python
+"""Benchmark of the fused star-join query pipeline.
+
+    python bench.py --gpus N --steps K --warmup W            (one rank per GPU under torchrun for N > 1)
+    python bench.py --impl reference --gpus N --steps K --warmup W
+
+A step is one whole query: plan and build every dimension table from the
+filtered dimension columns, then one fused pass over the fact table (and, for
+N > 1, an all-reduce of the dense result).  The workload is the four-join
+group-by over 600 M fact rows (14.4 GB of referenced fact columns, far larger
+than the 126 MB L2, so no L2 flush is needed between steps); every rank holds
+its own 600 M-row shard of the row space and a replica of the dimensions
+(weak scaling).  Rank 0 prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "fact_rows_per_s"
+UNIT = "rows/s"
+CONTRACT_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per fact row of the fused kernel from the ncu capture summarised in
+# profiles/fused_kernel_c3_100m.md (a 100 M-row case of the same workload; traffic grows with the rows)
+NCU_DRAM_BYTES_PER_ROW = {"c3": 16.7}
+
+
+def measured_hbm_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def make_workload(name: str, rows: int | None, sel: float, groups: int):
+    from datagen import workloads as W
+
+    if name == "c4":
+        return W.config4(rows or 600_000_000, sel, groups)
+    return W.CONFIGS[name](rows) if rows else W.CONFIGS[name]()
+
+
+def stage_selectivities(w):
+    """Exact pass fractions of the workload's filters, from its definition (uniform draws)."""
+    from datagen import DATE_ROWS
+
+    sel = {}
+    if w.name.startswith("c1"):
+        sel = {"pred:discount": 3 / 11, "pred:quantity": 29 / 50, "join:date": 365 / DATE_ROWS}
+    elif w.name.startswith("c2"):
+        sel = {"join:part": 1 / 25, "join:supplier": 1 / 5, "join:date": 1.0}
+    elif w.name.startswith("c3"):
+        sel = {"join:customer": 1 / 5, "join:supplier": 1 / 5, "join:part": 2 / 5, "join:date": 729 / DATE_ROWS}
+    elif w.name.startswith("c4"):
+        sel = {"pred:p": w.preds[0].lo / 10000.0, "join:dim": 1.0}
+    elif w.name.startswith("c5"):
+        sel = {"join:dim": 0.25}
+    return sel
+
+
+def algorithmic_bytes_per_row(w, order):
+    """Sector model: the first column is read whole; a later column is read for a 32-byte sector
+    iff at least one of its rows survived everything evaluated before it."""
+    sel = stage_selectivities(w)
+    names = [f"pred:{p.col}" for p in w.preds] + [f"join:{d}" for _, d in w.joins]
+    cols = [p.col for p in w.preds] + [fk for fk, _ in w.joins]
+    reach, total, seen = 1.0, 0.0, set()
+    for idx in order:
+        if idx < 0:
+            continue
+        col = cols[idx]
+        width = 8 if w.fact_col(col).is64 else 4
+        if col not in seen:
+            total += width * (1.0 - (1.0 - reach) ** (32 // width))
+            seen.add(col)
+        reach *= sel.get(names[idx], 1.0)
+    for c in w.fact_cols:  # columns only the key or the aggregate reads
+        if c.name not in seen:
+            width = 8 if c.is64 else 4
+            total += width * (1.0 - (1.0 - reach) ** (32 // width))
+    return total
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.stop_flag, self.samples, self.reasons, self.max_mhz = index, False, [], set(), None
+        self.error = None
+
+    def run(self):
+        try:
+            import pynvml as nv
+
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            names = {nv.nvmlClocksEventReasonHwSlowdown: "hw_slowdown",
+                     nv.nvmlClocksEventReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                     nv.nvmlClocksEventReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                     nv.nvmlClocksEventReasonSwPowerCap: "sw_power_cap"}
+            while not self.stop_flag:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                for bit, nm in names.items():
+                    if r & bit:
+                        self.reasons.add(nm)
+                time.sleep(0.01)
+        except Exception as e:  # pragma: no cover - depends on the box
+            self.error = repr(e)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0,
+                    "error": self.error}
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+def visible_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def oracle_rate(w, sample_rows: int, row0: int = 0):
+    """Time the CPU oracle (as it stands, one thread) on rows [row0, row0 + sample_rows) of the workload."""
+    import oracle
+    from datagen import workloads as W
+
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    fact = W.host_fact(w, row0, sample_rows)
+    t0 = time.perf_counter()
+    dims = oracle.build_dims(w, hd)
+    t_build = time.perf_counter() - t0
+    r = oracle.run(w, fact, dims)
+    return sample_rows / (r["seconds"] + t_build), r["seconds"], t_build
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on bounded samples of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    from datagen import workloads as W
+
+    w = make_workload(args.workload, args.rows, args.sel, args.groups)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    probe = min(w.n_rows, 2_000_000)
+    fact = W.host_fact(w, 0, probe)
+    dims = oracle.build_dims(w, hd)
+    t = oracle.run(w, fact, dims)["seconds"]
+    per_row = max(t / probe, 1e-9)
+    budget_s = 90.0
+    sample = int(min(w.n_rows, max(100_000, budget_s / per_row / (args.steps + args.warmup))))
+    times = []
+    for i in range(args.warmup + args.steps):
+        row0 = (i * sample) % max(1, w.n_rows - sample + 1)
+        fact = W.host_fact(w, row0, sample)
+        t0 = time.perf_counter()
+        dims = oracle.build_dims(w, hd)
+        oracle.run(w, fact, dims)
+        dt = time.perf_counter() - t0
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1000.0 * sum(times) / len(times)
+    value = sample / (ms / 1000.0)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+            "config": {"workload": w.name, "rows": w.n_rows, "rows_per_step": sample,
+                       "note": "CPU oracle (single thread) on a bounded sample of the workload per step"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": f"{sample} consecutive fact rows per step, dimension build included"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--rows", type=int, default=None, help="override the fact rows per GPU (debugging)")
+    ap.add_argument("--sel", type=float, default=0.1, help="c4: fact predicate selectivity")
+    ap.add_argument("--groups", type=int, default=1000, help="c4: number of groups")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-sample-rows", type=int, default=100_000_000)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--extras", action="store_true", help="also time the other configurations (N = 1 only)")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2607_07632_b200 as sjq
+    from datagen import workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=device)
+
+    w = make_workload(args.workload, args.rows, args.sel, args.groups)
+    n = w.n_rows
+    dims = {d.name: W.device_dim(w, d, device) for d in w.dims}
+    fact = W.device_fact(w, row0=rank * n, n=n, device=device)  # this rank's shard of the row space
+    torch.cuda.synchronize()
+
+    # every event pair is created (recorded once) up front; the library records them around the fused kernel
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+             for _ in range(args.steps)]
+    for a, b in pairs:
+        a.record()
+        b.record()
+    res = sjq.alloc_result(w.mode, w.num_groups, w.capacity, w.agg.want_count, device)
+    launches = 0
+    info = None
+
+    def step(i=None):
+        nonlocal launches, info
+        tables = sjq.build_workload_tables(w, dims)
+        opts = sjq.RunOpts(events=pairs[i]) if i is not None else None
+        r = sjq.run_workload(w, fact, tables, opts, result=res)
+        if world > 1 and w.mode != "HASHED":
+            dist.all_reduce(res.sums)
+            if res.counts is not None:
+                dist.all_reduce(res.counts)
+        if i is not None:
+            launches += r.info.kernel_launches + sum(sjq.build_launches(t) for t in tables.values())
+        info = r.info
+        return tables
+
+    for _ in range(args.warmup):
+        tables = step()
+    torch.cuda.synchronize()
+    assert res.status() == 0 and all(t.status() == 0 for t in tables.values())
+
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    ev0.record()
+    for i in range(args.steps):
+        step(i)
+    ev1.record()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.stop_flag = True
+    sampler.join(timeout=2.0)
+    ms_total = ev0.elapsed_time(ev1)
+    fused_ms = sum(a.elapsed_time(b) for a, b in pairs) / len(pairs)
+    t = torch.tensor([ms_total, fused_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, fused_ms = float(t[0]), float(t[1])
+    ms_per_step = ms_total / args.steps
+    value = world * n / (ms_per_step / 1000.0)
+    ref_bytes = w.referenced_bytes_per_row()
+    eff_gbs = world * n * ref_bytes / (ms_per_step / 1000.0) / 1e9
+
+    peak, peak_kind = measured_hbm_peak()
+    alg_bpr = algorithmic_bytes_per_row(w, list(info.order[: info.nstages]))
+    achieved = n * alg_bpr / (fused_ms / 1000.0) / 1e9
+    traffic_bpr = NCU_DRAM_BYTES_PER_ROW.get(args.workload)
+    roofline = {"bound": "hbm", "kernel": "fused_kernel", "achieved": achieved, "peak": peak,
+                "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                "traffic": traffic_bpr * n if traffic_bpr else None,
+                "algorithmic_bytes_per_row": alg_bpr, "kernel_ms": fused_ms,
+                "effective_gbs_kernel": n * ref_bytes / (fused_ms / 1000.0) / 1e9}
+
+    e2e = None
+    if not args.no_e2e:
+        try:
+            host_fact = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in fact.items()}
+            for k, v in fact.items():
+                host_fact[k].copy_(v)
+            torch.cuda.synchronize()
+            chunk = min(n, 32 << 20) // 4 * 4 or 4
+            staging = torch.empty(sjq.staging_bytes(host_fact, chunk), dtype=torch.uint8, device=device)
+            eres, ehost = None, None
+
+            def e2e_step():
+                nonlocal eres, ehost
+                tabs = sjq.build_workload_tables(w, dims)
+                eres, ehost = sjq.run_workload_host(w, host_fact, tabs, staging, chunk, result=eres, host=ehost)
+                torch.cuda.synchronize()  # the result is on the host when this returns
+                return tabs
+
+            e2e_step()
+            if world > 1:
+                dist.barrier()
+            t0 = time.perf_counter()
+            for _ in range(args.e2e_steps):
+                e2e_step()
+            dt = (time.perf_counter() - t0) / args.e2e_steps
+            tt = torch.tensor([dt], dtype=torch.float64, device=device)
+            if world > 1:
+                dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            dt = float(tt[0])
+            same = bool(torch.equal(ehost.sums, res.sums.cpu())) if world == 1 else None
+            cells = 1 if w.mode == "SCALAR" else w.num_groups if w.mode == "DENSE" else w.capacity
+            e2e = {"value": world * n / dt, "unit": UNIT, "h2d_bytes_per_step": n * ref_bytes,
+                   "d2h_bytes_per_step": cells * 8 * (2 if w.agg.want_count else 1) + 4, "ms_per_step": dt * 1000.0,
+                   "steps": args.e2e_steps, "chunk_rows": chunk, "matches_device_run": same,
+                   "api": "sjq_run_host (pinned host columns, chunked double-buffered copies, result copied back)"}
+            del host_fact, staging
+        except Exception as ex:  # e.g. not enough page-locked memory on the box
+            e2e = {"value": None, "unit": UNIT, "error": repr(ex)[:200]}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sample = min(n, args.cpu_sample_rows)
+        rate, secs, tb = oracle_rate(w, sample)
+        cpu = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"first {sample} fact rows of the workload; row loop {secs:.2f} s + dimension maps {tb:.2f} s",
+               "host_cores_available": os.cpu_count()}
+
+    extras = None
+    if args.extras and world == 1 and rank == 0:
+        del fact
+        torch.cuda.empty_cache()
+        extras = run_extras(sjq, W, device)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+                "config": {"workload": w.name, "rows_per_gpu": n, "referenced_bytes_per_row": ref_bytes,
+                           "step": "plan+build of every dimension table, then the fused pass"
+                                   + (", then all-reduce of the dense result" if world > 1 else ""),
+                           "l2": "inputs (%.1f GB) exceed the 126 MB L2; no flush needed" % (n * ref_bytes / 1e9),
+                           "parallelism": f"row-sharded x{world}, dimensions replicated", "plan": info.describe()},
+                "effective_gbs": eff_gbs, "pct_of_8tbs": 100.0 * eff_gbs / world / CONTRACT_HBM_GBS,
+                "pct_of_measured_copy_peak": 100.0 * eff_gbs / world / peak,
+                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
+                "clocks": sampler.summary()}
+        if extras is not None:
+            line["other_configs"] = extras
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def run_extras(sjq, W, device):
+    """Run-only timings (tables prebuilt) of the other configurations: min and mean of 10 after a warm-up."""
+    import torch
+
+    out = []
+
+    def timed(w):
+        dims = {d.name: W.device_dim(w, d, device) for d in w.dims}
+        tables = sjq.build_workload_tables(w, dims)
+        fact = W.device_fact(w, device=device)
+        res = sjq.run_workload(w, fact, tables)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ts = []
+        for _ in range(10):
+            e0.record()
+            sjq.run_workload(w, fact, tables, result=res)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        eff = w.n_rows * w.referenced_bytes_per_row() / (min(ts) / 1000.0) / 1e9
+        out.append({"workload": w.name, "rows": w.n_rows, "ms_min": min(ts), "ms_mean": sum(ts) / len(ts),
+                    "rows_per_s": w.n_rows / (min(ts) / 1000.0), "effective_gbs": eff,
+                    "pct_of_8tbs": 100.0 * eff / CONTRACT_HBM_GBS, "status": res.status(),
+                    "plan": res.info.describe()})
+        del fact, tables, dims, res
+        torch.cuda.empty_cache()
+
+    timed(W.config1())
+    timed(W.config2())
+    timed(W.config5())
+    for s in (0.0001, 0.01, 0.1, 0.5, 1.0):
+        for g in (1, 1000, 100000, 1000000):
+            timed(W.config4(600_000_000, s, g))
+    return out
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -225,15 +225,19 @@ typedef struct sjq_result {
 
 /* Tuning and ablation switches; a zeroed struct (or NULL) means defaults. */
 typedef struct sjq_run_opts {
-    int32_t block_threads; /* 0 = default; else 128..1024, multiple of 32 */
+    int32_t block_threads; /* 0 = default (512); else 128..512, multiple of 32 */
     int32_t ctas_per_sm;   /* 0 = as many as fit */
     int32_t eager_loads;   /* 1 = load every column for every row (ablation of lazy loading) */
     int32_t agg_path;      /* 0 auto, 1 shared-memory privatised table, 2 global atomics (DENSE) */
-    int32_t smem_tables;   /* 0 auto, 1 never copy small direct tables into shared memory */
-    int32_t compaction;    /* 0 auto, 1 never, 2 always compact survivors before the sparse tail */
+    int32_t smem_tables;   /* 0 auto (direct tables up to 16 KiB are copied into shared memory), 1 never,
+                              2 every direct table that fits */
+    int32_t compaction;    /* 0 auto; 1 never queue survivors (every stage on thread-owned rows);
+                              2 one queue only (first stage dense, everything else at the final level) */
     int32_t accumulate;    /* 1 = add into the result buffers instead of clearing them first */
     int32_t norder;        /* 0 = library chooses the evaluation order */
     int32_t order[SJQ_MAX_PREDS + SJQ_MAX_JOINS]; /* entry < npreds: predicate index; else npreds + join index */
+    void *event_before; /* optional cudaEvent_t recorded on `stream` right before the fused kernel */
+    void *event_after;  /* optional cudaEvent_t recorded right after it (both or neither) */
     int32_t reserved[8];
 } sjq_run_opts;
 
@@ -242,7 +246,8 @@ typedef struct sjq_run_info {
     int32_t nstages;
     int32_t order[SJQ_MAX_PREDS + SJQ_MAX_JOINS + 8]; /* as in sjq_run_opts.order; -1 = plain column load */
     int32_t stage_in_smem[SJQ_MAX_PREDS + SJQ_MAX_JOINS + 8];
-    int32_t first_sparse_stage; /* stages >= this run on compacted survivors; nstages = none */
+    int32_t first_sparse_stage; /* number of queue-fed levels: stage 0 is dense, stages 1 .. this-1 are
+                                   queue-fed filters, later stages run at the final level; 0 = no queues */
     int32_t agg_path;           /* 0 scalar registers, 1 shared-memory table, 2 global atomics, 3 global hash */
     int32_t grid, block;
     int32_t smem_bytes;
@@ -271,6 +276,33 @@ sjq_status sjq_run_workspace_bytes(const sjq_result_spec *spec, size_t *bytes);
 sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *preds, int npreds, const sjq_join *joins,
                    int njoins, const sjq_key_expr *key, const sjq_agg_expr *agg, const sjq_result_spec *spec,
                    const sjq_result *out, const sjq_run_opts *opts, void *stream, sjq_run_info *info);
+
+/*
+ * The same query over fact columns that live in HOST memory (page-locked for
+ * full copy speed): the table is cut into chunks of `chunk_rows` rows; each
+ * chunk's columns are copied into one half of the device staging buffer while
+ * the previous chunk is being processed from the other half (two internal
+ * streams, ordered after and joined back into `stream`), every chunk runs
+ * sjq_run with `accumulate` into `out`, and at the end the result arrays are
+ * copied to the host.
+ *   fact_host     columns whose `data` are HOST pointers (n = total rows)
+ *   staging_dev   device buffer of at least 2 * chunk_rows * (sum of column
+ *                 widths, each rounded up to 16 bytes per chunk) bytes
+ *   chunk_rows    rows per chunk, a positive multiple of 4
+ *   host_sums / host_counts / host_keys / host_n_groups / host_status
+ *                 host destinations (page-locked for an asynchronous copy) of
+ *                 the arrays of `out`; NULL = do not copy that one.  HASHED
+ *                 results copy `capacity` entries.
+ * Every column is copied whole: lazy loading cannot skip bytes that have to
+ * cross the bus before the predicates are known.  Enqueues only; the caller
+ * synchronises `stream`.  Errors as sjq_run, plus BUFFER_SMALL.
+ */
+sjq_status sjq_run_host(const sjq_col *fact_host, int nfact, const sjq_pred *preds, int npreds,
+                        const sjq_join *joins, int njoins, const sjq_key_expr *key, const sjq_agg_expr *agg,
+                        const sjq_result_spec *spec, const sjq_result *out, const sjq_run_opts *opts,
+                        void *staging_dev, size_t staging_bytes, int64_t chunk_rows, int64_t *host_sums,
+                        int64_t *host_counts, int64_t *host_keys, int64_t *host_n_groups, int32_t *host_status,
+                        void *stream);
 
 const char *sjq_strerror(sjq_status status);
 const char *sjq_version(void);

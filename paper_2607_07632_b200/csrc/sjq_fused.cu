@@ -1,128 +1,264 @@
 // The fused probe kernel: one pass over the fact table.
 //
-// Execution model (Section 3.2 of the paper, "grid-stride persistent
-// threads"): a machine-sized grid; each thread owns four consecutive rows of a
-// tile and strides over tiles, so one 128-bit load brings the four values of a
-// column; later columns are loaded only while at least one of the thread's
-// rows is still alive (lazy loading, Section 3.2 "Latency-hidden join"), a
-// probe is a range-checked single load from a direct-mapped table or a bounded
-// linear probe of an open-addressing table (Section 3.3), and the terminal is
-// a register accumulator, a shared-memory privatised group table or global
-// atomics (Section 3.3 "Shared-memory privatized group-by").
+// Execution model.  A machine-sized grid of persistent blocks strides over
+// tiles of the fact table (Section 3.2 of the paper, "grid-stride persistent
+// threads").  Every warp runs a small push pipeline of its own:
+//
+//  level 0   (dense) every thread owns kSlots groups of four consecutive
+//            rows, so one 128-bit load brings four values of the first
+//            column and a warp reads 512 contiguous bytes; the first stage
+//            keeps one bit per row.  The sixteen loads and probes of a thread
+//            are independent, which keeps enough bytes in flight to cover
+//            HBM latency.
+//  level l   the survivors of level l-1 are compacted (popcount + warp scan)
+//            into queue l of the warp in shared memory; whenever a queue
+//            holds a full batch (kRows per lane) the warp runs the next filter
+//            stage on it, loading that stage's column with one 4-byte load per
+//            surviving row only (lazy loading, Section 3.2: a later column is
+//            never read for an eliminated row), and pushes the survivors on.
+//  last      the final level gathers the group-key payloads and the measure
+//            columns of the survivors into register accumulators and runs the
+//            terminal.
+//
+// A probe is a range-checked single load from a direct-mapped table (global or
+// staged in shared memory) or a bounded lock-step linear probe of an
+// open-addressing table (Section 3.3).  The terminal is a register accumulator
+// with one atomic per block, a shared-memory privatised group table flushed
+// with one atomic per touched group per block, global atomics, or a global
+// group hash table (Section 3.3 "Shared-memory privatized group-by").
+#include <type_traits>
+
 #include "sjq_run.cuh"
 
 namespace sjq {
 
 namespace {
 
-__device__ __forceinline__ int4 ld_stream16(const void *p)
-{
-    return __ldcs(static_cast<const int4 *>(p));
-}
-__device__ __forceinline__ longlong2 ld_stream16ll(const void *p)
-{
-    return __ldcs(static_cast<const longlong2 *>(p));
-}
-
-// Probe of one table with key v.  Returns hit; on a hit `code` holds the
-// packed payload code.  SMEM: the direct table was staged into shared memory.
 template <typename T>
-__device__ __forceinline__ bool probe(const DStage &S, const unsigned char *smem, T v, uint64_t &code)
+struct Vec4;
+template <>
+struct Vec4<int32_t> {
+    static __device__ __forceinline__ void load(const int32_t *p, int32_t *v)
+    {
+        const int4 a = __ldcs(reinterpret_cast<const int4 *>(p));
+        v[0] = a.x, v[1] = a.y, v[2] = a.z, v[3] = a.w;
+    }
+};
+template <>
+struct Vec4<int64_t> {
+    static __device__ __forceinline__ void load(const int64_t *p, int64_t *v)
+    {
+        const longlong2 a = __ldcs(reinterpret_cast<const longlong2 *>(p));
+        const longlong2 b = __ldcs(reinterpret_cast<const longlong2 *>(p) + 1);
+        v[0] = a.x, v[1] = a.y, v[2] = b.x, v[3] = b.y;
+    }
+};
+
+template <typename T>
+struct Index {
+    typedef uint64_t type;
+};
+template <>
+struct Index<int32_t> {
+    typedef uint32_t type;
+};
+
+// ------------------------------------------------------------------ stage bodies
+// Each body takes the values v[0..NR) of the rows whose bit is set in m and
+// returns the mask of rows that pass.  Values of rows outside m are ignored.
+
+template <typename T, int NR>
+__device__ __forceinline__ uint32_t body_pred_range(const DStage &S, const T (&v)[NR], uint32_t m)
 {
-    if (S.tkind <= SJQ_TABLE_DIRECT_U64) {
-        const uint64_t idx = (uint64_t)(int64_t)v - (uint64_t)S.kmin;
-        if (idx >= S.span) return false; // outside the key range: a miss, never an access
-        if (S.in_smem) {
-            const unsigned char *t = smem + S.smem_off;
-            switch (S.tkind) {
-            case SJQ_TABLE_DIRECT_BITMAP:
-                return (reinterpret_cast<const uint32_t *>(t)[idx >> 5] >> (idx & 31)) & 1u;
-            case SJQ_TABLE_DIRECT_U8: code = t[idx]; return code != 0xFFu;
-            case SJQ_TABLE_DIRECT_U16: code = reinterpret_cast<const uint16_t *>(t)[idx]; return code != 0xFFFFu;
-            case SJQ_TABLE_DIRECT_U32: code = reinterpret_cast<const uint32_t *>(t)[idx]; return code != 0xFFFFFFFFu;
-            default: code = reinterpret_cast<const uint64_t *>(t)[idx]; return code != ~0ULL;
-            }
+    uint32_t pass = 0;
+    if (sizeof(T) == 4) {
+        if (!S.never) {
+#pragma unroll
+            for (int i = 0; i < NR; ++i)
+                pass |= (uint32_t)(((uint32_t)v[i] - (uint32_t)S.lo32) <= S.width32) << i;
         }
-        switch (S.tkind) {
-        case SJQ_TABLE_DIRECT_BITMAP:
-            return (__ldg(static_cast<const uint32_t *>(S.tab) + (idx >> 5)) >> (idx & 31)) & 1u;
-        case SJQ_TABLE_DIRECT_U8: code = __ldg(static_cast<const uint8_t *>(S.tab) + idx); return code != 0xFFu;
-        case SJQ_TABLE_DIRECT_U16: code = __ldg(static_cast<const uint16_t *>(S.tab) + idx); return code != 0xFFFFu;
-        case SJQ_TABLE_DIRECT_U32:
-            code = __ldg(static_cast<const uint32_t *>(S.tab) + idx);
-            return code != 0xFFFFFFFFu;
-        default: code = __ldg(static_cast<const uint64_t *>(S.tab) + idx); return code != ~0ULL;
+    } else {
+#pragma unroll
+        for (int i = 0; i < NR; ++i) pass |= (uint32_t)(((int64_t)v[i] >= S.lo) & ((int64_t)v[i] <= S.hi)) << i;
+    }
+    if (S.neg) pass = ~pass;
+    return m & pass;
+}
+
+template <typename T, int NR>
+__device__ __forceinline__ uint32_t body_pred_set(const RunParams &P, const DStage &S, const T (&v)[NR], uint32_t m)
+{
+    uint32_t pass = 0;
+    for (int k = 0; k < S.nset; ++k) {
+        const int64_t lit = P.sets[S.set_idx][k];
+#pragma unroll
+        for (int i = 0; i < NR; ++i) pass |= (uint32_t)((int64_t)v[i] == lit) << i;
+    }
+    return m & pass;
+}
+
+template <typename T, int OP, bool SMEM, int NR, bool WANT>
+__device__ __forceinline__ uint32_t body_direct(const DStage &S, const unsigned char *smem, const T (&v)[NR],
+                                                uint32_t m, uint64_t (&code)[NR])
+{
+    const unsigned char *base = SMEM ? smem + S.smem_off : static_cast<const unsigned char *>(S.tab);
+    typename Index<T>::type idx[NR];
+    uint32_t in = 0;
+#pragma unroll
+    for (int i = 0; i < NR; ++i) {
+        if (sizeof(T) == 4) {
+            const uint32_t d = (uint32_t)v[i] - (uint32_t)S.kmin32;
+            idx[i] = d;
+            in |= (uint32_t)(d <= S.last32) << i;
+        } else {
+            const uint64_t d = (uint64_t)v[i] - (uint64_t)S.kmin;
+            idx[i] = d;
+            in |= (uint32_t)(d <= S.last) << i;
         }
     }
-    if (S.tkind == SJQ_TABLE_HASH_I64) {
-        const int64_t k = (int64_t)v;
-        if (k == kEmptyKey64) return false;
-        const int64_t *keys = static_cast<const int64_t *>(S.tab);
-        uint64_t slot = hash64((uint64_t)k) & S.hmask;
-        for (uint64_t it = 0; it <= S.hmask; ++it) {
-            const int64_t cur = __ldg(keys + slot);
-            if (cur == k) {
-                if (S.codes)
-                    code = (S.code_bits == 64) ? __ldg(static_cast<const uint64_t *>(S.codes) + slot)
-                                         : (uint64_t)__ldg(static_cast<const uint32_t *>(S.codes) + slot);
-                return true;
+    in &= m; // a key outside the table's range is a miss, never an access
+    uint32_t hit = 0;
+    if (OP == OP_DIRECT_BITMAP) {
+        uint32_t w[NR];
+#pragma unroll
+        for (int i = 0; i < NR; ++i) {
+            w[i] = 0;
+            if ((in >> i) & 1u) {
+                const uint32_t *p = reinterpret_cast<const uint32_t *>(base) + (idx[i] >> 5);
+                w[i] = SMEM ? *p : __ldg(p);
             }
-            if (cur == kEmptyKey64) return false;
-            slot = (slot + 1) & S.hmask;
         }
-        return false;
+#pragma unroll
+        for (int i = 0; i < NR; ++i) hit |= ((w[i] >> (idx[i] & 31)) & 1u) << i;
+        return in & hit;
     }
-    { // HASH_I32
-        const int32_t k = (int32_t)v;
-        if ((int64_t)v != (int64_t)k || k == kEmptyKey32) return false;
-        const int32_t *keys = static_cast<const int32_t *>(S.tab);
-        uint64_t slot = hash64((uint64_t)(int64_t)k) & S.hmask;
-        for (uint64_t it = 0; it <= S.hmask; ++it) {
-            const int32_t cur = __ldg(keys + slot);
-            if (cur == k) {
-                if (S.codes)
-                    code = (S.code_bits == 64) ? __ldg(static_cast<const uint64_t *>(S.codes) + slot)
-                                         : (uint64_t)__ldg(static_cast<const uint32_t *>(S.codes) + slot);
-                return true;
+    uint64_t c[NR];
+#pragma unroll
+    for (int i = 0; i < NR; ++i) {
+        c[i] = ~0ULL;
+        if ((in >> i) & 1u) {
+            if (OP == OP_DIRECT_U8) {
+                const uint8_t *p = base + idx[i];
+                c[i] = SMEM ? *p : __ldg(p);
+            } else if (OP == OP_DIRECT_U16) {
+                const uint16_t *p = reinterpret_cast<const uint16_t *>(base) + idx[i];
+                c[i] = SMEM ? *p : __ldg(p);
+            } else if (OP == OP_DIRECT_U32) {
+                const uint32_t *p = reinterpret_cast<const uint32_t *>(base) + idx[i];
+                c[i] = SMEM ? *p : __ldg(p);
+            } else {
+                const uint64_t *p = reinterpret_cast<const uint64_t *>(base) + idx[i];
+                c[i] = SMEM ? *p : __ldg(p);
             }
-            if (cur == kEmptyKey32) return false;
-            slot = (slot + 1) & S.hmask;
         }
-        return false;
+    }
+    const uint64_t miss = OP == OP_DIRECT_U8 ? 0xFFull : OP == OP_DIRECT_U16 ? 0xFFFFull
+                          : OP == OP_DIRECT_U32 ? 0xFFFFFFFFull : ~0ULL;
+#pragma unroll
+    for (int i = 0; i < NR; ++i) {
+        hit |= (uint32_t)(c[i] != miss) << i;
+        if (WANT) code[i] = c[i];
+    }
+    return in & hit;
+}
+
+// Open addressing, linear probing, all rows of the thread in lock step so that
+// their loads overlap; bounded by the slot count.
+template <typename T, int NR, bool WANT>
+__device__ __forceinline__ uint32_t body_hash(const DStage &S, const T (&v)[NR], uint32_t m, uint64_t (&code)[NR])
+{
+    const T empty = sizeof(T) == 4 ? (T)kEmptyKey32 : (T)kEmptyKey64;
+    const T *keys = static_cast<const T *>(S.tab);
+    const uint32_t hmask = (uint32_t)S.hmask;
+    uint32_t slot[NR];
+    uint32_t pending = 0;
+#pragma unroll
+    for (int i = 0; i < NR; ++i) {
+        slot[i] = (uint32_t)hash64((uint64_t)(int64_t)v[i]) & hmask;
+        pending |= (uint32_t)(v[i] != empty) << i; // the reserved marker is never a key
+    }
+    pending &= m;
+    uint32_t hit = 0;
+    for (uint32_t it = 0; pending != 0 && it <= hmask; ++it) {
+        T cur[NR];
+#pragma unroll
+        for (int i = 0; i < NR; ++i) {
+            cur[i] = empty;
+            if ((pending >> i) & 1u) cur[i] = __ldg(keys + slot[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < NR; ++i) {
+            if ((pending >> i) & 1u) {
+                if (cur[i] == v[i]) {
+                    hit |= 1u << i;
+                    pending &= ~(1u << i);
+                } else if (cur[i] == empty) {
+                    pending &= ~(1u << i);
+                } else {
+                    slot[i] = (slot[i] + 1) & hmask;
+                }
+            }
+        }
+    }
+    if (WANT && S.codes) {
+#pragma unroll
+        for (int i = 0; i < NR; ++i) {
+            code[i] = 0;
+            if ((hit >> i) & 1u)
+                code[i] = S.code_bits == 64 ? __ldg(static_cast<const uint64_t *>(S.codes) + slot[i])
+                                            : (uint64_t)__ldg(static_cast<const uint32_t *>(S.codes) + slot[i]);
+        }
+    }
+    return hit;
+}
+
+template <typename T, int NR, bool WANT>
+__device__ __forceinline__ uint32_t run_stage(const RunParams &P, const DStage &S, const unsigned char *smem,
+                                              const T (&v)[NR], uint32_t m, uint64_t (&code)[NR])
+{
+    switch (S.op * 2 + S.in_smem) {
+    case OP_PRED_RANGE * 2: return body_pred_range<T, NR>(S, v, m);
+    case OP_PRED_SET * 2: return body_pred_set<T, NR>(P, S, v, m);
+    case OP_DIRECT_BITMAP * 2: return body_direct<T, OP_DIRECT_BITMAP, false, NR, WANT>(S, smem, v, m, code);
+    case OP_DIRECT_BITMAP * 2 + 1: return body_direct<T, OP_DIRECT_BITMAP, true, NR, WANT>(S, smem, v, m, code);
+    case OP_DIRECT_U8 * 2: return body_direct<T, OP_DIRECT_U8, false, NR, WANT>(S, smem, v, m, code);
+    case OP_DIRECT_U8 * 2 + 1: return body_direct<T, OP_DIRECT_U8, true, NR, WANT>(S, smem, v, m, code);
+    case OP_DIRECT_U16 * 2: return body_direct<T, OP_DIRECT_U16, false, NR, WANT>(S, smem, v, m, code);
+    case OP_DIRECT_U16 * 2 + 1: return body_direct<T, OP_DIRECT_U16, true, NR, WANT>(S, smem, v, m, code);
+    case OP_DIRECT_U32 * 2: return body_direct<T, OP_DIRECT_U32, false, NR, WANT>(S, smem, v, m, code);
+    case OP_DIRECT_U32 * 2 + 1: return body_direct<T, OP_DIRECT_U32, true, NR, WANT>(S, smem, v, m, code);
+    case OP_DIRECT_U64 * 2: return body_direct<T, OP_DIRECT_U64, false, NR, WANT>(S, smem, v, m, code);
+    case OP_DIRECT_U64 * 2 + 1: return body_direct<T, OP_DIRECT_U64, true, NR, WANT>(S, smem, v, m, code);
+    case OP_HASH32 * 2:
+    case OP_HASH64 * 2: return body_hash<T, NR, WANT>(S, v, m, code);
+    default: return m; // OP_LOAD
     }
 }
 
-// One stage applied to one row: filter, then feed the accumulators.
-template <typename T, bool MUL>
-__device__ __forceinline__ bool apply(const DStage &S, const unsigned char *smem, T v, int64_t &key, int64_t &X,
-                                      int64_t &Y)
+// ------------------------------------------------------------------ accumulators
+
+template <bool MUL>
+__device__ __forceinline__ void accumulate(const DStage &S, int64_t raw, uint64_t code, int64_t &key, int64_t &X,
+                                           int64_t &Y)
 {
-    uint64_t code = 0;
-    bool pass = true;
-    if (S.kind == ST_PRED) pass = pred_eval<T>(S.pred, v);
-    else if (S.kind == ST_PROBE) pass = probe<T>(S, smem, v, code);
-    if (pass && S.acc) {
-        const uint32_t acc = S.acc;
-        if (acc & 0x7u) {
-            const int64_t raw = (int64_t)v;
-            if (acc & 1u) key += S.mult[0] * raw;
-            if (acc & 2u) X += S.mult[1] * raw;
-            if (MUL && (acc & 4u)) Y += S.mult[2] * raw;
-        }
-        if (acc & 0x38u) {
-            const int64_t p0 = (int64_t)(code & S.pmask0) + S.pmin0;
-            if (acc & 8u) key += S.mult[3] * p0;
-            if (acc & 16u) X += S.mult[4] * p0;
-            if (MUL && (acc & 32u)) Y += S.mult[5] * p0;
-        }
-        if (acc & 0x1C0u) {
-            const int64_t p1 = (int64_t)(code >> S.pbits0) + S.pmin1;
-            if (acc & 64u) key += S.mult[6] * p1;
-            if (acc & 128u) X += S.mult[7] * p1;
-            if (MUL && (acc & 256u)) Y += S.mult[8] * p1;
-        }
+    const uint32_t acc = S.acc;
+    if (acc & 0x7u) {
+        if (acc & 1u) key += S.mult[0] * raw;
+        if (acc & 2u) X += S.mult[1] * raw;
+        if (MUL && (acc & 4u)) Y += S.mult[2] * raw;
     }
-    return pass;
+    if (acc & 0x38u) {
+        const int64_t p0 = (int64_t)(code & S.pmask0) + S.pmin0;
+        if (acc & 8u) key += S.mult[3] * p0;
+        if (acc & 16u) X += S.mult[4] * p0;
+        if (MUL && (acc & 32u)) Y += S.mult[5] * p0;
+    }
+    if (acc & 0x1C0u) {
+        const int64_t p1 = (int64_t)(code >> S.pbits0) + S.pmin1;
+        if (acc & 64u) key += S.mult[6] * p1;
+        if (acc & 128u) X += S.mult[7] * p1;
+        if (MUL && (acc & 256u)) Y += S.mult[8] * p1;
+    }
 }
 
 __device__ __forceinline__ int64_t reduce_key(const RunParams &P, int64_t g)
@@ -171,6 +307,19 @@ __device__ __forceinline__ void hash_aggregate(const RunParams &P, int64_t g, in
     atomicAdd(reinterpret_cast<unsigned long long *>(P.counts) + slot, 1ull);
 }
 
+// 64-bit add into shared memory as two native 32-bit atomics: the low word's
+// returned old value tells this thread whether its own add carried, so every
+// carry is propagated exactly once and the 64-bit total is exact.
+__device__ __forceinline__ void smem_add64(unsigned long long *cell, uint64_t val)
+{
+    unsigned int *w = reinterpret_cast<unsigned int *>(cell);
+    const unsigned int lo = (unsigned int)val;
+    unsigned int hi = (unsigned int)(val >> 32);
+    const unsigned int old = atomicAdd(w, lo);
+    hi += (unsigned int)((old + lo) < old);
+    if (hi) atomicAdd(w + 1, hi);
+}
+
 template <int AGG, bool MUL>
 __device__ __forceinline__ void terminal(const RunParams &P, unsigned char *smem, int64_t key, int64_t X, int64_t Y,
                                          int64_t &lsum, int64_t &lcnt)
@@ -199,24 +348,181 @@ __device__ __forceinline__ void terminal(const RunParams &P, unsigned char *smem
     }
     if (AGG == AGG_SMEM) {
         unsigned long long *ss = reinterpret_cast<unsigned long long *>(smem + P.smem_groups);
-        atomicAdd(ss + g, (unsigned long long)val);
-        if (P.want_count) atomicAdd(ss + P.num_groups + g, 1ull);
+        smem_add64(ss + g, (uint64_t)val);
+        if (P.want_count) smem_add64(ss + P.num_groups + g, 1ull);
     } else {
         atomicAdd(reinterpret_cast<unsigned long long *>(P.sums) + g, (unsigned long long)val);
         if (P.want_count) atomicAdd(reinterpret_cast<unsigned long long *>(P.counts) + g, 1ull);
     }
 }
 
+// ------------------------------------------------------------------ row batches
+// A batch is up to kRows rows per lane, named by 32-bit offsets from a base
+// row that is uniform over the warp (so a column address costs one multiply-
+// add per row).  CONTIG: the lane owns four consecutive rows (one 128-bit
+// load); otherwise the rows are survivors popped from a queue (one 4- or
+// 8-byte load each).
+
+template <typename T, bool CONTIG>
+__device__ __forceinline__ void load_rows(const DStage &S, int64_t base, const uint32_t (&off)[kRows], uint32_t valid,
+                                          uint32_t need, T (&v)[kRows])
+{
+    const T *c = static_cast<const T *>(S.col) + base;
+    if (CONTIG && valid == 0xFu) {
+        Vec4<T>::load(c + off[0], v);
+        return;
+    }
+#pragma unroll
+    for (int k = 0; k < kRows; ++k) {
+        v[k] = 0;
+        if ((need >> k) & 1u) v[k] = __ldg(c + off[k]);
+    }
+}
+
+// One pure filter stage on a batch: returns the mask of rows that pass.
+__device__ __forceinline__ uint32_t filter_rows(const RunParams &P, const DStage &S, const unsigned char *smem,
+                                                int64_t base, const uint32_t (&off)[kRows], uint32_t valid)
+{
+    uint64_t unused[kRows];
+    if (S.is64) {
+        int64_t v[kRows];
+        load_rows<int64_t, false>(S, base, off, valid, valid, v);
+        return run_stage<int64_t, kRows, false>(P, S, smem, v, valid, unused);
+    }
+    int32_t v[kRows];
+    load_rows<int32_t, false>(S, base, off, valid, valid, v);
+    return run_stage<int32_t, kRows, false>(P, S, smem, v, valid, unused);
+}
+
+// Stages [first, nstages) with accumulators, then the terminal.  The column of
+// the next stage is requested before the current stage's probe is resolved, so
+// a stage costs one memory latency, not two.
+template <int AGG, bool MUL, bool CONTIG>
+__device__ __forceinline__ void final_rows(const RunParams &P, const DStage *st, unsigned char *smem, int first,
+                                           int64_t base, const uint32_t (&off)[kRows], uint32_t valid, int64_t &lsum,
+                                           int64_t &lcnt)
+{
+    uint32_t m = valid;
+    int64_t key[kRows], X[kRows], Y[kRows];
+#pragma unroll
+    for (int k = 0; k < kRows; ++k) {
+        key[k] = P.key_offset;
+        X[k] = 0;
+        Y[k] = 0;
+    }
+    int32_t vnext[kRows];
+    bool have_next = false;
+    for (int s = first; s < P.nstages; ++s) {
+        const DStage &S = st[s];
+        const uint32_t need = P.eager ? valid : m;
+        if (!need) break;
+        uint64_t code[kRows];
+#pragma unroll
+        for (int k = 0; k < kRows; ++k) code[k] = 0;
+        if (S.is64) {
+            int64_t v[kRows];
+            load_rows<int64_t, CONTIG>(S, base, off, valid, need, v);
+            have_next = false;
+            m = run_stage<int64_t, kRows, true>(P, S, smem, v, m, code);
+            if (S.acc) {
+#pragma unroll
+                for (int k = 0; k < kRows; ++k)
+                    if ((m >> k) & 1u) accumulate<MUL>(S, v[k], code[k], key[k], X[k], Y[k]);
+            }
+        } else {
+            int32_t v[kRows];
+            if (have_next) {
+#pragma unroll
+                for (int k = 0; k < kRows; ++k) v[k] = vnext[k];
+            } else {
+                load_rows<int32_t, CONTIG>(S, base, off, valid, need, v);
+            }
+            have_next = (s + 1 < P.nstages) && !st[s + 1].is64;
+            if (have_next) load_rows<int32_t, CONTIG>(st[s + 1], base, off, valid, need, vnext);
+            m = run_stage<int32_t, kRows, true>(P, S, smem, v, m, code);
+            if (S.acc) {
+#pragma unroll
+                for (int k = 0; k < kRows; ++k)
+                    if ((m >> k) & 1u) accumulate<MUL>(S, (int64_t)v[k], code[k], key[k], X[k], Y[k]);
+            }
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < kRows; ++k)
+        if ((m >> k) & 1u) terminal<AGG, MUL>(P, smem, key[k], X[k], Y[k], lsum, lcnt);
+}
+
+// ------------------------------------------------------------------ level 0
+// The first stage on the thread's own kSlots groups of four consecutive rows
+// of a tile.  FULL: the whole tile lies inside the table (no bounds masks).
+template <typename T, bool FULL>
+__device__ __forceinline__ uint32_t dense_stage(const RunParams &P, const DStage &S, const unsigned char *smem,
+                                                int64_t row0, int32_t slot_stride, uint32_t valid)
+{
+    T v[kDenseRows];
+    const T *c = static_cast<const T *>(S.col) + row0;
+#pragma unroll
+    for (int u = 0; u < kSlots; ++u) {
+        if (FULL) {
+            Vec4<T>::load(c + u * slot_stride, &v[4 * u]);
+        } else {
+            const uint32_t nv = (valid >> (4 * u)) & 0xFu;
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                v[4 * u + r] = 0;
+                if ((nv >> r) & 1u) v[4 * u + r] = __ldcs(c + u * slot_stride + r);
+            }
+        }
+    }
+    uint64_t unused[kDenseRows];
+    return run_stage<T, kDenseRows, false>(P, S, smem, v, valid, unused);
+}
+
+// ------------------------------------------------------------------ per-warp queues
+// Queue l of a warp (a ring of 32-bit row offsets in shared memory) holds the
+// rows that passed stages 0 .. l.  The level fed by queue l runs filter stage
+// l+1 and pushes to queue l+1, or, for the last queue, runs the remaining
+// stages and the terminal.  Heads and counts live in registers and are
+// selected without indexing so that they never spill to local memory.
+struct QueueState {
+    uint32_t h0, h1, h2, c0, c1, c2;
+    __device__ __forceinline__ uint32_t head(int l) const { return l == 0 ? h0 : (l == 1 ? h1 : h2); }
+    __device__ __forceinline__ uint32_t count(int l) const { return l == 0 ? c0 : (l == 1 ? c1 : c2); }
+    __device__ __forceinline__ void set_head(int l, uint32_t v)
+    {
+        h0 = l == 0 ? v : h0;
+        h1 = l == 1 ? v : h1;
+        h2 = l == 2 ? v : h2;
+    }
+    __device__ __forceinline__ void set_count(int l, uint32_t v)
+    {
+        c0 = l == 0 ? v : c0;
+        c1 = l == 1 ? v : c1;
+        c2 = l == 2 ? v : c2;
+    }
+};
+__device__ __forceinline__ uint32_t queue_cap(int l) { return l == 0 ? (uint32_t)kQueue0Cap : (uint32_t)kQueueCap; }
+__device__ __forceinline__ uint32_t queue_base(int l) { return l == 0 ? 0u : (uint32_t)(kQueue0Cap + (l - 1) * kQueueCap); }
+
 template <int AGG, bool MUL>
-__global__ void __launch_bounds__(1024) fused_kernel(const __grid_constant__ RunParams P)
+__global__ void __launch_bounds__(512, 2) fused_kernel(const __grid_constant__ RunParams P)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
 
-    // Stage small direct tables into shared memory (one copy per CTA).
+    // Stage descriptors and small direct tables -> shared memory (once per block).
+    DStage *st = reinterpret_cast<DStage *>(smem + P.smem_stages);
+    {
+        const uint32_t words = (uint32_t)(P.nstages * sizeof(DStage) / 8);
+        const uint64_t *src = reinterpret_cast<const uint64_t *>(&P.st[0]);
+        uint64_t *dst = reinterpret_cast<uint64_t *>(st);
+        for (uint32_t i = tid; i < words; i += blockDim.x) dst[i] = src[i];
+    }
     for (int s = 0; s < P.nstages; ++s) {
         const DStage &S = P.st[s];
-        if (S.kind == ST_PROBE && S.in_smem) {
+        if (S.in_smem) {
             const uint4 *src = static_cast<const uint4 *>(S.tab);
             uint4 *dst = reinterpret_cast<uint4 *>(smem + S.smem_off);
             for (uint32_t i = tid; i < S.tab_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
@@ -230,59 +536,150 @@ __global__ void __launch_bounds__(1024) fused_kernel(const __grid_constant__ Run
     __syncthreads();
 
     int64_t lsum = 0, lcnt = 0;
-    const int64_t tile_rows = (int64_t)blockDim.x * 4;
-    const int64_t ntiles = (P.n + tile_rows - 1) / tile_rows;
-    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-        const int64_t row0 = tile * tile_rows + 4 * (int64_t)tid;
-        const int64_t rem = P.n - row0;
-        const uint32_t valid = rem >= 4 ? 0xFu : (rem > 0 ? ((1u << (int)rem) - 1u) : 0u);
-        uint32_t alive = valid;
-        int64_t key[4], X[4], Y[4];
+
+    if (P.nq == 0) {
+        // No queue: every stage runs on the thread's own four consecutive rows.
+        const int64_t tile_rows = (int64_t)blockDim.x * kRows;
+        const int64_t ntiles = (P.n + tile_rows - 1) / tile_rows;
+        uint32_t off[kRows];
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            key[r] = P.key_offset;
-            X[r] = 0;
-            Y[r] = 0;
+        for (int k = 0; k < kRows; ++k) off[k] = (uint32_t)(4 * tid + k);
+        for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+            const int64_t base = tile * tile_rows;
+            const int64_t rem = P.n - base - 4 * (int64_t)tid;
+            const uint32_t valid = rem >= 4 ? 0xFu : (rem > 0 ? ((1u << (int)rem) - 1u) : 0u);
+            final_rows<AGG, MUL, true>(P, st, smem, 0, base, off, valid, lsum, lcnt);
         }
-        for (int s = 0; s < P.nstages; ++s) {
-            const DStage &S = P.st[s];
-            const uint32_t need = P.eager ? valid : alive;
-            if (!need) continue;
-            if (S.is64) {
-                int64_t v[4] = {0, 0, 0, 0};
-                const int64_t *c = static_cast<const int64_t *>(S.col) + row0;
-                if (valid == 0xFu) {
-                    const longlong2 a = ld_stream16ll(c), b = ld_stream16ll(c + 2);
-                    v[0] = a.x, v[1] = a.y, v[2] = b.x, v[3] = b.y;
+    } else {
+        const int nq = P.nq;
+        uint32_t *const qmem = reinterpret_cast<uint32_t *>(smem + P.smem_queue) +
+                               warp * (kQueue0Cap + (nq - 1) * kQueueCap);
+        QueueState Q{0, 0, 0, 0, 0, 0};
+        const bool wide = P.n > 0xFFFFFFFFll; // offsets are tile-relative and the queues are flushed per tile
+        const int32_t slot_stride = (int32_t)blockDim.x * 4;
+        const int32_t tile_rows = slot_stride * kSlots;
+        const uint32_t ntiles = (uint32_t)((P.n + tile_rows - 1) / tile_rows); // host checks n / tile_rows < 2^31
+        int64_t qbase = 0;
+        uint32_t tile = blockIdx.x;
+        bool flushing = false;
+
+        // One loop, one call site per piece of work: pick the deepest queue holding a full
+        // batch (so that a push never meets a full queue); else filter the next tile and push
+        // its survivors; at the end drain what is left.
+        for (;;) {
+            int l = (nq >= 3 && Q.c2 >= (uint32_t)kBatch) ? 2
+                    : (nq >= 2 && Q.c1 >= (uint32_t)kBatch) ? 1
+                    : (Q.c0 >= (uint32_t)kBatch)            ? 0
+                                                            : -1;
+            uint32_t nb = kBatch;
+            if (l < 0) {
+                if (flushing) {
+                    l = Q.c0 ? 0 : (Q.c1 ? 1 : (Q.c2 ? 2 : -1));
+                    if (l < 0) {
+                        flushing = false;
+                        if (tile >= ntiles) break;
+                        continue;
+                    }
+                    nb = Q.count(l) < (uint32_t)kBatch ? Q.count(l) : (uint32_t)kBatch;
+                } else if (tile < ntiles) {
+                    // level 0: the first stage on the thread's own rows of the next tile
+                    const int64_t tile_base = (int64_t)tile * tile_rows;
+                    const int64_t row0 = tile_base + 4 * tid;
+                    if (wide) qbase = tile_base;
+                    const DStage &S = st[0];
+                    uint32_t alive;
+                    if (tile_base + tile_rows <= P.n) {
+                        alive = S.is64 ? dense_stage<int64_t, true>(P, S, smem, row0, slot_stride, 0xFFu)
+                                       : dense_stage<int32_t, true>(P, S, smem, row0, slot_stride, 0xFFu);
+                    } else {
+                        uint32_t valid = 0;
+#pragma unroll
+                        for (int k = 0; k < kSlots; ++k) {
+                            const int64_t rem = P.n - (row0 + k * slot_stride);
+                            const uint32_t nv = rem >= 4 ? 0xFu : (rem > 0 ? ((1u << (int)rem) - 1u) : 0u);
+                            valid |= nv << (4 * k);
+                        }
+                        alive = S.is64 ? dense_stage<int64_t, false>(P, S, smem, row0, slot_stride, valid)
+                                       : dense_stage<int32_t, false>(P, S, smem, row0, slot_stride, valid);
+                    }
+                    // compact the warp's survivors into queue 0
+                    const uint32_t mine = (uint32_t)__popc(alive);
+                    uint32_t incl = mine;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+                        if (lane >= o) incl += t;
+                    }
+                    const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
+                    if (tot) {
+                        uint32_t pos = Q.h0 + Q.c0 + incl - mine;
+                        const uint32_t off0 = (uint32_t)(row0 - qbase);
+#pragma unroll
+                        for (int k = 0; k < kDenseRows; ++k) {
+                            if ((alive >> k) & 1u) {
+                                qmem[pos & (kQueue0Cap - 1)] = off0 + (uint32_t)((k >> 2) * slot_stride + (k & 3));
+                                ++pos;
+                            }
+                        }
+                        Q.c0 += tot;
+                        __syncwarp();
+                    }
+                    tile += gridDim.x;
+                    if (wide) flushing = true;
+                    continue;
                 } else {
-#pragma unroll
-                    for (int r = 0; r < 4; ++r)
-                        if ((valid >> r) & 1u) v[r] = __ldcs(c + r);
+                    if ((Q.c0 | Q.c1 | Q.c2) == 0) break;
+                    flushing = true;
+                    continue;
                 }
+            }
+
+            // Run one batch of nb rows at the level fed by queue l.
+            uint32_t off[kRows];
+            uint32_t valid = 0;
+            {
+                const uint32_t *q = qmem + queue_base(l);
+                const uint32_t h = Q.head(l), cap = queue_cap(l);
 #pragma unroll
-                for (int r = 0; r < 4; ++r)
-                    if ((alive >> r) & 1u)
-                        if (!apply<int64_t, MUL>(S, smem, v[r], key[r], X[r], Y[r])) alive &= ~(1u << r);
+                for (int k = 0; k < kRows; ++k) {
+                    const uint32_t e = (uint32_t)(k * 32 + lane);
+                    off[k] = 0;
+                    if (e < nb) {
+                        off[k] = q[(h + e) & (cap - 1)];
+                        valid |= 1u << k;
+                    }
+                }
+                __syncwarp();
+                Q.set_head(l, (h + nb) & (cap - 1));
+                Q.set_count(l, Q.count(l) - nb);
+            }
+            if (l + 1 == nq) {
+                final_rows<AGG, MUL, false>(P, st, smem, nq, qbase, off, valid, lsum, lcnt);
             } else {
-                int32_t v[4] = {0, 0, 0, 0};
-                const int32_t *c = static_cast<const int32_t *>(S.col) + row0;
-                if (valid == 0xFu) {
-                    const int4 a = ld_stream16(c);
-                    v[0] = a.x, v[1] = a.y, v[2] = a.z, v[3] = a.w;
-                } else {
+                const uint32_t m = filter_rows(P, st[l + 1], smem, qbase, off, valid);
+                const uint32_t mine = (uint32_t)__popc(m);
+                uint32_t incl = mine;
 #pragma unroll
-                    for (int r = 0; r < 4; ++r)
-                        if ((valid >> r) & 1u) v[r] = __ldcs(c + r);
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += t;
                 }
+                const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
+                if (tot) {
+                    uint32_t *q = qmem + queue_base(l + 1);
+                    uint32_t pos = Q.head(l + 1) + Q.count(l + 1) + incl - mine;
 #pragma unroll
-                for (int r = 0; r < 4; ++r)
-                    if ((alive >> r) & 1u)
-                        if (!apply<int32_t, MUL>(S, smem, v[r], key[r], X[r], Y[r])) alive &= ~(1u << r);
+                    for (int k = 0; k < kRows; ++k) {
+                        if ((m >> k) & 1u) {
+                            q[pos & (kQueueCap - 1)] = off[k];
+                            ++pos;
+                        }
+                    }
+                    Q.set_count(l + 1, Q.count(l + 1) + tot);
+                    __syncwarp();
+                }
             }
         }
-#pragma unroll
-        for (int r = 0; r < 4; ++r)
-            if ((alive >> r) & 1u) terminal<AGG, MUL>(P, smem, key[r], X[r], Y[r], lsum, lcnt);
     }
 
     if (AGG == AGG_SCALAR) {
@@ -292,7 +689,6 @@ __global__ void __launch_bounds__(1024) fused_kernel(const __grid_constant__ Run
             lcnt += __shfl_xor_sync(0xffffffffu, lcnt, o);
         }
         __shared__ int64_t part[64];
-        const int warp = tid >> 5, lane = tid & 31;
         if (lane == 0) {
             part[warp] = lsum;
             part[32 + warp] = lcnt;

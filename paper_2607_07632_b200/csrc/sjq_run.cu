@@ -127,7 +127,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     }
     if (!valid_term(agg->x, nfact, joins, njoins)) return SJQ_ERR_INVALID_ARG;
     if (agg->op != SJQ_AGG_COL && !valid_term(agg->y, nfact, joins, njoins)) return SJQ_ERR_INVALID_ARG;
-    if (opts.block_threads && (opts.block_threads < 128 || opts.block_threads > 1024 || opts.block_threads % 32))
+    if (opts.block_threads && (opts.block_threads < 128 || opts.block_threads > 512 || opts.block_threads % 32))
         return SJQ_ERR_INVALID_ARG;
     if (opts.norder && opts.norder != npreds + njoins) return SJQ_ERR_INVALID_ARG;
 
@@ -188,25 +188,50 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     std::memset(&P, 0, sizeof(P));
     P.n = n;
     int ns = 0;
+    int nsets = 0;
     std::vector<int> stage_of_join(njoins, -1);
     std::vector<int> stage_of_col(nfact, -1);
     std::vector<int> stage_label;
-    for (int i = 0; i < nfilter; ++i) {
-        const StageSpec &sp = specs[order[i]];
-        DStage &S = P.st[ns];
+    auto fill_stage = [&](DStage &S, const StageSpec &sp) -> sjq_status {
         S.kind = (uint8_t)sp.kind;
         S.col = fact[sp.col].data;
         S.is64 = (uint8_t)(fact[sp.col].dtype == SJQ_I64);
+        S.op = OP_LOAD;
         if (sp.kind == ST_PRED) {
-            if (!canon_pred(preds[sp.index], fact[sp.col].dtype, &S.pred)) return SJQ_ERR_INVALID_ARG;
-        } else {
+            DPred d;
+            if (!canon_pred(preds[sp.index], fact[sp.col].dtype, &d)) return SJQ_ERR_INVALID_ARG;
+            if (d.nset) {
+                S.op = OP_PRED_SET;
+                S.nset = d.nset;
+                S.set_idx = (uint8_t)nsets;
+                for (int k = 0; k < d.nset; ++k) P.sets[nsets][k] = d.set[k];
+                ++nsets;
+            } else {
+                S.op = OP_PRED_RANGE;
+                S.lo = d.lo;
+                S.hi = d.hi;
+                S.neg = d.neg;
+                S.never = d.never;
+                S.lo32 = d.lo32;
+                S.width32 = d.never ? 0u : (uint32_t)d.hi32 - (uint32_t)d.lo32;
+            }
+        } else if (sp.kind == ST_PROBE) {
             const sjq_table *T = joins[sp.index].table;
             const sjq_dim_layout &L = T->layout;
-            S.tkind = (uint8_t)L.kind;
+            if (L.slots > ((int64_t)1 << 31) && L.kind >= SJQ_TABLE_HASH_I32) return SJQ_ERR_UNSUPPORTED;
+            S.op = (uint8_t)(L.kind == SJQ_TABLE_DIRECT_BITMAP ? OP_DIRECT_BITMAP
+                             : L.kind == SJQ_TABLE_DIRECT_U8   ? OP_DIRECT_U8
+                             : L.kind == SJQ_TABLE_DIRECT_U16  ? OP_DIRECT_U16
+                             : L.kind == SJQ_TABLE_DIRECT_U32  ? OP_DIRECT_U32
+                             : L.kind == SJQ_TABLE_DIRECT_U64  ? OP_DIRECT_U64
+                             : L.kind == SJQ_TABLE_HASH_I32    ? OP_HASH32
+                                                               : OP_HASH64);
             S.tab = T->slots;
             S.codes = T->codes;
             S.kmin = L.kmin;
-            S.span = (uint64_t)L.slots;
+            S.last = (uint64_t)L.slots - 1;
+            S.kmin32 = (int32_t)L.kmin;
+            S.last32 = (uint32_t)std::min<uint64_t>((uint64_t)L.slots - 1, 0xFFFFFFFFull);
             S.hmask = (uint64_t)L.slots - 1;
             S.pmin0 = L.pay_min[0];
             S.pmin1 = L.pay_min[1];
@@ -214,39 +239,17 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
             S.pmask0 = L.pay_bits[0] >= 64 ? ~0ULL : ((1ULL << L.pay_bits[0]) - 1ULL);
             S.code_bits = (uint8_t)L.code_bits;
             S.tab_bytes = (uint32_t)std::min<size_t>(T->slots_bytes, 0xFFFFFFF0u);
-            stage_of_join[sp.index] = ns;
         }
+        return SJQ_OK;
+    };
+    for (int i = 0; i < nfilter; ++i) {
+        const StageSpec &sp = specs[order[i]];
+        if ((st = fill_stage(P.st[ns], sp)) != SJQ_OK) return st;
+        if (sp.kind == ST_PROBE) stage_of_join[sp.index] = ns;
         if (stage_of_col[sp.col] < 0) stage_of_col[sp.col] = ns;
         stage_label.push_back(order[i]);
         ++ns;
     }
-    for (const Contribution &c : contrib) {
-        int s, src;
-        if (c.src == SJQ_SRC_FACT) {
-            if (stage_of_col[c.a] < 0) { // a column nobody filters on: plain load stage at the end
-                if (ns >= kMaxStages) return SJQ_ERR_UNSUPPORTED;
-                DStage &S = P.st[ns];
-                S.kind = ST_LOAD;
-                S.col = fact[c.a].data;
-                S.is64 = (uint8_t)(fact[c.a].dtype == SJQ_I64);
-                stage_of_col[c.a] = ns;
-                stage_label.push_back(-1);
-                ++ns;
-            }
-            s = stage_of_col[c.a];
-            src = 0;
-        } else {
-            s = stage_of_join[c.a];
-            src = 1 + c.b;
-        }
-        DStage &S = P.st[s];
-        const int slot = 3 * src + c.dest;
-        S.mult[slot] = (int64_t)((uint64_t)S.mult[slot] + (uint64_t)c.mult);
-        S.acc |= (uint16_t)(1u << slot);
-    }
-    P.nstages = ns;
-    P.first_sparse = ns;
-    P.eager = opts.eager_loads ? 1 : 0;
     P.want_count = agg->want_count ? 1 : 0;
     P.status = out->status;
     if (key) {
@@ -256,14 +259,78 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         P.mod32 = key->modulo > 0 && key->modulo <= 0xFFFFFFFFLL;
     }
 
-    // ------------------------------------------------------------ survivors estimate
-    double cum = 1.0;
-    std::vector<double> reach(ns, 1.0); // fraction of rows reaching each stage
-    for (int s = 0; s < ns; ++s) {
-        reach[s] = cum;
-        if (s < nfilter) cum *= specs[order[s]].sel;
+    // ------------------------------------------------------------ dense / sparse split
+    // Fraction of rows reaching each filter stage, from the estimates.
+    std::vector<double> reach(nfilter + 1, 1.0);
+    for (int s = 0; s < nfilter; ++s) reach[s + 1] = reach[s] * specs[order[s]].sel;
+    const double survivors = (double)n * reach[nfilter];
+    // Stage 0 filters thread-owned rows (level 0); up to kMaxQueues - 1 further
+    // stages run as queue-fed pure filters while they really filter and enough
+    // rows still reach them; everything after runs at the final level.  Eager
+    // loading and compaction = never use no queue at all.
+    int ndense = 0;
+    const bool direct = opts.eager_loads || opts.compaction == 1 || nfilter == 0;
+    if (!direct) {
+        ndense = 1;
+        if (opts.compaction != 2) {
+            for (int s = 1; s < nfilter && s < kMaxQueues; ++s) {
+                if (specs[order[s]].sel < 0.9 && reach[s] > 0.01) ndense = s + 1;
+                else break;
+            }
+        }
     }
-    const double survivors = (double)n * cum;
+    P.nq = ndense;
+
+    // Sources of the accumulators.  A dense stage cannot feed an accumulator
+    // (it only keeps a bit per row), so a value it would supply is gathered
+    // again for the survivors by a sparse copy of the stage.
+    std::vector<int> gather_of_stage(ns, -1);
+    for (const Contribution &c : contrib) {
+        int s, src;
+        if (c.src == SJQ_SRC_FACT) {
+            if (stage_of_col[c.a] < 0) { // a column nobody filters on: plain load stage at the end
+                if (ns >= kMaxStages) return SJQ_ERR_UNSUPPORTED;
+                StageSpec sp{ST_LOAD, -1, c.a, 1.0, 1.0};
+                fill_stage(P.st[ns], sp);
+                stage_of_col[c.a] = ns;
+                stage_label.push_back(-1);
+                gather_of_stage.push_back(-1);
+                ++ns;
+            }
+            s = stage_of_col[c.a];
+            src = 0;
+        } else {
+            s = stage_of_join[c.a];
+            src = 1 + c.b;
+        }
+        if (s < ndense) {
+            if (gather_of_stage[s] < 0) {
+                if (ns >= kMaxStages) return SJQ_ERR_UNSUPPORTED;
+                P.st[ns] = P.st[s];
+                gather_of_stage[s] = ns;
+                stage_label.push_back(stage_label[s]);
+                gather_of_stage.push_back(-1);
+                ++ns;
+            }
+            s = gather_of_stage[s];
+        }
+        DStage &S = P.st[s];
+        const int slot = 3 * src + c.dest;
+        S.mult[slot] = (int64_t)((uint64_t)S.mult[slot] + (uint64_t)c.mult);
+        S.acc |= (uint16_t)(1u << slot);
+    }
+    // a gathered copy that only needs the raw value need not filter again
+    for (int s = ndense; s < ns; ++s) {
+        DStage &S = P.st[s];
+        bool is_copy = false;
+        for (int d = 0; d < ndense; ++d) is_copy |= gather_of_stage[d] == s;
+        if (is_copy && (S.acc & ~0x7u) == 0) {
+            S.kind = ST_LOAD;
+            S.op = OP_LOAD;
+        }
+    }
+    P.nstages = ns;
+    P.eager = opts.eager_loads ? 1 : 0;
 
     // ------------------------------------------------------------ aggregation path
     int aggp;
@@ -313,14 +380,20 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         P.counts = agg->want_count ? out->counts : nullptr;
     }
 
-    // ------------------------------------------------------------ shared-memory tables
-    size_t smem = 0;
+    // ------------------------------------------------------------ shared memory layout
+    // [stage descriptors][staged tables][group table][per-warp survivor queues]
+    int block = opts.block_threads ? opts.block_threads : 512;
     const size_t smem_cap = (size_t)dev.max_smem_optin - 1024; // static reduce scratch + slack
-    const size_t table_budget = smem_cap > group_bytes ? smem_cap - group_bytes : 0;
+    const size_t stage_bytes = align_up((size_t)ns * sizeof(DStage), 16);
+    auto queue_bytes = [&](int threads) { return P.nq ? (size_t)(threads / 32) * (size_t)(kQueue0Cap + (P.nq - 1) * kQueueCap) * 4 : (size_t)0; };
+    const size_t fixed = stage_bytes + group_bytes + queue_bytes(block);
+    if (fixed > smem_cap) return SJQ_ERR_UNSUPPORTED;
+    const size_t table_budget = smem_cap - fixed;
+    size_t tables = 0;
     if (opts.smem_tables != 1) {
         std::vector<int> cand;
         for (int s = 0; s < nfilter; ++s)
-            if (P.st[s].kind == ST_PROBE && P.st[s].tkind <= SJQ_TABLE_DIRECT_U64) cand.push_back(s);
+            if (P.st[s].op >= OP_DIRECT_BITMAP && P.st[s].op <= OP_DIRECT_U64) cand.push_back(s);
         // most probes per staged byte first
         std::stable_sort(cand.begin(), cand.end(), [&](int a, int b) {
             return reach[a] / (double)P.st[a].tab_bytes > reach[b] / (double)P.st[b].tab_bytes;
@@ -328,31 +401,34 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         for (int s : cand) {
             DStage &S = P.st[s];
             const size_t tb = align_up(S.tab_bytes, 16);
-            if (smem + tb > table_budget) continue;
-            // worth it only if a CTA probes it more often than it costs to copy
+            if (tables + tb > table_budget) continue;
+            // larger tables are left to L1/L2: shared memory taken here is L1 capacity lost to every other table
+            if (opts.smem_tables == 0 && tb > (size_t)16 << 10) continue;
+            // worth it only if a block probes the table more often than it costs to copy
             const double probes_per_cta = (double)n * reach[s] / approx_grid;
             if (probes_per_cta * 4.0 < (double)tb) continue;
             S.in_smem = 1;
-            S.smem_off = (uint32_t)smem;
-            smem += tb;
+            S.smem_off = (uint32_t)(stage_bytes + tables);
+            tables += tb;
+            if (s < ndense && gather_of_stage[s] >= 0) { // the sparse copy reads the same staged table
+                P.st[gather_of_stage[s]].in_smem = 1;
+                P.st[gather_of_stage[s]].smem_off = S.smem_off;
+            }
         }
     }
-    P.smem_groups = (uint32_t)smem;
-    smem += group_bytes;
-    P.smem_queue = (uint32_t)smem;
+    P.smem_stages = 0;
+    P.smem_groups = (uint32_t)(stage_bytes + tables);
+    P.smem_queue = (uint32_t)(stage_bytes + tables + group_bytes);
+    size_t smem = stage_bytes + tables + group_bytes + queue_bytes(block);
 
     // ------------------------------------------------------------ launch shape
-    int block = opts.block_threads ? opts.block_threads : 512;
     int per_sm = 0;
     if ((st = fused_occupancy(aggp, mul, block, smem, &per_sm)) != SJQ_OK) return st;
-    if (!opts.block_threads && per_sm <= 1) { // big shared-memory footprint: one large CTA per SM
-        block = 1024;
-        if ((st = fused_occupancy(aggp, mul, block, smem, &per_sm)) != SJQ_OK) return st;
-    }
     if (per_sm < 1) return SJQ_ERR_UNSUPPORTED;
     if (opts.ctas_per_sm > 0) per_sm = std::min(per_sm, opts.ctas_per_sm);
-    const int64_t tile_rows = (int64_t)block * 4;
+    const int64_t tile_rows = (int64_t)block * (P.nq ? kDenseRows : kRows);
     const int64_t ntiles = (n + tile_rows - 1) / tile_rows;
+    if (ntiles >= ((int64_t)1 << 31)) return SJQ_ERR_UNSUPPORTED;
     int grid = (int)std::min<int64_t>((int64_t)dev.sm_count * per_sm, std::max<int64_t>(ntiles, 1));
 
     // ------------------------------------------------------------ launches
@@ -367,10 +443,15 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     } else if (spec->mode == SJQ_HASHED) {
         if (cudaMemsetAsync(out->n_groups, 0, sizeof(int64_t), stream) != cudaSuccess) return SJQ_ERR_CUDA;
     }
+    if ((opts.event_before != nullptr) != (opts.event_after != nullptr)) return SJQ_ERR_INVALID_ARG;
+    if (opts.event_before && cudaEventRecord((cudaEvent_t)opts.event_before, stream) != cudaSuccess)
+        return SJQ_ERR_CUDA;
     if (n > 0) {
         if ((st = fused_launch(aggp, mul, grid, block, smem, P, stream)) != SJQ_OK) return st;
         ++launches;
     }
+    if (opts.event_after && cudaEventRecord((cudaEvent_t)opts.event_after, stream) != cudaSuccess)
+        return SJQ_ERR_CUDA;
     if (spec->mode == SJQ_HASHED) {
         st = compact_launch(gkeys, gsums, gcounts, (int64_t)gslots, out->keys, out->sums, out->counts, spec->capacity,
                             out->n_groups, out->status, dev.sm_count, stream);
@@ -384,7 +465,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
             info->order[s] = stage_label[s];
             info->stage_in_smem[s] = P.st[s].in_smem;
         }
-        info->first_sparse_stage = P.first_sparse;
+        info->first_sparse_stage = P.nq;
         info->agg_path = aggp;
         info->grid = grid;
         info->block = block;
@@ -392,4 +473,112 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         info->kernel_launches = launches;
     }
     return SJQ_OK;
+}
+
+
+// ---------------------------------------------------------------------------
+// Host-buffer entry point: chunked, double-buffered copy + run.
+namespace {
+
+struct HostPipe {
+    cudaStream_t s[2] = {nullptr, nullptr};
+    cudaEvent_t start = nullptr, done[2] = {nullptr, nullptr};
+    bool ok = false;
+};
+
+HostPipe *host_pipe()
+{
+    static thread_local HostPipe pipes[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    HostPipe &p = pipes[dev];
+    if (!p.ok) {
+        if (cudaStreamCreateWithFlags(&p.s[0], cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&p.s[1], cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&p.done[0], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&p.done[1], cudaEventDisableTiming) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        p.ok = true;
+    }
+    return &p;
+}
+
+} // namespace
+
+extern "C" sjq_status sjq_run_host(const sjq_col *fact_host, int nfact, const sjq_pred *preds, int npreds,
+                                   const sjq_join *joins, int njoins, const sjq_key_expr *key,
+                                   const sjq_agg_expr *agg, const sjq_result_spec *spec, const sjq_result *out,
+                                   const sjq_run_opts *opts_, void *staging_dev, size_t staging_bytes,
+                                   int64_t chunk_rows, int64_t *host_sums, int64_t *host_counts, int64_t *host_keys,
+                                   int64_t *host_n_groups, int32_t *host_status, void *stream_)
+{
+    if (!fact_host || nfact <= 0 || nfact > 64 || !staging_dev || chunk_rows <= 0 || (chunk_rows & 3) || !spec ||
+        !out || !agg)
+        return SJQ_ERR_INVALID_ARG;
+    if (!aligned16(staging_dev)) return SJQ_ERR_ALIGN;
+    const int64_t n = fact_host[0].n;
+    if (n < 0) return SJQ_ERR_INVALID_ARG;
+    size_t half = 0;
+    std::vector<size_t> col_off(nfact);
+    for (int c = 0; c < nfact; ++c) {
+        if (fact_host[c].n != n || (fact_host[c].dtype != SJQ_I32 && fact_host[c].dtype != SJQ_I64) ||
+            (n > 0 && !fact_host[c].data))
+            return SJQ_ERR_INVALID_ARG;
+        col_off[c] = half;
+        half += align_up((size_t)chunk_rows * (fact_host[c].dtype == SJQ_I64 ? 8 : 4), 256);
+    }
+    if (staging_bytes < 2 * half) return SJQ_ERR_BUFFER_SMALL;
+    HostPipe *hp = host_pipe();
+    if (!hp) return SJQ_ERR_CUDA;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    sjq_run_opts opts{};
+    if (opts_) opts = *opts_;
+    opts.event_before = opts.event_after = nullptr;
+
+    // internal streams start after whatever is already queued on the caller's stream
+    if (cudaEventRecord(hp->start, stream) != cudaSuccess) return SJQ_ERR_CUDA;
+    for (int b = 0; b < 2; ++b)
+        if (cudaStreamWaitEvent(hp->s[b], hp->start, 0) != cudaSuccess) return SJQ_ERR_CUDA;
+
+    const int64_t nchunks = n == 0 ? 1 : (n + chunk_rows - 1) / chunk_rows;
+    std::vector<sjq_col> dev_cols(nfact);
+    for (int64_t k = 0; k < nchunks; ++k) {
+        const int b = (int)(k & 1);
+        const int64_t r0 = k * chunk_rows;
+        const int64_t rows = std::min<int64_t>(chunk_rows, n - r0);
+        char *base = static_cast<char *>(staging_dev) + (size_t)b * half;
+        // copies into this half follow run k-2 by stream order and overlap run k-1 on the other stream
+        for (int c = 0; c < nfact; ++c) {
+            const size_t w = fact_host[c].dtype == SJQ_I64 ? 8 : 4;
+            dev_cols[c] = sjq_col{base + col_off[c], fact_host[c].dtype, rows};
+            if (rows > 0 &&
+                cudaMemcpyAsync(base + col_off[c], static_cast<const char *>(fact_host[c].data) + (size_t)r0 * w,
+                                (size_t)rows * w, cudaMemcpyHostToDevice, hp->s[b]) != cudaSuccess)
+                return SJQ_ERR_CUDA;
+        }
+        // runs accumulate into the same result and must not overlap: run k waits for run k-1
+        if (k > 0 && cudaStreamWaitEvent(hp->s[b], hp->done[b ^ 1], 0) != cudaSuccess) return SJQ_ERR_CUDA;
+        opts.accumulate = (k > 0 || (opts_ && opts_->accumulate)) ? 1 : 0;
+        sjq_status st = sjq_run(dev_cols.data(), nfact, preds, npreds, joins, njoins, key, agg, spec, out, &opts,
+                                hp->s[b], nullptr);
+        if (st != SJQ_OK) return st;
+        if (cudaEventRecord(hp->done[b], hp->s[b]) != cudaSuccess) return SJQ_ERR_CUDA;
+    }
+    const int last = (int)((nchunks - 1) & 1);
+    if (cudaStreamWaitEvent(stream, hp->done[last], 0) != cudaSuccess) return SJQ_ERR_CUDA;
+    if (nchunks > 1 && cudaStreamWaitEvent(stream, hp->done[last ^ 1], 0) != cudaSuccess) return SJQ_ERR_CUDA;
+    const int64_t cells = spec->mode == SJQ_SCALAR ? 1 : spec->mode == SJQ_DENSE ? spec->num_groups : spec->capacity;
+    bool ok = true;
+    if (host_sums) ok = ok && cudaMemcpyAsync(host_sums, out->sums, (size_t)cells * 8, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (host_counts && out->counts)
+        ok = ok && cudaMemcpyAsync(host_counts, out->counts, (size_t)cells * 8, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (host_keys && out->keys)
+        ok = ok && cudaMemcpyAsync(host_keys, out->keys, (size_t)cells * 8, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (host_n_groups && out->n_groups)
+        ok = ok && cudaMemcpyAsync(host_n_groups, out->n_groups, 8, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (host_status) ok = ok && cudaMemcpyAsync(host_status, out->status, 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    return ok ? SJQ_OK : SJQ_ERR_CUDA;
 }

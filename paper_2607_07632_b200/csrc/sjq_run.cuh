@@ -12,51 +12,80 @@ namespace sjq {
 enum : uint8_t { ST_PRED = 0, ST_PROBE = 1, ST_LOAD = 2 };
 enum : int32_t { AGG_SCALAR = 0, AGG_SMEM = 1, AGG_GLOBAL = 2, AGG_HASH = 3 };
 
+// Stage bodies (uniform switch per stage, straight-line code inside).
+enum : uint8_t {
+    OP_LOAD = 0,
+    OP_PRED_RANGE = 1,
+    OP_PRED_SET = 2,
+    OP_DIRECT_BITMAP = 3,
+    OP_DIRECT_U8 = 4,
+    OP_DIRECT_U16 = 5,
+    OP_DIRECT_U32 = 6,
+    OP_DIRECT_U64 = 7,
+    OP_HASH32 = 8,
+    OP_HASH64 = 9
+};
+
 // which accumulators a stage's values feed: bit = 3 * source + destination,
 // source 0 = the fact value itself, 1 = payload 0, 2 = payload 1;
 // destination 0 = group key, 1 = X, 2 = Y.  value = X (or X*Y for a product).
 constexpr int kAccKey = 0, kAccX = 1, kAccY = 2;
 
-constexpr int kMaxStages = SJQ_MAX_PREDS + SJQ_MAX_JOINS + 8;
+constexpr int kMaxStages = SJQ_MAX_PREDS + SJQ_MAX_JOINS + 8 + SJQ_MAX_JOINS + SJQ_MAX_PREDS;
+
+// Geometry of the fused kernel.
+constexpr int kSlots = 2;                // level 0: 128-bit loads per thread per tile
+constexpr int kDenseRows = 4 * kSlots;   // rows a thread owns at level 0
+constexpr int kRows = 4;                 // rows a lane handles per batch at the queue-fed levels
+constexpr int kBatch = 32 * kRows;       // rows a warp processes at once at those levels
+constexpr int kQueue0Cap = 512;          // entries of a warp's first queue: a batch minus one plus a whole tile
+constexpr int kQueueCap = 256;           // entries of its later queues: a batch minus one plus a batch
+constexpr int kMaxQueues = 3;            // queue-fed levels per warp (the last one is the final level)
 
 struct DStage {
     const void *col;   // fact column read by this stage
     const void *tab;   // direct: code array / bitmap words; hash: key array
     const void *codes; // hash: payload codes
     int64_t kmin;      // direct: slot index = key - kmin
-    uint64_t span;     // direct: number of slots
+    uint64_t last;     // direct: last valid slot index (slots - 1)
+    int64_t lo, hi;    // 64-bit predicate range
     uint64_t hmask;    // hash: slots - 1
     int64_t pmin0, pmin1;
     uint64_t pmask0;
     int64_t mult[9];
-    DPred pred;
+    int32_t lo32;      // 32-bit predicate: pass iff (uint32)(v - lo32) <= width32
+    uint32_t width32;
+    int32_t kmin32;    // 32-bit direct probe: idx = (uint32)v - (uint32)kmin32, hit range idx <= last32
+    uint32_t last32;
     uint32_t smem_off;  // byte offset of the staged copy in dynamic shared memory
     uint32_t tab_bytes; // bytes to stage
     uint16_t acc;
-    uint8_t kind, is64, tkind, in_smem, pbits0, code_bits;
+    uint8_t op, is64, neg, never, nset, set_idx, pbits0, code_bits, in_smem, kind;
 };
 
 struct RunParams {
     DStage st[kMaxStages];
+    int64_t sets[SJQ_MAX_PREDS][SJQ_MAX_IN_SET];
     int64_t n;
     int64_t key_offset;
     int64_t modulo;   // 0 = none
     uint64_t modmask; // modulo - 1 when modulo is a power of two, else 0
     int64_t num_groups;
-    uint64_t gmask;    // hashed: group-table slots - 1
-    int64_t *sums;     // scalar/dense: result; hashed: table sums
-    int64_t *counts;   // may be NULL
-    int64_t *gkeys;    // hashed: table keys
+    uint64_t gmask; // hashed: group-table slots - 1
+    int64_t *sums;  // scalar/dense: result; hashed: table sums
+    int64_t *counts; // may be NULL
+    int64_t *gkeys;  // hashed: table keys
     int32_t *status;
     int32_t nstages;
-    int32_t first_sparse; // stages >= this run on compacted survivors
+    int32_t nq;     // queue-fed levels: 0 = none (every stage on thread-owned rows); else stage 0 is the
+                    // dense level, stages 1 .. nq-1 are queue-fed filters, stages nq .. run at the final level
     int32_t want_count;
-    int32_t eager;
-    int32_t has_key;      // compute and range-check the key (dense with one group in scalar path)
-    int32_t mod32;        // modulo fits in 32 bits
+    int32_t eager;   // load every column for every row
+    int32_t has_key; // scalar path of a one-group dense result: key is computed and range-checked
+    int32_t mod32;   // modulo fits in 32 bits
+    uint32_t smem_stages; // byte offset of the stage descriptors copied to shared memory
     uint32_t smem_groups; // byte offset of the shared group table
     uint32_t smem_queue;  // byte offset of the per-warp survivor queues
-    uint32_t carry;       // bit 0 key, 1 X, 2 Y: accumulators live at the dense->sparse switch
 };
 
 } // namespace sjq

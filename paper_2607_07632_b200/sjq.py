@@ -90,7 +90,8 @@ class _RunOpts(ctypes.Structure):
     _fields_ = [("block_threads", ctypes.c_int32), ("ctas_per_sm", ctypes.c_int32), ("eager_loads", ctypes.c_int32),
                 ("agg_path", ctypes.c_int32), ("smem_tables", ctypes.c_int32), ("compaction", ctypes.c_int32),
                 ("accumulate", ctypes.c_int32), ("norder", ctypes.c_int32),
-                ("order", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS)), ("reserved", ctypes.c_int32 * 8)]
+                ("order", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS)), ("event_before", ctypes.c_void_p),
+                ("event_after", ctypes.c_void_p), ("reserved", ctypes.c_int32 * 8)]
 
 
 class RunInfo(ctypes.Structure):
@@ -116,6 +117,7 @@ class RunOpts:
     compaction: int = 0
     accumulate: bool = False
     order: Sequence[int] = ()
+    events: Optional[tuple] = None  # (torch.cuda.Event, torch.cuda.Event), both already recorded once
 
     def to_c(self) -> _RunOpts:
         o = _RunOpts()
@@ -125,6 +127,8 @@ class RunOpts:
         o.norder = len(self.order)
         for i, v in enumerate(self.order):
             o.order[i] = v
+        if self.events is not None:
+            o.event_before, o.event_after = self.events[0].cuda_event, self.events[1].cuda_event
         return o
 
 
@@ -156,6 +160,11 @@ def lib():
         L.sjq_run.argtypes = [ctypes.POINTER(_Col), ip, ctypes.POINTER(_Pred), ip, ctypes.POINTER(_Join), ip,
                               ctypes.POINTER(_KeyExpr), ctypes.POINTER(_AggExpr), ctypes.POINTER(_ResultSpec),
                               ctypes.POINTER(_Result), ctypes.POINTER(_RunOpts), vp, ctypes.POINTER(RunInfo)]
+        L.sjq_run_host.restype = ctypes.c_int32
+        L.sjq_run_host.argtypes = [ctypes.POINTER(_Col), ip, ctypes.POINTER(_Pred), ip, ctypes.POINTER(_Join), ip,
+                                   ctypes.POINTER(_KeyExpr), ctypes.POINTER(_AggExpr), ctypes.POINTER(_ResultSpec),
+                                   ctypes.POINTER(_Result), ctypes.POINTER(_RunOpts), vp, ctypes.c_size_t,
+                                   ctypes.c_int64, vp, vp, vp, vp, vp, vp]
         L.sjq_strerror.restype = ctypes.c_char_p
         L.sjq_strerror.argtypes = [ctypes.c_int32]
         L.sjq_version.restype = ctypes.c_char_p
@@ -333,6 +342,91 @@ def run(fact: dict, preds=(), joins=(), key=None, agg=None, mode: str = "SCALAR"
         if rc != 0:
             raise SjqError(rc, "sjq_run")
     return res
+
+
+@dataclass
+class HostResult:
+    """Pinned host copies of a result (filled when the stream has synchronised)."""
+    sums: torch.Tensor
+    counts: Optional[torch.Tensor]
+    keys: Optional[torch.Tensor]
+    n_groups: Optional[torch.Tensor]
+    status: torch.Tensor
+
+
+def staging_bytes(fact: dict, chunk_rows: int) -> int:
+    per = 0
+    for t in fact.values():
+        per += (chunk_rows * t.element_size() + 255) // 256 * 256
+    return 2 * per
+
+
+def run_host(fact: dict, staging: torch.Tensor, chunk_rows: int, preds=(), joins=(), key=None, agg=None,
+             mode: str = "SCALAR", num_groups: int = 1, capacity: int = 0, opts: Optional[RunOpts] = None,
+             result: Optional[Result] = None, host: Optional[HostResult] = None):
+    """sjq_run_host: `fact` is a dict of HOST tensors (pinned for full speed), `staging` a CUDA uint8
+    tensor of at least staging_bytes(fact, chunk_rows).  Returns (Result, HostResult); synchronise the
+    current stream before reading the host copies."""
+    names = list(fact.keys())
+    tensors = [fact[n] for n in names]
+    device = staging.device
+    with torch.cuda.device(device):
+        carr = (_Col * len(tensors))()
+        for i, t in enumerate(tensors):
+            if t.is_cuda or t.dtype not in (torch.int32, torch.int64) or not t.is_contiguous():
+                raise ValueError("run_host takes contiguous int32/int64 host tensors")
+            carr[i] = _Col(t.data_ptr(), 1 if t.dtype == torch.int64 else 0, t.numel())
+        parr, keep = _preds(preds, names)
+        jarr = (_Join * max(1, len(joins)))()
+        for j, (fk, table) in enumerate(joins):
+            jarr[j] = _Join(names.index(fk), table.handle)
+        kexpr = None
+        if key is not None:
+            kexpr = _KeyExpr()
+            for i, t in enumerate(key.terms):
+                kexpr.t[i] = _term(t, names)
+            kexpr.nterms, kexpr.offset, kexpr.modulo = len(key.terms), key.offset, key.modulo
+        aexpr = _AggExpr(AGGS[agg.op], _term(agg.x, names), _term(agg.y, names), int(agg.want_count))
+        spec = _ResultSpec(MODES[mode], num_groups, capacity)
+        res = result if result is not None else alloc_result(mode, num_groups, capacity, agg.want_count, device)
+        if host is None:
+            pin = dict(pin_memory=True)
+            host = HostResult(torch.empty_like(res.sums, device="cpu", **pin),
+                              torch.empty_like(res.counts, device="cpu", **pin) if res.counts is not None else None,
+                              torch.empty_like(res.keys, device="cpu", **pin) if res.keys is not None else None,
+                              torch.zeros(1, dtype=torch.int64, **pin) if res.n_groups is not None else None,
+                              torch.zeros(1, dtype=torch.int32, **pin))
+        cres = _Result(res.sums.data_ptr(), res.counts.data_ptr() if res.counts is not None else None,
+                       res.keys.data_ptr() if res.keys is not None else None,
+                       res.n_groups.data_ptr() if res.n_groups is not None else None, res.status_dev.data_ptr(),
+                       res.workspace.data_ptr() if res.workspace is not None else None,
+                       res.workspace.numel() if res.workspace is not None else 0)
+        copts = (opts or RunOpts()).to_c()
+        rc = lib().sjq_run_host(carr, len(names), parr, len(preds), jarr, len(joins),
+                                ctypes.byref(kexpr) if kexpr is not None else None, ctypes.byref(aexpr),
+                                ctypes.byref(spec), ctypes.byref(cres), ctypes.byref(copts), staging.data_ptr(),
+                                staging.numel(), chunk_rows, host.sums.data_ptr(),
+                                host.counts.data_ptr() if host.counts is not None else None,
+                                host.keys.data_ptr() if host.keys is not None else None,
+                                host.n_groups.data_ptr() if host.n_groups is not None else None,
+                                host.status.data_ptr(), _stream_ptr(device))
+        if rc != 0:
+            raise SjqError(rc, "sjq_run_host")
+    return res, host
+
+
+def run_workload_host(w, fact: dict, tables: dict, staging: torch.Tensor, chunk_rows: int,
+                      opts: Optional[RunOpts] = None, result=None, host=None):
+    fact = {c.name: fact[c.name] for c in w.fact_cols}
+    return run_host(fact, staging, chunk_rows, w.preds, [(fk, tables[dn]) for fk, dn in w.joins], w.key, w.agg,
+                    w.mode, w.num_groups, w.capacity, opts, result, host)
+
+
+def build_launches(table: "Table") -> int:
+    """Kernels enqueued by sjq_dim_plan + sjq_build_dim for this table (cudaMemset calls not counted)."""
+    direct = table.layout.kind <= 5
+    rows = table.layout.dim_rows > 0
+    return 1 + (1 if rows else 0) + (1 if rows else 0) + (2 if direct else 1)
 
 
 def build_workload_tables(w, dims: dict) -> dict:

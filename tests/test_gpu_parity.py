@@ -48,7 +48,7 @@ def test_random_queries_option_matrix(seed):
     dev_fact = to_dev(fact)
     tables = None
     for opts in (sjq.RunOpts(), sjq.RunOpts(eager_loads=True), sjq.RunOpts(smem_tables=1),
-                 sjq.RunOpts(block_threads=128, ctas_per_sm=1), sjq.RunOpts(agg_path=2),
+                 sjq.RunOpts(block_threads=128, ctas_per_sm=1), sjq.RunOpts(block_threads=256, compaction=2, smem_tables=1), sjq.RunOpts(agg_path=2),
                  sjq.RunOpts(compaction=2), sjq.RunOpts(compaction=1),
                  sjq.RunOpts(order=tuple(reversed(range(len(w.preds) + len(w.joins)))))):
         res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)
@@ -212,3 +212,39 @@ def test_invalid_arguments_are_rejected():
     with pytest.raises(sjq.SjqError) as e:  # int32 fk into an int64-keyed table
         sjq.run(ok, joins=[("a", dim)], agg=AggExpr("COL", Term("FACT", "a")))
     assert e.value.status == 2
+
+
+def test_host_buffer_entry_point_matches_oracle():
+    for w in (W.config3(1_000_003), W.config4(500_001, 0.5, 100000, dim_rows=50000), W.config1(300_001)):
+        fact = W.host_fact(w)
+        hd = {d.name: W.host_dim(w, d) for d in w.dims}
+        res, exp, tables = run_both(w, fact, hd)
+        host_fact = {k: torch.from_numpy(v).pin_memory() for k, v in fact.items()}
+        chunk = 65536 * 3  # several chunks and a ragged last one
+        staging = torch.empty(sjq.staging_bytes(host_fact, chunk), dtype=torch.uint8, device="cuda")
+        r, h = sjq.run_workload_host(w, host_fact, tables, staging, chunk)
+        torch.cuda.synchronize()
+        assert int(h.status[0]) == 0
+        compare(w, r, exp)
+        if w.mode == "SCALAR":
+            assert int(h.sums[0]) == exp["sum"] and int(h.counts[0]) == exp["count"]
+        elif w.mode == "DENSE":
+            assert np.array_equal(h.sums.numpy(), exp["sums"]) and np.array_equal(h.counts.numpy(), exp["counts"])
+        else:
+            n = int(h.n_groups[0])
+            order = np.argsort(h.keys.numpy()[:n])
+            assert np.array_equal(h.keys.numpy()[:n][order], exp["keys"])
+            assert np.array_equal(h.sums.numpy()[:n][order], exp["sums"])
+
+
+def test_event_hooks_bracket_the_fused_kernel():
+    w = W.config3(2_000_003)
+    dims = {d.name: W.device_dim(w, d) for d in w.dims}
+    tables = sjq.build_workload_tables(w, dims)
+    fact = W.device_fact(w)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    b.record()
+    sjq.run_workload(w, fact, tables, sjq.RunOpts(events=(a, b)))
+    torch.cuda.synchronize()
+    assert 0.0 < a.elapsed_time(b) < 1000.0
