@@ -224,6 +224,7 @@ def main():
 
     import paper_2607_07632_b200 as sjq
     from datagen import workloads as W
+    from paper_2607_07632_b200 import shard
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -258,9 +259,7 @@ def main():
         opts = sjq.RunOpts(events=pairs[i]) if i is not None else None
         r = sjq.run_workload(w, fact, tables, opts, result=res)
         if world > 1 and w.mode != "HASHED":
-            dist.all_reduce(res.sums)
-            if res.counts is not None:
-                dist.all_reduce(res.counts)
+            shard.merge_dense(res.sums, res.counts)
         if i is not None:
             launches += r.info.kernel_launches + sum(sjq.build_launches(t) for t in tables.values())
         info = r.info

@@ -1,0 +1,71 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py
+times (default options, inputs generated on the device): the result must equal,
+bit for bit, the expected values the CPU oracle wrote to tests/golden/full_*.json
+(tests/golden/make_full_size.py).  Hashed results are compared through the
+SHA-256 of their (key, sum, count) triples in ascending key order."""
+import hashlib
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from datagen import workloads as W
+
+pytestmark = pytest.mark.gpu
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+
+
+def _golden(tag):
+    path = os.path.join(GOLDEN, f"full_{tag}.json")
+    if not os.path.exists(path):
+        pytest.skip(f"{path} not generated")
+    with open(path) as f:
+        return json.load(f)
+
+
+def _run(w):
+    import paper_2607_07632_b200 as sjq
+
+    dims = {d.name: W.device_dim(w, d) for d in w.dims}
+    tables = sjq.build_workload_tables(w, dims)
+    fact = W.device_fact(w)
+    res = sjq.run_workload(w, fact, tables)
+    torch.cuda.synchronize()
+    assert res.status() == 0 and all(t.status() == 0 for t in tables.values())
+    entries = {k: t.layout.entries for k, t in tables.items()}
+    del fact
+    torch.cuda.empty_cache()
+    return res, entries
+
+
+def _check(w, tag):
+    g = _golden(tag)
+    assert g["rows"] == w.n_rows and g["workload"] == w.name
+    res, entries = _run(w)
+    assert entries == g["dim_entries"]
+    if w.mode == "SCALAR":
+        assert int(res.sums[0].item()) == g["sum"] and int(res.counts[0].item()) == g["count"]
+    elif w.mode == "DENSE":
+        assert res.sums.cpu().tolist() == g["sums"]
+        assert res.counts.cpu().tolist() == g["counts"]
+    else:
+        k, s, c = res.hashed_sorted()
+        k, s, c = k.cpu().numpy(), s.cpu().numpy(), c.cpu().numpy()
+        assert k.size == g["groups"] and int(s.sum()) == g["total_sum"] and int(c.sum()) == g["total_count"]
+        h = hashlib.sha256()
+        for a in (k, s, c):
+            h.update(np.ascontiguousarray(a, dtype="<i8").tobytes())
+        assert h.hexdigest() == g["sha256"]
+
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c3", "c5"])
+def test_full_size_config(name):
+    _check(W.CONFIGS[name](), name)
+
+
+@pytest.mark.parametrize("sel", list(W.C4_THRESHOLDS))
+@pytest.mark.parametrize("groups", W.C4_GROUPS)
+def test_full_size_sweep_point(sel, groups):
+    _check(W.config4(600_000_000, sel, groups), f"c4_s{sel:g}_g{groups}")
