@@ -49,6 +49,7 @@ enum {
     SJQ_ERR_ALIGN = 3,        /* a device pointer is not 16-byte aligned */
     SJQ_ERR_CUDA = 4,         /* a CUDA runtime call failed (no device, launch error) */
     SJQ_ERR_BUFFER_SMALL = 5, /* caller-provided table / workspace memory too small */
+    SJQ_ERR_STATIC_LIMIT = 6, /* request exceeds the built-in scratch of a no-allocation entry point */
     /* device-detected (written to the status word) */
     SJQ_ERR_DUP_KEY = 16,        /* two dimension rows passing the filter share a key */
     SJQ_ERR_TABLE_FULL = 17,     /* open-addressing insert found no free slot */
@@ -303,6 +304,45 @@ sjq_status sjq_run_host(const sjq_col *fact_host, int nfact, const sjq_pred *pre
                         void *staging_dev, size_t staging_bytes, int64_t chunk_rows, int64_t *host_sums,
                         int64_t *host_counts, int64_t *host_keys, int64_t *host_n_groups, int32_t *host_status,
                         void *stream);
+
+/*
+ * Hashed group-by without any workspace from the caller.  (The paper has no
+ * counterpart: this entry point exists for embedders, not for the method.)
+ *
+ * Who needs it: code that runs where device allocation is forbidden or
+ * impossible -- a plug-in handed a fixed arena by its host process, a
+ * real-time or safety-certified loop whose rules ban allocator calls after
+ * start-up, a process whose memory pool is owned by another runtime.  Such a
+ * caller can still own its input columns and result arrays (they were given
+ * to it), but it has nowhere to get the group hash table that sjq_run takes
+ * as `workspace` in HASHED mode.
+ *
+ * What it does: exactly sjq_run with spec->mode == SJQ_HASHED, except that the
+ * group table lives in a fixed array inside the library's device image
+ * (SJQ_STATIC_WORKSPACE_BYTES, about 3 MiB, held by every GPU that loads the
+ * library until the process exits).  `out->workspace` and
+ * `out->workspace_bytes` are ignored; `out->keys/sums/counts` need `capacity`
+ * entries, `out->n_groups` and `out->status` as for sjq_run.
+ *
+ * Limits and rules:
+ *   - capacity must be 1 .. SJQ_STATIC_MAX_GROUPS; a larger request returns
+ *     SJQ_ERR_STATIC_LIMIT and enqueues nothing.
+ *   - `opts->accumulate` is ignored: the table is cleared at the start of
+ *     every call, because it is shared by all calls and still holds the
+ *     previous call's groups.
+ *   - Calls whose kernels could overlap on the GPU (different streams, several
+ *     host threads) race on the one table; run them one after another.
+ *   - The first call on a device looks the array's device address up once; make
+ *     that first call outside any stream capture.
+ *   - No cudaMalloc, cudaFree or other allocating CUDA call is made, here or in
+ *     anything this entry point calls.
+ */
+#define SJQ_STATIC_MAX_GROUPS 65536
+#define SJQ_STATIC_WORKSPACE_BYTES ((size_t)3 * 1024 * 1024 + 768 + 3 * 256)
+sjq_status sjq_run_hashed_static(const sjq_col *fact, int nfact, const sjq_pred *preds, int npreds,
+                                 const sjq_join *joins, int njoins, const sjq_key_expr *key,
+                                 const sjq_agg_expr *agg, int64_t capacity, const sjq_result *out,
+                                 const sjq_run_opts *opts, void *stream, sjq_run_info *info);
 
 const char *sjq_strerror(sjq_status status);
 const char *sjq_version(void);

@@ -582,3 +582,51 @@ extern "C" sjq_status sjq_run_host(const sjq_col *fact_host, int nfact, const sj
     if (host_status) ok = ok && cudaMemcpyAsync(host_status, out->status, 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
     return ok ? SJQ_OK : SJQ_ERR_CUDA;
 }
+
+
+// ---------------------------------------------------------------------------
+// Hashed group-by with the group table in the library's own device image, for
+// callers that cannot allocate device memory.
+namespace {
+
+// 2 * SJQ_STATIC_MAX_GROUPS slots + the side slot, three int64 arrays, each padded to 256 bytes.
+static __device__ __align__(256) unsigned char g_static_group_table[SJQ_STATIC_WORKSPACE_BYTES];
+
+} // namespace
+
+extern "C" sjq_status sjq_run_hashed_static(const sjq_col *fact, int nfact, const sjq_pred *preds, int npreds,
+                                            const sjq_join *joins, int njoins, const sjq_key_expr *key,
+                                            const sjq_agg_expr *agg, int64_t capacity, const sjq_result *out,
+                                            const sjq_run_opts *opts_, void *stream, sjq_run_info *info)
+{
+    if (!out || capacity <= 0) return SJQ_ERR_INVALID_ARG;
+    if (capacity > SJQ_STATIC_MAX_GROUPS) return SJQ_ERR_STATIC_LIMIT;
+    sjq_result_spec spec{SJQ_HASHED, 0, capacity};
+    size_t need = 0;
+    if (sjq_run_workspace_bytes(&spec, &need) != SJQ_OK || need > SJQ_STATIC_WORKSPACE_BYTES)
+        return SJQ_ERR_STATIC_LIMIT;
+
+    // In host code the array's name is only a stand-in; the kernels need its device address,
+    // looked up once per device with that device current.
+    static thread_local void *table_addr[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        (void)cudaGetLastError();
+        return SJQ_ERR_CUDA;
+    }
+    if (!table_addr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_group_table) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return SJQ_ERR_CUDA;
+        }
+        table_addr[dev] = p;
+    }
+    sjq_result r = *out;
+    r.workspace = table_addr[dev];
+    r.workspace_bytes = SJQ_STATIC_WORKSPACE_BYTES;
+    sjq_run_opts opts{};
+    if (opts_) opts = *opts_;
+    opts.accumulate = 0; // the shared table holds the last call's groups: always start from a cleared table
+    return sjq_run(fact, nfact, preds, npreds, joins, njoins, key, agg, &spec, &r, &opts, stream, info);
+}

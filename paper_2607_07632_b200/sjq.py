@@ -165,6 +165,11 @@ def lib():
                                    ctypes.POINTER(_KeyExpr), ctypes.POINTER(_AggExpr), ctypes.POINTER(_ResultSpec),
                                    ctypes.POINTER(_Result), ctypes.POINTER(_RunOpts), vp, ctypes.c_size_t,
                                    ctypes.c_int64, vp, vp, vp, vp, vp, vp]
+        L.sjq_run_hashed_static.restype = ctypes.c_int32
+        L.sjq_run_hashed_static.argtypes = [ctypes.POINTER(_Col), ip, ctypes.POINTER(_Pred), ip,
+                                            ctypes.POINTER(_Join), ip, ctypes.POINTER(_KeyExpr),
+                                            ctypes.POINTER(_AggExpr), ctypes.c_int64, ctypes.POINTER(_Result),
+                                            ctypes.POINTER(_RunOpts), vp, ctypes.POINTER(RunInfo)]
         L.sjq_strerror.restype = ctypes.c_char_p
         L.sjq_strerror.argtypes = [ctypes.c_int32]
         L.sjq_version.restype = ctypes.c_char_p
@@ -342,6 +347,47 @@ def run(fact: dict, preds=(), joins=(), key=None, agg=None, mode: str = "SCALAR"
         if rc != 0:
             raise SjqError(rc, "sjq_run")
     return res
+
+
+STATIC_MAX_GROUPS = 65536
+
+
+def run_hashed_static(fact: dict, preds=(), joins=(), key=None, agg=None, capacity: int = 0,
+                      opts: Optional[RunOpts] = None, result: Optional[Result] = None) -> Result:
+    """sjq_run_hashed_static: a hashed group-by whose group table is a fixed array inside the library,
+    for callers that cannot allocate device memory.  The caller still supplies the result arrays
+    (`result`, or fresh tensors here for convenience); no workspace is passed.  At most
+    STATIC_MAX_GROUPS groups; calls must not overlap on the GPU because they share the one table."""
+    names = list(fact.keys())
+    tensors = [fact[n] for n in names]
+    device = tensors[0].device
+    with torch.cuda.device(device):
+        carr = _cols(tensors)
+        parr, keep = _preds(preds, names)
+        jarr = (_Join * max(1, len(joins)))()
+        for j, (fk, table) in enumerate(joins):
+            jarr[j] = _Join(names.index(fk), table.handle)
+        kexpr = _KeyExpr()
+        for i, t in enumerate(key.terms):
+            kexpr.t[i] = _term(t, names)
+        kexpr.nterms, kexpr.offset, kexpr.modulo = len(key.terms), key.offset, key.modulo
+        aexpr = _AggExpr(AGGS[agg.op], _term(agg.x, names), _term(agg.y, names), int(agg.want_count))
+        if result is None:
+            n = max(1, capacity)
+            result = Result("HASHED", torch.empty(n, dtype=torch.int64, device=device),
+                            torch.empty(n, dtype=torch.int64, device=device),
+                            torch.empty(n, dtype=torch.int64, device=device),
+                            torch.zeros(1, dtype=torch.int64, device=device),
+                            torch.zeros(1, dtype=torch.int32, device=device), None)
+        cres = _Result(result.sums.data_ptr(), result.counts.data_ptr(), result.keys.data_ptr(),
+                       result.n_groups.data_ptr(), result.status_dev.data_ptr(), None, 0)
+        copts = (opts or RunOpts()).to_c()
+        rc = lib().sjq_run_hashed_static(carr, len(names), parr, len(preds), jarr, len(joins), ctypes.byref(kexpr),
+                                         ctypes.byref(aexpr), capacity, ctypes.byref(cres), ctypes.byref(copts),
+                                         _stream_ptr(device), ctypes.byref(result.info))
+        if rc != 0:
+            raise SjqError(rc, "sjq_run_hashed_static")
+    return result
 
 
 @dataclass
