@@ -169,6 +169,21 @@ sjq_status sjq_dim_plan(const sjq_col *cols, int ncols, const sjq_pred *preds, i
                         void *stream, sjq_dim_layout *layout);
 
 /*
+ * The same in two halves, so that several dimensions can be planned with one
+ * wait: `_begin` enqueues the scan on `stream` and an asynchronous copy of the
+ * eight int64 statistics into `host_stats` (page-locked host memory, 64 bytes)
+ * and returns at once; after the caller has synchronised that stream (or an
+ * event recorded on it), `_end` turns the statistics into the layout on the
+ * host.  `cols`/`ncols`/`key_col`/`npayload`/`opts` must describe the same
+ * dimension in both calls.
+ */
+sjq_status sjq_dim_plan_begin(const sjq_col *cols, int ncols, const sjq_pred *preds, int npreds, int key_col,
+                              const int *payload_cols, int npayload, void *scratch_dev, int64_t *host_stats,
+                              void *stream);
+sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_col, int npayload, const sjq_build_opts *opts,
+                            const int64_t *host_stats, sjq_dim_layout *layout);
+
+/*
  * Build the table described by `layout` into caller memory `table_mem`
  * (>= layout->table_bytes, else BUFFER_SMALL) and return a handle.  Enqueues
  * a fill, the build kernel and a verification kernel; does not synchronise.
@@ -247,8 +262,9 @@ typedef struct sjq_run_info {
     int32_t nstages;
     int32_t order[SJQ_MAX_PREDS + SJQ_MAX_JOINS + 8]; /* as in sjq_run_opts.order; -1 = plain column load */
     int32_t stage_in_smem[SJQ_MAX_PREDS + SJQ_MAX_JOINS + 8];
-    int32_t first_sparse_stage; /* number of queue-fed levels: stage 0 is dense, stages 1 .. this-1 are
-                                   queue-fed filters, later stages run at the final level; 0 = no queues */
+    int32_t first_sparse_stage; /* stages before this one filter thread-owned rows (level 0); later stages run
+                                   on compacted survivors; 0 = no queues at all */
+    int32_t reserved_levels;    /* number of queue-fed levels (the last one is the final level) */
     int32_t agg_path;           /* 0 scalar registers, 1 shared-memory table, 2 global atomics, 3 global hash */
     int32_t grid, block;
     int32_t smem_bytes;

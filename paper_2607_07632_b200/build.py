@@ -24,7 +24,8 @@ def _deps() -> list[str]:
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and os.path.exists(LIB) and all(os.path.getmtime(d) <= os.path.getmtime(LIB) for d in _deps()):
         return LIB
-    cmd = ["nvcc", *NVCC_FLAGS, "-I" + os.path.join(ROOT, "include"), "-o", LIB, *sources()]
+    extra = os.environ.get("SJQ_NVCC_EXTRA", "").split()  # e.g. -D switches for kernel experiments
+    cmd = ["nvcc", *NVCC_FLAGS, *extra, "-I" + os.path.join(ROOT, "include"), "-o", LIB, *sources()]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

@@ -386,11 +386,11 @@ sjq_status device_info(DeviceInfo *out)
 
 using namespace sjq;
 
-extern "C" sjq_status sjq_dim_plan(const sjq_col *cols, int ncols, const sjq_pred *preds, int npreds, int key_col,
-                                   const int *payload_cols, int npayload, const sjq_build_opts *opts,
-                                   void *scratch_dev, void *stream_, sjq_dim_layout *layout)
+extern "C" sjq_status sjq_dim_plan_begin(const sjq_col *cols, int ncols, const sjq_pred *preds, int npreds,
+                                         int key_col, const int *payload_cols, int npayload, void *scratch_dev,
+                                         int64_t *host_stats, void *stream_)
 {
-    if (!layout || !scratch_dev) return SJQ_ERR_INVALID_ARG;
+    if (!scratch_dev || !host_stats) return SJQ_ERR_INVALID_ARG;
     if (!aligned16(scratch_dev)) return SJQ_ERR_ALIGN;
     DimParams P{};
     sjq_status st = fill_dim_params(cols, ncols, preds, npreds, key_col, payload_cols, npayload, &P);
@@ -401,13 +401,36 @@ extern "C" sjq_status sjq_dim_plan(const sjq_col *cols, int ncols, const sjq_pre
     int64_t *scratch = static_cast<int64_t *>(scratch_dev);
     plan_init_kernel<<<1, 32, 0, stream>>>(scratch);
     if (P.n > 0) plan_scan_kernel<<<grid_for(P.n, dev.sm_count), 256, 0, stream>>>(P, scratch);
-    int64_t h[8];
     if (cudaGetLastError() != cudaSuccess ||
-        cudaMemcpyAsync(h, scratch, sizeof(h), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-        cudaStreamSynchronize(stream) != cudaSuccess) {
+        cudaMemcpyAsync(host_stats, scratch, 8 * sizeof(int64_t), cudaMemcpyDeviceToHost, stream) != cudaSuccess) {
         (void)cudaGetLastError();
         return SJQ_ERR_CUDA;
     }
+    return SJQ_OK;
+}
+
+extern "C" sjq_status sjq_dim_plan(const sjq_col *cols, int ncols, const sjq_pred *preds, int npreds, int key_col,
+                                   const int *payload_cols, int npayload, const sjq_build_opts *opts,
+                                   void *scratch_dev, void *stream_, sjq_dim_layout *layout)
+{
+    int64_t h[8];
+    sjq_status st = sjq_dim_plan_begin(cols, ncols, preds, npreds, key_col, payload_cols, npayload, scratch_dev, h,
+                                       stream_);
+    if (st != SJQ_OK) return st;
+    if (cudaStreamSynchronize((cudaStream_t)stream_) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SJQ_ERR_CUDA;
+    }
+    return sjq_dim_plan_end(cols, ncols, key_col, npayload, opts, h, layout);
+}
+
+extern "C" sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_col, int npayload,
+                                       const sjq_build_opts *opts, const int64_t *h, sjq_dim_layout *layout)
+{
+    if (!layout || !h || !cols || ncols <= 0 || key_col < 0 || key_col >= ncols || npayload < 0 ||
+        npayload > SJQ_MAX_PAYLOADS)
+        return SJQ_ERR_INVALID_ARG;
+    struct { int64_t n; } P{cols[key_col].n};
 
     sjq_dim_layout L{};
     L.key_dtype = cols[key_col].dtype;

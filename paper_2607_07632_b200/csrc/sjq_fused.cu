@@ -237,11 +237,35 @@ __device__ __forceinline__ uint32_t run_stage(const RunParams &P, const DStage &
 
 // ------------------------------------------------------------------ accumulators
 
+// Feed one row's values into the accumulators.  acc32: every multiplier of the
+// stage and every value it can see fits in 32 bits, so each contribution is one
+// widening multiply-add.
 template <bool MUL>
 __device__ __forceinline__ void accumulate(const DStage &S, int64_t raw, uint64_t code, int64_t &key, int64_t &X,
                                            int64_t &Y)
 {
     const uint32_t acc = S.acc;
+    if (S.acc32) {
+        if (acc & 0x7u) {
+            const int32_t r = (int32_t)raw;
+            if (acc & 1u) key += (int64_t)S.mult32[0] * r;
+            if (acc & 2u) X += (int64_t)S.mult32[1] * r;
+            if (MUL && (acc & 4u)) Y += (int64_t)S.mult32[2] * r;
+        }
+        if (acc & 0x38u) {
+            const int32_t p0 = (int32_t)((uint32_t)code & (uint32_t)S.pmask0) + (int32_t)S.pmin0;
+            if (acc & 8u) key += (int64_t)S.mult32[3] * p0;
+            if (acc & 16u) X += (int64_t)S.mult32[4] * p0;
+            if (MUL && (acc & 32u)) Y += (int64_t)S.mult32[5] * p0;
+        }
+        if (acc & 0x1C0u) {
+            const int32_t p1 = (int32_t)((uint32_t)(code >> S.pbits0)) + (int32_t)S.pmin1;
+            if (acc & 64u) key += (int64_t)S.mult32[6] * p1;
+            if (acc & 128u) X += (int64_t)S.mult32[7] * p1;
+            if (MUL && (acc & 256u)) Y += (int64_t)S.mult32[8] * p1;
+        }
+        return;
+    }
     if (acc & 0x7u) {
         if (acc & 1u) key += S.mult[0] * raw;
         if (acc & 2u) X += S.mult[1] * raw;
@@ -453,36 +477,53 @@ __device__ __forceinline__ void final_rows(const RunParams &P, const DStage *st,
 }
 
 // ------------------------------------------------------------------ level 0
-// The first stage on the thread's own kSlots groups of four consecutive rows
-// of a tile.  FULL: the whole tile lies inside the table (no bounds masks).
+// One filter stage on the thread's own kSlots groups of four consecutive rows
+// of a tile: the column is loaded for a group only while one of its rows is
+// alive.  FULL: the whole tile lies inside the table (no bounds masks).
 template <typename T, bool FULL>
 __device__ __forceinline__ uint32_t dense_stage(const RunParams &P, const DStage &S, const unsigned char *smem,
-                                                int64_t row0, int32_t slot_stride, uint32_t valid)
+                                                int64_t row0, int32_t slot_stride, uint32_t valid, uint32_t alive)
 {
     T v[kDenseRows];
     const T *c = static_cast<const T *>(S.col) + row0;
 #pragma unroll
     for (int u = 0; u < kSlots; ++u) {
-        if (FULL) {
-            Vec4<T>::load(c + u * slot_stride, &v[4 * u]);
-        } else {
-            const uint32_t nv = (valid >> (4 * u)) & 0xFu;
 #pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                v[4 * u + r] = 0;
-                if ((nv >> r) & 1u) v[4 * u + r] = __ldcs(c + u * slot_stride + r);
+        for (int r = 0; r < 4; ++r) v[4 * u + r] = 0;
+        if ((alive >> (4 * u)) & 0xFu) {
+            if (FULL) {
+                Vec4<T>::load(c + u * slot_stride, &v[4 * u]);
+            } else {
+                const uint32_t nv = (valid >> (4 * u)) & 0xFu;
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+                    if ((nv >> r) & 1u) v[4 * u + r] = __ldcs(c + u * slot_stride + r);
             }
         }
     }
     uint64_t unused[kDenseRows];
-    return run_stage<T, kDenseRows, false>(P, S, smem, v, valid, unused);
+    return run_stage<T, kDenseRows, false>(P, S, smem, v, alive, unused);
+}
+
+template <bool FULL>
+__device__ __forceinline__ uint32_t level0(const RunParams &P, const DStage *st, const unsigned char *smem,
+                                           int64_t row0, int32_t slot_stride, uint32_t valid)
+{
+    uint32_t alive = valid;
+    for (int s = 0; s < P.nd0; ++s) {
+        if (!alive) break;
+        const DStage &S = st[s];
+        alive = S.is64 ? dense_stage<int64_t, FULL>(P, S, smem, row0, slot_stride, valid, alive)
+                       : dense_stage<int32_t, FULL>(P, S, smem, row0, slot_stride, valid, alive);
+    }
+    return alive;
 }
 
 // ------------------------------------------------------------------ per-warp queues
 // Queue l of a warp (a ring of 32-bit row offsets in shared memory) holds the
-// rows that passed stages 0 .. l.  The level fed by queue l runs filter stage
-// l+1 and pushes to queue l+1, or, for the last queue, runs the remaining
-// stages and the terminal.  Heads and counts live in registers and are
+// rows that passed stages 0 .. nd0+l-1.  The level fed by queue l runs filter
+// stage nd0+l and pushes to queue l+1, or, for the last queue, runs the
+// remaining stages and the terminal.  Heads and counts live in registers and are
 // selected without indexing so that they never spill to local memory.
 struct QueueState {
     uint32_t h0, h1, h2, c0, c1, c2;
@@ -501,8 +542,12 @@ struct QueueState {
         c2 = l == 2 ? v : c2;
     }
 };
+
 __device__ __forceinline__ uint32_t queue_cap(int l) { return l == 0 ? (uint32_t)kQueue0Cap : (uint32_t)kQueueCap; }
-__device__ __forceinline__ uint32_t queue_base(int l) { return l == 0 ? 0u : (uint32_t)(kQueue0Cap + (l - 1) * kQueueCap); }
+__device__ __forceinline__ uint32_t queue_base(int l)
+{
+    return l == 0 ? 0u : (uint32_t)(kQueue0Cap + (l - 1) * kQueueCap);
+}
 
 template <int AGG, bool MUL>
 __global__ void __launch_bounds__(512, 2) fused_kernel(const __grid_constant__ RunParams P)
@@ -586,11 +631,9 @@ __global__ void __launch_bounds__(512, 2) fused_kernel(const __grid_constant__ R
                     const int64_t tile_base = (int64_t)tile * tile_rows;
                     const int64_t row0 = tile_base + 4 * tid;
                     if (wide) qbase = tile_base;
-                    const DStage &S = st[0];
                     uint32_t alive;
                     if (tile_base + tile_rows <= P.n) {
-                        alive = S.is64 ? dense_stage<int64_t, true>(P, S, smem, row0, slot_stride, 0xFFu)
-                                       : dense_stage<int32_t, true>(P, S, smem, row0, slot_stride, 0xFFu);
+                        alive = level0<true>(P, st, smem, row0, slot_stride, kDenseRows >= 32 ? 0xFFFFFFFFu : ((1u << kDenseRows) - 1u));
                     } else {
                         uint32_t valid = 0;
 #pragma unroll
@@ -599,9 +642,13 @@ __global__ void __launch_bounds__(512, 2) fused_kernel(const __grid_constant__ R
                             const uint32_t nv = rem >= 4 ? 0xFu : (rem > 0 ? ((1u << (int)rem) - 1u) : 0u);
                             valid |= nv << (4 * k);
                         }
-                        alive = S.is64 ? dense_stage<int64_t, false>(P, S, smem, row0, slot_stride, valid)
-                                       : dense_stage<int32_t, false>(P, S, smem, row0, slot_stride, valid);
+                        alive = level0<false>(P, st, smem, row0, slot_stride, valid);
                     }
+#if defined(SJQ_EXP_NO_QUEUE)
+                    lcnt += __popc(alive);
+                    tile += gridDim.x;
+                    continue;
+#endif
                     // compact the warp's survivors into queue 0
                     const uint32_t mine = (uint32_t)__popc(alive);
                     uint32_t incl = mine;
@@ -654,9 +701,9 @@ __global__ void __launch_bounds__(512, 2) fused_kernel(const __grid_constant__ R
                 Q.set_count(l, Q.count(l) - nb);
             }
             if (l + 1 == nq) {
-                final_rows<AGG, MUL, false>(P, st, smem, nq, qbase, off, valid, lsum, lcnt);
+                final_rows<AGG, MUL, false>(P, st, smem, P.nd0 + l, qbase, off, valid, lsum, lcnt);
             } else {
-                const uint32_t m = filter_rows(P, st[l + 1], smem, qbase, off, valid);
+                const uint32_t m = filter_rows(P, st[P.nd0 + l], smem, qbase, off, valid);
                 const uint32_t mine = (uint32_t)__popc(m);
                 uint32_t incl = mine;
 #pragma unroll

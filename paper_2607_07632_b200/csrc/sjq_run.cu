@@ -264,22 +264,26 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     std::vector<double> reach(nfilter + 1, 1.0);
     for (int s = 0; s < nfilter; ++s) reach[s + 1] = reach[s] * specs[order[s]].sel;
     const double survivors = (double)n * reach[nfilter];
-    // Stage 0 filters thread-owned rows (level 0); up to kMaxQueues - 1 further
-    // stages run as queue-fed pure filters while they really filter and enough
-    // rows still reach them; everything after runs at the final level.  Eager
-    // loading and compaction = never use no queue at all.
-    int ndense = 0;
+    // Level 0 runs, on thread-owned rows, the leading filter stages that still see a fair share of
+    // the rows (a dense stage costs about the same per table row whatever survives, a queue-fed
+    // level costs per surviving row, roughly fifteen times more: measured break-even near 6 %).
+    // Up to kMaxQueues - 1 later filter stages run as queue-fed levels; the rest at the final level.
+    // Eager loading and compaction = never use no queue at all.
+    int nd0 = 0, nfq = 0;
     const bool direct = opts.eager_loads || opts.compaction == 1 || nfilter == 0;
     if (!direct) {
-        ndense = 1;
+        nd0 = 1;
         if (opts.compaction != 2) {
-            for (int s = 1; s < nfilter && s < kMaxQueues; ++s) {
-                if (specs[order[s]].sel < 0.9 && reach[s] > 0.01) ndense = s + 1;
-                else break;
-            }
+            const double dense_reach = opts.reserved[0] > 0 ? opts.reserved[0] / 1000.0 : 0.06;
+            while (nd0 < nfilter && specs[order[nd0]].sel < 0.9 && reach[nd0] > dense_reach) ++nd0;
+            while (nd0 + nfq < nfilter && nfq < kMaxQueues - 1 && specs[order[nd0 + nfq]].sel < 0.9 &&
+                   reach[nd0 + nfq] > 0.002)
+                ++nfq;
         }
     }
-    P.nq = ndense;
+    const int ndense = nd0 + nfq; // stages that only filter (no accumulators)
+    P.nd0 = nd0;
+    P.nq = direct ? 0 : nfq + 1;
 
     // Sources of the accumulators.  A dense stage cannot feed an accumulator
     // (it only keeps a bit per row), so a value it would supply is gathered
@@ -328,6 +332,24 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
             S.kind = ST_LOAD;
             S.op = OP_LOAD;
         }
+    }
+    // 32-bit fast path of the accumulators: int32 column, multipliers and payload ranges within int32
+    for (int s2 = 0; s2 < ns; ++s2) {
+        DStage &S = P.st[s2];
+        bool ok = !S.is64;
+        for (int i = 0; i < 9; ++i) {
+            ok = ok && S.mult[i] >= INT32_MIN && S.mult[i] <= INT32_MAX;
+            S.mult32[i] = (int32_t)S.mult[i];
+        }
+        if (S.kind == ST_PROBE) {
+            const int64_t hi0 = S.pmin0 + (int64_t)std::min<uint64_t>(S.pmask0, (uint64_t)INT32_MAX);
+            ok = ok && S.code_bits <= 32 && S.pmin0 >= INT32_MIN && hi0 <= INT32_MAX && S.pmask0 <= 0x7FFFFFFFull;
+            if (S.acc & 0x1C0u) {
+                const int bits1 = (int)S.code_bits - (int)S.pbits0;
+                ok = ok && bits1 < 31 && S.pmin1 >= INT32_MIN && S.pmin1 + ((int64_t)1 << std::max(bits1, 0)) <= INT32_MAX;
+            }
+        }
+        S.acc32 = ok ? 1 : 0;
     }
     P.nstages = ns;
     P.eager = opts.eager_loads ? 1 : 0;
@@ -465,7 +487,8 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
             info->order[s] = stage_label[s];
             info->stage_in_smem[s] = P.st[s].in_smem;
         }
-        info->first_sparse_stage = P.nq;
+        info->first_sparse_stage = P.nq ? P.nd0 : 0;
+        info->reserved_levels = P.nq;
         info->agg_path = aggp;
         info->grid = grid;
         info->block = block;

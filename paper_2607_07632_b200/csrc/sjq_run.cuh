@@ -34,12 +34,15 @@ constexpr int kAccKey = 0, kAccX = 1, kAccY = 2;
 constexpr int kMaxStages = SJQ_MAX_PREDS + SJQ_MAX_JOINS + 8 + SJQ_MAX_JOINS + SJQ_MAX_PREDS;
 
 // Geometry of the fused kernel.
-constexpr int kSlots = 2;                // level 0: 128-bit loads per thread per tile
+#ifndef SJQ_SLOTS
+#define SJQ_SLOTS 2
+#endif
+constexpr int kSlots = SJQ_SLOTS;        // level 0: 128-bit loads per thread per tile
 constexpr int kDenseRows = 4 * kSlots;   // rows a thread owns at level 0
 constexpr int kRows = 4;                 // rows a lane handles per batch at the queue-fed levels
 constexpr int kBatch = 32 * kRows;       // rows a warp processes at once at those levels
-constexpr int kQueue0Cap = 512;          // entries of a warp's first queue: a batch minus one plus a whole tile
-constexpr int kQueueCap = 256;           // entries of its later queues: a batch minus one plus a batch
+constexpr int kQueue0Cap = kSlots <= 2 ? 512 : 1024; // first queue of a warp: a batch minus one plus a whole tile fit
+constexpr int kQueueCap = 256;           // its later queues: a batch minus one plus a batch fit
 constexpr int kMaxQueues = 3;            // queue-fed levels per warp (the last one is the final level)
 
 struct DStage {
@@ -53,6 +56,8 @@ struct DStage {
     int64_t pmin0, pmin1;
     uint64_t pmask0;
     int64_t mult[9];
+    int32_t mult32[9]; // the same multipliers when acc32
+    int32_t acc32;     // every multiplier, raw value and payload of this stage fits in 32 bits
     int32_t lo32;      // 32-bit predicate: pass iff (uint32)(v - lo32) <= width32
     uint32_t width32;
     int32_t kmin32;    // 32-bit direct probe: idx = (uint32)v - (uint32)kmin32, hit range idx <= last32
@@ -77,8 +82,10 @@ struct RunParams {
     int64_t *gkeys;  // hashed: table keys
     int32_t *status;
     int32_t nstages;
-    int32_t nq;     // queue-fed levels: 0 = none (every stage on thread-owned rows); else stage 0 is the
-                    // dense level, stages 1 .. nq-1 are queue-fed filters, stages nq .. run at the final level
+    int32_t nq;     // queue-fed levels: 0 = none (every stage on thread-owned rows); else stages 0 .. nd0-1
+                    // filter thread-owned rows at level 0, stages nd0 .. nd0+nq-2 are queue-fed filters and
+                    // stages from nd0+nq-1 on run at the final level
+    int32_t nd0;
     int32_t want_count;
     int32_t eager;   // load every column for every row
     int32_t has_key; // scalar path of a one-group dense result: key is computed and range-checked

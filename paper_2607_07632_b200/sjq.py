@@ -97,12 +97,13 @@ class _RunOpts(ctypes.Structure):
 class RunInfo(ctypes.Structure):
     _fields_ = [("nstages", ctypes.c_int32), ("order", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS + 8)),
                 ("stage_in_smem", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS + 8)),
-                ("first_sparse_stage", ctypes.c_int32), ("agg_path", ctypes.c_int32), ("grid", ctypes.c_int32),
+                ("first_sparse_stage", ctypes.c_int32), ("reserved_levels", ctypes.c_int32),
+                ("agg_path", ctypes.c_int32), ("grid", ctypes.c_int32),
                 ("block", ctypes.c_int32), ("smem_bytes", ctypes.c_int32), ("kernel_launches", ctypes.c_int32)]
 
     def describe(self) -> dict:
         return {"order": list(self.order[: self.nstages]), "in_smem": list(self.stage_in_smem[: self.nstages]),
-                "first_sparse_stage": self.first_sparse_stage, "agg_path": AGG_PATHS.get(self.agg_path),
+                "first_sparse_stage": self.first_sparse_stage, "queue_levels": self.reserved_levels, "agg_path": AGG_PATHS.get(self.agg_path),
                 "grid": self.grid, "block": self.block, "smem_bytes": self.smem_bytes,
                 "kernel_launches": self.kernel_launches}
 
@@ -118,6 +119,7 @@ class RunOpts:
     accumulate: bool = False
     order: Sequence[int] = ()
     events: Optional[tuple] = None  # (torch.cuda.Event, torch.cuda.Event), both already recorded once
+    dense_reach_permille: int = 0  # experiment knob: level 0 keeps stages reached by more than this share of rows
 
     def to_c(self) -> _RunOpts:
         o = _RunOpts()
@@ -127,6 +129,7 @@ class RunOpts:
         o.norder = len(self.order)
         for i, v in enumerate(self.order):
             o.order[i] = v
+        o.reserved[0] = self.dense_reach_permille
         if self.events is not None:
             o.event_before, o.event_after = self.events[0].cuda_event, self.events[1].cuda_event
         return o
@@ -147,6 +150,12 @@ def lib():
         L.sjq_dim_plan.restype = ctypes.c_int32
         L.sjq_dim_plan.argtypes = [ctypes.POINTER(_Col), ip, ctypes.POINTER(_Pred), ip, ip, ctypes.POINTER(ip), ip,
                                    ctypes.POINTER(_BuildOpts), vp, vp, ctypes.POINTER(DimLayout)]
+        L.sjq_dim_plan_begin.restype = ctypes.c_int32
+        L.sjq_dim_plan_begin.argtypes = [ctypes.POINTER(_Col), ip, ctypes.POINTER(_Pred), ip, ip, ctypes.POINTER(ip),
+                                         ip, vp, vp, vp]
+        L.sjq_dim_plan_end.restype = ctypes.c_int32
+        L.sjq_dim_plan_end.argtypes = [ctypes.POINTER(_Col), ip, ip, ip, ctypes.POINTER(_BuildOpts), vp,
+                                       ctypes.POINTER(DimLayout)]
         L.sjq_build_dim.restype = ctypes.c_int32
         L.sjq_build_dim.argtypes = [ctypes.POINTER(_Col), ip, ctypes.POINTER(_Pred), ip, ip, ctypes.POINTER(ip), ip,
                                     ctypes.POINTER(DimLayout), vp, ctypes.c_size_t, vp, vp, ctypes.POINTER(vp)]
@@ -256,6 +265,75 @@ def build_dim(cols: dict, key: str, preds=(), payloads=(), force_kind: int = 0, 
         if rc != 0:
             raise SjqError(rc, "sjq_build_dim")
     return Table(handle.value, layout, mem, status)
+
+
+class TableBuilder:
+    """A dimension prepared for repeated builds: the argument structures are marshalled once, scratch,
+    statistics and table memory are kept, and plan + build run on a side stream so that several
+    dimensions can be planned with a single wait (sjq_dim_plan_begin / _end, sjq_build_dim)."""
+
+    def __init__(self, cols: dict, key: str, preds=(), payloads=(), force_kind: int = 0, hash_load_pct: int = 0,
+                 max_direct_bytes: int = 0):
+        self.names = list(cols.keys())
+        self.tensors = [cols[n] for n in self.names]
+        self.device = self.tensors[0].device
+        with torch.cuda.device(self.device):
+            self.carr = _cols(self.tensors)
+            self.parr, self._keep = _preds(preds, self.names)
+            self.npreds, self.npay = len(preds), len(payloads)
+            self.key_col = self.names.index(key)
+            self.pay = (ctypes.c_int * max(1, len(payloads)))(*[self.names.index(p) for p in payloads])
+            self.opts = _BuildOpts(force_kind, hash_load_pct, max_direct_bytes)
+            self.scratch = torch.empty(PLAN_SCRATCH_BYTES, dtype=torch.uint8, device=self.device)
+            self.stats = torch.zeros(8, dtype=torch.int64, pin_memory=True)
+            self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
+            self.side = torch.cuda.Stream(self.device)
+            self.mem = None
+            self.layout = DimLayout()
+
+    def begin(self):
+        """Enqueue the key-range scan on the side stream (after everything queued on the current stream)."""
+        self.side.wait_stream(torch.cuda.current_stream(self.device))
+        rc = lib().sjq_dim_plan_begin(self.carr, len(self.names), self.parr, self.npreds, self.key_col, self.pay,
+                                      self.npay, self.scratch.data_ptr(), self.stats.data_ptr(),
+                                      self.side.cuda_stream)
+        if rc != 0:
+            raise SjqError(rc, "sjq_dim_plan_begin")
+
+    def finish(self) -> Table:
+        """Wait for the scan, choose the layout, enqueue the build on the side stream."""
+        self.side.synchronize()
+        rc = lib().sjq_dim_plan_end(self.carr, len(self.names), self.key_col, self.npay, ctypes.byref(self.opts),
+                                    self.stats.data_ptr(), ctypes.byref(self.layout))
+        if rc != 0:
+            raise SjqError(rc, "sjq_dim_plan_end")
+        if self.mem is None or self.mem.numel() < self.layout.table_bytes:
+            with torch.cuda.device(self.device):
+                self.mem = torch.empty(self.layout.table_bytes, dtype=torch.uint8, device=self.device)
+        handle = ctypes.c_void_p()
+        rc = lib().sjq_build_dim(self.carr, len(self.names), self.parr, self.npreds, self.key_col, self.pay,
+                                 self.npay, ctypes.byref(self.layout), self.mem.data_ptr(), self.mem.numel(),
+                                 self.status.data_ptr(), self.side.cuda_stream, ctypes.byref(handle))
+        if rc != 0:
+            raise SjqError(rc, "sjq_build_dim")
+        layout = DimLayout.from_buffer_copy(self.layout)
+        return Table(handle.value, layout, self.mem, self.status)
+
+
+def workload_builders(w, dims: dict) -> dict:
+    return {d.name: TableBuilder(dims[d.name], d.key, d.preds, d.payloads,
+                                 force_kind=FORCE_HASH if d.force_hash else 0) for d in w.dims}
+
+
+def build_tables(builders: dict) -> dict:
+    """Plan all dimensions (one wait each, scans overlapping on side streams), build them concurrently,
+    and make the current stream wait for the builds."""
+    for b in builders.values():
+        b.begin()
+    tables = {name: b.finish() for name, b in builders.items()}
+    for b in builders.values():
+        torch.cuda.current_stream(b.device).wait_stream(b.side)
+    return tables
 
 
 @dataclass

@@ -248,3 +248,20 @@ def test_event_hooks_bracket_the_fused_kernel():
     sjq.run_workload(w, fact, tables, sjq.RunOpts(events=(a, b)))
     torch.cuda.synchronize()
     assert 0.0 < a.elapsed_time(b) < 1000.0
+
+
+def test_prepared_builders_rebuild_identical_tables():
+    w = W.config3(400_003)
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    res, exp, tables = run_both(w, fact, hd)
+    builders = sjq.workload_builders(w, {k: to_dev(v) for k, v in hd.items()})
+    dev_fact = to_dev(fact)
+    for _ in range(3):  # rebuilding into the same memory, back to back with runs
+        tabs = sjq.build_tables(builders)
+        r = sjq.run_workload(w, dev_fact, tabs)
+    torch.cuda.synchronize()
+    assert all(t.status() == 0 for t in tabs.values())
+    for k in tabs:
+        assert tabs[k].layout.entries == tables[k].layout.entries and tabs[k].layout.kind == tables[k].layout.kind
+    compare(w, r, exp)
