@@ -30,6 +30,14 @@
 
 #include "sjq_run.cuh"
 
+#ifndef SJQ_LB_THREADS
+#define SJQ_LB_THREADS 384
+#define SJQ_LB_BLOCKS 2
+#endif
+#ifndef SJQ_PREFETCH_DIST
+#define SJQ_PREFETCH_DIST 2
+#endif
+
 namespace sjq {
 
 namespace {
@@ -237,51 +245,85 @@ __device__ __forceinline__ uint32_t run_stage(const RunParams &P, const DStage &
 
 // ------------------------------------------------------------------ accumulators
 
-// Feed one row's values into the accumulators.  acc32: every multiplier of the
-// stage and every value it can see fits in 32 bits, so each contribution is one
-// widening multiply-add.
-template <bool MUL>
-__device__ __forceinline__ void accumulate(const DStage &S, int64_t raw, uint64_t code, int64_t &key, int64_t &X,
-                                           int64_t &Y)
+// Feed a batch's values into the accumulators.  Every test on the stage's
+// recipe is uniform and sits outside the row loop; a row contributes iff its
+// bit is set in m.  acc32: every multiplier of the stage and every value it
+// can see fits in 32 bits, so a contribution is one widening multiply-add.
+template <int NR, typename V>
+__device__ __forceinline__ void add_scaled(int64_t (&dst)[NR], int64_t mult, const V (&val)[NR], uint32_t m)
+{
+#pragma unroll
+    for (int k = 0; k < NR; ++k)
+        if ((m >> k) & 1u) dst[k] += mult * (int64_t)val[k];
+}
+template <int NR>
+__device__ __forceinline__ void add_scaled32(int64_t (&dst)[NR], int32_t mult, const int32_t (&val)[NR], uint32_t m)
+{
+#pragma unroll
+    for (int k = 0; k < NR; ++k)
+        if ((m >> k) & 1u) dst[k] += (int64_t)mult * val[k]; // one widening multiply-add
+}
+
+template <bool MUL, typename T, int NR>
+__device__ __forceinline__ void accumulate(const DStage &S, const T (&v)[NR], const uint64_t (&code)[NR], uint32_t m,
+                                           int64_t (&key)[NR], int64_t (&X)[NR], int64_t (&Y)[NR])
 {
     const uint32_t acc = S.acc;
-    if (S.acc32) {
+    if (S.acc32 && sizeof(T) == 4) {
         if (acc & 0x7u) {
-            const int32_t r = (int32_t)raw;
-            if (acc & 1u) key += (int64_t)S.mult32[0] * r;
-            if (acc & 2u) X += (int64_t)S.mult32[1] * r;
-            if (MUL && (acc & 4u)) Y += (int64_t)S.mult32[2] * r;
+            int32_t r[NR];
+#pragma unroll
+            for (int k = 0; k < NR; ++k) r[k] = (int32_t)v[k];
+            if (acc & 1u) add_scaled32<NR>(key, S.mult32[0], r, m);
+            if (acc & 2u) add_scaled32<NR>(X, S.mult32[1], r, m);
+            if (MUL && (acc & 4u)) add_scaled32<NR>(Y, S.mult32[2], r, m);
         }
         if (acc & 0x38u) {
-            const int32_t p0 = (int32_t)((uint32_t)code & (uint32_t)S.pmask0) + (int32_t)S.pmin0;
-            if (acc & 8u) key += (int64_t)S.mult32[3] * p0;
-            if (acc & 16u) X += (int64_t)S.mult32[4] * p0;
-            if (MUL && (acc & 32u)) Y += (int64_t)S.mult32[5] * p0;
+            const uint32_t mask0 = (uint32_t)S.pmask0;
+            const int32_t min0 = (int32_t)S.pmin0;
+            int32_t p0[NR];
+#pragma unroll
+            for (int k = 0; k < NR; ++k) p0[k] = (int32_t)((uint32_t)code[k] & mask0) + min0;
+            if (acc & 8u) add_scaled32<NR>(key, S.mult32[3], p0, m);
+            if (acc & 16u) add_scaled32<NR>(X, S.mult32[4], p0, m);
+            if (MUL && (acc & 32u)) add_scaled32<NR>(Y, S.mult32[5], p0, m);
         }
         if (acc & 0x1C0u) {
-            const int32_t p1 = (int32_t)((uint32_t)(code >> S.pbits0)) + (int32_t)S.pmin1;
-            if (acc & 64u) key += (int64_t)S.mult32[6] * p1;
-            if (acc & 128u) X += (int64_t)S.mult32[7] * p1;
-            if (MUL && (acc & 256u)) Y += (int64_t)S.mult32[8] * p1;
+            const uint32_t sh = S.pbits0;
+            const int32_t min1 = (int32_t)S.pmin1;
+            int32_t p1[NR];
+#pragma unroll
+            for (int k = 0; k < NR; ++k) p1[k] = (int32_t)((uint32_t)code[k] >> sh) + min1;
+            if (acc & 64u) add_scaled32<NR>(key, S.mult32[6], p1, m);
+            if (acc & 128u) add_scaled32<NR>(X, S.mult32[7], p1, m);
+            if (MUL && (acc & 256u)) add_scaled32<NR>(Y, S.mult32[8], p1, m);
         }
         return;
     }
     if (acc & 0x7u) {
-        if (acc & 1u) key += S.mult[0] * raw;
-        if (acc & 2u) X += S.mult[1] * raw;
-        if (MUL && (acc & 4u)) Y += S.mult[2] * raw;
+        if (acc & 1u) add_scaled<NR>(key, S.mult[0], v, m);
+        if (acc & 2u) add_scaled<NR>(X, S.mult[1], v, m);
+        if (MUL && (acc & 4u)) add_scaled<NR>(Y, S.mult[2], v, m);
     }
     if (acc & 0x38u) {
-        const int64_t p0 = (int64_t)(code & S.pmask0) + S.pmin0;
-        if (acc & 8u) key += S.mult[3] * p0;
-        if (acc & 16u) X += S.mult[4] * p0;
-        if (MUL && (acc & 32u)) Y += S.mult[5] * p0;
+        const uint64_t mask0 = S.pmask0;
+        const int64_t min0 = S.pmin0;
+        int64_t p0[NR];
+#pragma unroll
+        for (int k = 0; k < NR; ++k) p0[k] = (int64_t)(code[k] & mask0) + min0;
+        if (acc & 8u) add_scaled<NR>(key, S.mult[3], p0, m);
+        if (acc & 16u) add_scaled<NR>(X, S.mult[4], p0, m);
+        if (MUL && (acc & 32u)) add_scaled<NR>(Y, S.mult[5], p0, m);
     }
     if (acc & 0x1C0u) {
-        const int64_t p1 = (int64_t)(code >> S.pbits0) + S.pmin1;
-        if (acc & 64u) key += S.mult[6] * p1;
-        if (acc & 128u) X += S.mult[7] * p1;
-        if (MUL && (acc & 256u)) Y += S.mult[8] * p1;
+        const uint32_t sh = S.pbits0;
+        const int64_t min1 = S.pmin1;
+        int64_t p1[NR];
+#pragma unroll
+        for (int k = 0; k < NR; ++k) p1[k] = (int64_t)(code[k] >> sh) + min1;
+        if (acc & 64u) add_scaled<NR>(key, S.mult[6], p1, m);
+        if (acc & 128u) add_scaled<NR>(X, S.mult[7], p1, m);
+        if (MUL && (acc & 256u)) add_scaled<NR>(Y, S.mult[8], p1, m);
     }
 }
 
@@ -344,39 +386,87 @@ __device__ __forceinline__ void smem_add64(unsigned long long *cell, uint64_t va
     if (hi) atomicAdd(w + 1, hi);
 }
 
-template <int AGG, bool MUL>
-__device__ __forceinline__ void terminal(const RunParams &P, unsigned char *smem, int64_t key, int64_t X, int64_t Y,
-                                         int64_t &lsum, int64_t &lcnt)
+// The terminal on a batch: group keys of all rows first (their divisions overlap), then the
+// aggregation; every test on the query shape is uniform and outside the row loops.
+template <int AGG, bool MUL, int NR>
+__device__ __forceinline__ void terminal(const RunParams &P, unsigned char *smem, const int64_t (&key)[NR],
+                                         const int64_t (&X)[NR], const int64_t (&Y)[NR], uint32_t m, int64_t &lsum,
+                                         int64_t &lcnt)
 {
-    const int64_t val = MUL ? X * Y : X;
+    if (!m) return;
+    int64_t val[NR];
+#pragma unroll
+    for (int k = 0; k < NR; ++k) val[k] = MUL ? X[k] * Y[k] : X[k];
+    int64_t g[NR];
+    if (AGG != AGG_SCALAR || P.has_key) {
+        const int64_t modulo = P.modulo;
+        if (modulo == 0) {
+#pragma unroll
+            for (int k = 0; k < NR; ++k) g[k] = key[k];
+        } else if (P.modmask) {
+            const int64_t mask = (int64_t)P.modmask;
+#pragma unroll
+            for (int k = 0; k < NR; ++k) g[k] = key[k] >= 0 ? (key[k] & mask) : (key[k] % modulo);
+        } else if (P.mod32) {
+            const uint32_t d = (uint32_t)modulo;
+#pragma unroll
+            for (int k = 0; k < NR; ++k)
+                g[k] = (uint64_t)key[k] <= 0xFFFFFFFFull ? (int64_t)((uint32_t)key[k] % d) : (key[k] % modulo);
+        } else {
+#pragma unroll
+            for (int k = 0; k < NR; ++k) g[k] = key[k] % modulo;
+        }
+    }
     if (AGG == AGG_SCALAR) {
         if (P.has_key) {
-            const int64_t g = reduce_key(P, key);
-            if (g != 0) {
-                set_status(P.status, SJQ_ERR_GROUP_RANGE);
-                return;
-            }
+#pragma unroll
+            for (int k = 0; k < NR; ++k)
+                if (((m >> k) & 1u) && g[k] != 0) {
+                    set_status(P.status, SJQ_ERR_GROUP_RANGE);
+                    m &= ~(1u << k);
+                }
         }
-        lsum += val;
-        lcnt += 1;
+#pragma unroll
+        for (int k = 0; k < NR; ++k)
+            if ((m >> k) & 1u) lsum += val[k];
+        lcnt += __popc(m);
         return;
     }
-    const int64_t g = reduce_key(P, key);
     if (AGG == AGG_HASH) {
-        hash_aggregate(P, g, val);
+#pragma unroll
+        for (int k = 0; k < NR; ++k)
+            if ((m >> k) & 1u) hash_aggregate(P, g[k], val[k]);
         return;
     }
-    if ((uint64_t)g >= (uint64_t)P.num_groups) {
-        set_status(P.status, SJQ_ERR_GROUP_RANGE);
-        return;
-    }
+    const uint64_t ng = (uint64_t)P.num_groups;
+#pragma unroll
+    for (int k = 0; k < NR; ++k)
+        if (((m >> k) & 1u) && (uint64_t)g[k] >= ng) {
+            set_status(P.status, SJQ_ERR_GROUP_RANGE);
+            m &= ~(1u << k);
+        }
+    const bool want_count = P.want_count != 0;
     if (AGG == AGG_SMEM) {
         unsigned long long *ss = reinterpret_cast<unsigned long long *>(smem + P.smem_groups);
-        smem_add64(ss + g, (uint64_t)val);
-        if (P.want_count) smem_add64(ss + P.num_groups + g, 1ull);
+#pragma unroll
+        for (int k = 0; k < NR; ++k)
+            if ((m >> k) & 1u) smem_add64(ss + g[k], (uint64_t)val[k]);
+        if (want_count) {
+#pragma unroll
+            for (int k = 0; k < NR; ++k)
+                if ((m >> k) & 1u) smem_add64(ss + ng + g[k], 1ull);
+        }
     } else {
-        atomicAdd(reinterpret_cast<unsigned long long *>(P.sums) + g, (unsigned long long)val);
-        if (P.want_count) atomicAdd(reinterpret_cast<unsigned long long *>(P.counts) + g, 1ull);
+        unsigned long long *gs = reinterpret_cast<unsigned long long *>(P.sums);
+#pragma unroll
+        for (int k = 0; k < NR; ++k)
+            if ((m >> k) & 1u) atomicAdd(gs + g[k], (unsigned long long)val[k]);
+        if (want_count) {
+            unsigned long long *gc = reinterpret_cast<unsigned long long *>(P.counts);
+#pragma unroll
+            for (int k = 0; k < NR; ++k)
+                if ((m >> k) & 1u) atomicAdd(gc + g[k], 1ull);
+        }
     }
 }
 
@@ -448,11 +538,7 @@ __device__ __forceinline__ void final_rows(const RunParams &P, const DStage *st,
             load_rows<int64_t, CONTIG>(S, base, off, valid, need, v);
             have_next = false;
             m = run_stage<int64_t, kRows, true>(P, S, smem, v, m, code);
-            if (S.acc) {
-#pragma unroll
-                for (int k = 0; k < kRows; ++k)
-                    if ((m >> k) & 1u) accumulate<MUL>(S, v[k], code[k], key[k], X[k], Y[k]);
-            }
+            if (S.acc) accumulate<MUL, int64_t, kRows>(S, v, code, m, key, X, Y);
         } else {
             int32_t v[kRows];
             if (have_next) {
@@ -464,16 +550,10 @@ __device__ __forceinline__ void final_rows(const RunParams &P, const DStage *st,
             have_next = (s + 1 < P.nstages) && !st[s + 1].is64;
             if (have_next) load_rows<int32_t, CONTIG>(st[s + 1], base, off, valid, need, vnext);
             m = run_stage<int32_t, kRows, true>(P, S, smem, v, m, code);
-            if (S.acc) {
-#pragma unroll
-                for (int k = 0; k < kRows; ++k)
-                    if ((m >> k) & 1u) accumulate<MUL>(S, (int64_t)v[k], code[k], key[k], X[k], Y[k]);
-            }
+            if (S.acc) accumulate<MUL, int32_t, kRows>(S, v, code, m, key, X, Y);
         }
     }
-#pragma unroll
-    for (int k = 0; k < kRows; ++k)
-        if ((m >> k) & 1u) terminal<AGG, MUL>(P, smem, key[k], X[k], Y[k], lsum, lcnt);
+    terminal<AGG, MUL, kRows>(P, smem, key, X, Y, m, lsum, lcnt);
 }
 
 // ------------------------------------------------------------------ level 0
@@ -550,7 +630,7 @@ __device__ __forceinline__ uint32_t queue_base(int l)
 }
 
 template <int AGG, bool MUL>
-__global__ void __launch_bounds__(512, 2) fused_kernel(const __grid_constant__ RunParams P)
+__global__ void __launch_bounds__(SJQ_LB_THREADS, SJQ_LB_BLOCKS) fused_kernel(const __grid_constant__ RunParams P)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     const int tid = threadIdx.x;
@@ -631,6 +711,18 @@ __global__ void __launch_bounds__(512, 2) fused_kernel(const __grid_constant__ R
                     const int64_t tile_base = (int64_t)tile * tile_rows;
                     const int64_t row0 = tile_base + 4 * tid;
                     if (wide) qbase = tile_base;
+#if !defined(SJQ_NO_PREFETCH)
+                    {   // ask L2 for the first column of the tile this block filters next
+                        const int64_t nrow = row0 + (int64_t)gridDim.x * tile_rows * SJQ_PREFETCH_DIST;
+                        if (nrow + tile_rows <= P.n) {
+                            const DStage &S0 = st[0];
+                            const char *pc = static_cast<const char *>(S0.col) + nrow * (S0.is64 ? 8 : 4);
+#pragma unroll
+                            for (int k = 0; k < kSlots; ++k)
+                                asm volatile("prefetch.global.L2 [%0];" ::"l"(pc + (int64_t)k * slot_stride * (S0.is64 ? 8 : 4)));
+                        }
+                    }
+#endif
                     uint32_t alive;
                     if (tile_base + tile_rows <= P.n) {
                         alive = level0<true>(P, st, smem, row0, slot_stride, kDenseRows >= 32 ? 0xFFFFFFFFu : ((1u << kDenseRows) - 1u));

@@ -15,6 +15,12 @@
 
 #include "sjq_run.cuh"
 
+#ifndef SJQ_LB_THREADS
+#define SJQ_LB_THREADS_MAX 384
+#else
+#define SJQ_LB_THREADS_MAX SJQ_LB_THREADS
+#endif
+
 namespace sjq {
 
 sjq_status fused_occupancy(int agg, bool mul, int block, size_t smem, int *ctas_per_sm);
@@ -127,7 +133,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     }
     if (!valid_term(agg->x, nfact, joins, njoins)) return SJQ_ERR_INVALID_ARG;
     if (agg->op != SJQ_AGG_COL && !valid_term(agg->y, nfact, joins, njoins)) return SJQ_ERR_INVALID_ARG;
-    if (opts.block_threads && (opts.block_threads < 128 || opts.block_threads > 512 || opts.block_threads % 32))
+    if (opts.block_threads && (opts.block_threads < 128 || opts.block_threads > SJQ_LB_THREADS_MAX || opts.block_threads % 32))
         return SJQ_ERR_INVALID_ARG;
     if (opts.norder && opts.norder != npreds + njoins) return SJQ_ERR_INVALID_ARG;
 
@@ -404,7 +410,10 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
 
     // ------------------------------------------------------------ shared memory layout
     // [stage descriptors][staged tables][group table][per-warp survivor queues]
-    int block = opts.block_threads ? opts.block_threads : 512;
+    #ifndef SJQ_LB_THREADS
+#define SJQ_LB_THREADS 384
+#endif
+    int block = opts.block_threads ? opts.block_threads : SJQ_LB_THREADS;
     const size_t smem_cap = (size_t)dev.max_smem_optin - 1024; // static reduce scratch + slack
     const size_t stage_bytes = align_up((size_t)ns * sizeof(DStage), 16);
     auto queue_bytes = [&](int threads) { return P.nq ? (size_t)(threads / 32) * (size_t)(kQueue0Cap + (P.nq - 1) * kQueueCap) * 4 : (size_t)0; };
