@@ -31,7 +31,7 @@ CONTRACT_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per fact row of the fused kernel from the ncu capture summarised in
 # profiles/fused_kernel_c3_100m.md (a 100 M-row case of the same workload; traffic grows with the rows)
-NCU_DRAM_BYTES_PER_ROW = {"c3": 16.7}
+NCU_DRAM_BYTES_PER_ROW = {"c3": 15.6}
 
 
 def measured_hbm_peak():

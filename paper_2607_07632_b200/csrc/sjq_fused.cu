@@ -62,6 +62,25 @@ struct Vec4<int64_t> {
     }
 };
 
+// One value of a later column for one surviving row.
+#if defined(SJQ_SPARSE_PLAIN)
+__device__ __forceinline__ int32_t ld_sparse(const int32_t *p)
+{
+    int32_t v;
+    asm volatile("ld.global.b32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ int64_t ld_sparse(const int64_t *p)
+{
+    int64_t v;
+    asm volatile("ld.global.b64 %0, [%1];" : "=l"(v) : "l"(p));
+    return v;
+}
+#else
+__device__ __forceinline__ int32_t ld_sparse(const int32_t *p) { return __ldg(p); }
+__device__ __forceinline__ int64_t ld_sparse(const int64_t *p) { return __ldg(p); }
+#endif
+
 template <typename T>
 struct Index {
     typedef uint64_t type;
@@ -489,7 +508,7 @@ __device__ __forceinline__ void load_rows(const DStage &S, int64_t base, const u
 #pragma unroll
     for (int k = 0; k < kRows; ++k) {
         v[k] = 0;
-        if ((need >> k) & 1u) v[k] = __ldg(c + off[k]);
+        if ((need >> k) & 1u) v[k] = ld_sparse(c + off[k]);
     }
 }
 
