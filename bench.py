@@ -213,6 +213,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--extras", action="store_true", help="also time the other configurations (N = 1 only)")
+    ap.add_argument("--ablation", action="store_true",
+                    help="also run the A/B switches (lazy vs eager loads, queues, table forms, group-by paths)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -359,6 +361,12 @@ def main():
         del fact
         torch.cuda.empty_cache()
         extras = run_extras(sjq, W, device)
+    ablation = None
+    if args.ablation and world == 1 and rank == 0:
+        if "fact" in locals():
+            del fact
+        torch.cuda.empty_cache()
+        ablation = run_ablation(sjq, W, device)
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -375,6 +383,8 @@ def main():
                 "clocks": sampler.summary()}
         if extras is not None:
             line["other_configs"] = extras
+        if ablation is not None:
+            line["ablation"] = ablation
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -415,6 +425,60 @@ def run_extras(sjq, W, device):
     for s in (0.0001, 0.01, 0.1, 0.5, 1.0):
         for g in (1, 1000, 100000, 1000000):
             timed(W.config4(600_000_000, s, g))
+    return out
+
+
+def run_ablation(sjq, W, device):
+    """The paper's A/B experiments restated on this kernel (run-only, min of 5 after a warm-up):
+    lazy vs unconditional column loads (its tile-vs-direct table), survivor queues on/off, packed
+    direct-mapped vs open-addressing tables, privatised vs global group-by (its ablation figure)."""
+    import torch
+
+    out = []
+
+    def timed(w, label, opts=None, force_hash=False, tables=None, fact=None, dims=None):
+        if dims is None:
+            dims = {d.name: W.device_dim(w, d, device) for d in w.dims}
+        if tables is None:
+            tables = {d.name: sjq.build_dim(dims[d.name], d.key, d.preds, d.payloads,
+                                            force_kind=sjq.sjq.FORCE_HASH if (force_hash or d.force_hash) else 0)
+                      for d in w.dims}
+        if fact is None:
+            fact = W.device_fact(w, device=device)
+        res = sjq.run_workload(w, fact, tables, opts)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ts = []
+        for _ in range(5):
+            e0.record()
+            sjq.run_workload(w, fact, tables, opts, result=res)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        out.append({"workload": w.name, "variant": label, "ms_min": min(ts),
+                    "rows_per_s": w.n_rows / (min(ts) / 1000.0), "status": res.status(),
+                    "table_kinds": {k: t.layout.kind_name for k, t in tables.items()},
+                    "table_bytes": {k: int(t.layout.table_bytes) for k, t in tables.items()},
+                    "plan": res.info.describe()})
+        return fact, dims
+
+    for mk in (W.config3, W.config2):
+        w = mk()
+        fact, dims = timed(w, "default")
+        for label, opts in (("eager loads (every column for every row)", sjq.RunOpts(eager_loads=True)),
+                            ("no survivor queues (thread-owned rows throughout)", sjq.RunOpts(compaction=1)),
+                            ("one queue only", sjq.RunOpts(compaction=2)),
+                            ("global atomics group-by", sjq.RunOpts(agg_path=2)),
+                            ("shared-memory privatised group-by", sjq.RunOpts(agg_path=1)),
+                            ("every direct table in shared memory that fits", sjq.RunOpts(smem_tables=2)),
+                            ("no table in shared memory", sjq.RunOpts(smem_tables=1))):
+            try:
+                timed(w, label, opts, fact=fact, dims=dims)
+            except sjq.SjqError as e:
+                out.append({"workload": w.name, "variant": label, "error": str(e)})
+        timed(w, "open-addressing tables instead of packed direct maps", None, force_hash=True, fact=fact, dims=dims)
+        del fact, dims
+        torch.cuda.empty_cache()
     return out
 
 
