@@ -182,7 +182,7 @@ __global__ void __launch_bounds__(256) build_kernel(const __grid_constant__ Buil
                 continue;
             }
             unsigned long long *keys = static_cast<unsigned long long *>(B.slots);
-            uint64_t slot = hash64((uint64_t)k) & B.hmask;
+            uint64_t slot = (hash64((uint64_t)k) * kBucketKeys64) & B.hmask; // first slot of the home bucket
             bool done = false;
             for (uint64_t it = 0; it <= B.hmask; ++it) {
                 unsigned long long old = atomicCAS(&keys[slot], (unsigned long long)kEmptyKey64, (unsigned long long)k);
@@ -206,7 +206,7 @@ __global__ void __launch_bounds__(256) build_kernel(const __grid_constant__ Buil
                 continue;
             }
             int *keys = static_cast<int *>(B.slots);
-            uint64_t slot = hash64((uint64_t)(int64_t)k32) & B.hmask;
+            uint64_t slot = (hash64((uint64_t)(int64_t)k32) * kBucketKeys32) & B.hmask; // first slot of the home bucket
             bool done = false;
             for (uint64_t it = 0; it <= B.hmask; ++it) {
                 int old = atomicCAS(&keys[slot], kEmptyKey32, k32);

@@ -189,40 +189,73 @@ __device__ __forceinline__ uint32_t body_direct(const DStage &S, const unsigned 
     return in & hit;
 }
 
-// Open addressing, linear probing, all rows of the thread in lock step so that
-// their loads overlap; bounded by the slot count.
+// Open addressing with 32-byte buckets (4 int64 or 8 int32 keys): a key's linear probe starts at the
+// first slot of its home bucket, so a lookup loads one whole bucket per step (two 128-bit loads),
+// compares every key in it, and stops at a match or at the first bucket with a free slot.  The rows of
+// a chunk advance in lock step so that their loads overlap; bounded by the bucket count.
+__device__ __forceinline__ void load_bucket(const int64_t *p, int64_t (&k)[kBucketKeys64])
+{
+    const longlong2 a = __ldg(reinterpret_cast<const longlong2 *>(p));
+    const longlong2 b = __ldg(reinterpret_cast<const longlong2 *>(p) + 1);
+    k[0] = a.x, k[1] = a.y, k[2] = b.x, k[3] = b.y;
+}
+__device__ __forceinline__ void load_bucket(const int32_t *p, int32_t (&k)[kBucketKeys32])
+{
+    const int4 a = __ldg(reinterpret_cast<const int4 *>(p));
+    const int4 b = __ldg(reinterpret_cast<const int4 *>(p) + 1);
+    k[0] = a.x, k[1] = a.y, k[2] = a.z, k[3] = a.w, k[4] = b.x, k[5] = b.y, k[6] = b.z, k[7] = b.w;
+}
+
 template <typename T, int NR, bool WANT>
 __device__ __forceinline__ uint32_t body_hash(const DStage &S, const T (&v)[NR], uint32_t m, uint64_t (&code)[NR])
 {
+    constexpr int KPB = sizeof(T) == 4 ? kBucketKeys32 : kBucketKeys64;
+    constexpr int CH = 2; // rows advancing together
     const T empty = sizeof(T) == 4 ? (T)kEmptyKey32 : (T)kEmptyKey64;
     const T *keys = static_cast<const T *>(S.tab);
-    const uint32_t hmask = (uint32_t)S.hmask;
-    uint32_t slot[NR];
-    uint32_t pending = 0;
-#pragma unroll
-    for (int i = 0; i < NR; ++i) {
-        slot[i] = (uint32_t)hash64((uint64_t)(int64_t)v[i]) & hmask;
-        pending |= (uint32_t)(v[i] != empty) << i; // the reserved marker is never a key
-    }
-    pending &= m;
+    const uint32_t bmask = (uint32_t)(S.hmask / KPB); // buckets - 1
     uint32_t hit = 0;
-    for (uint32_t it = 0; pending != 0 && it <= hmask; ++it) {
-        T cur[NR];
+    uint32_t slot[NR];
 #pragma unroll
-        for (int i = 0; i < NR; ++i) {
-            cur[i] = empty;
-            if ((pending >> i) & 1u) cur[i] = __ldg(keys + slot[i]);
+    for (int base = 0; base < NR; base += CH) {
+        uint32_t bucket[CH];
+        uint32_t pending = 0;
+#pragma unroll
+        for (int i = 0; i < CH; ++i) {
+            bucket[i] = (uint32_t)hash64((uint64_t)(int64_t)v[base + i]) & bmask;
+            slot[base + i] = 0;
+            pending |= (uint32_t)(((m >> (base + i)) & 1u) && v[base + i] != empty) << i; // the marker is never a key
         }
+        for (uint32_t it = 0; pending != 0 && it <= bmask; ++it) {
+            T bk[CH][KPB];
 #pragma unroll
-        for (int i = 0; i < NR; ++i) {
-            if ((pending >> i) & 1u) {
-                if (cur[i] == v[i]) {
-                    hit |= 1u << i;
-                    pending &= ~(1u << i);
-                } else if (cur[i] == empty) {
-                    pending &= ~(1u << i);
-                } else {
-                    slot[i] = (slot[i] + 1) & hmask;
+            for (int i = 0; i < CH; ++i) {
+#pragma unroll
+                for (int j = 0; j < KPB; ++j) bk[i][j] = empty;
+                if ((pending >> i) & 1u) load_bucket(keys + (size_t)bucket[i] * KPB, bk[i]);
+            }
+#pragma unroll
+            for (int i = 0; i < CH; ++i) {
+                if ((pending >> i) & 1u) {
+                    bool found = false, has_free = false;
+                    uint32_t at = 0;
+#pragma unroll
+                    for (int j = 0; j < KPB; ++j) {
+                        if (bk[i][j] == v[base + i]) {
+                            found = true;
+                            at = j;
+                        }
+                        has_free |= bk[i][j] == empty;
+                    }
+                    if (found) {
+                        hit |= 1u << (base + i);
+                        slot[base + i] = bucket[i] * KPB + at;
+                        pending &= ~(1u << i);
+                    } else if (has_free) {
+                        pending &= ~(1u << i);
+                    } else {
+                        bucket[i] = (bucket[i] + 1) & bmask;
+                    }
                 }
             }
         }

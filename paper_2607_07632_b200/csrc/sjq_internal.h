@@ -28,6 +28,11 @@ bool canon_pred(const sjq_pred &p, int dtype, DPred *out);
 // ---------------------------------------------------------------- tables
 constexpr int64_t kEmptyKey64 = INT64_MIN;
 constexpr int32_t kEmptyKey32 = INT32_MIN;
+// An open-addressing table is read one 32-byte bucket at a time: a key's linear probe starts at the
+// first slot of its home bucket, so a lookup loads whole buckets and stops at the first one with a
+// free slot.
+constexpr int kBucketKeys64 = 4;
+constexpr int kBucketKeys32 = 8;
 constexpr size_t kTableHeaderBytes = 256; // device-side counters at the start of table_mem
 
 } // namespace sjq

@@ -373,8 +373,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         P.has_key = 1;
     } else {
         const size_t gb = (size_t)spec->num_groups * 8 * (P.want_count ? 2 : 1);
-        const bool fits = gb <= (size_t)64 << 10;        // what agg_path = 1 may force
-        const bool small = gb <= (size_t)32 << 10;       // auto: a larger private table costs more L1 than it saves
+        const bool fits = gb <= (size_t)64 << 10;
         bool contended = survivors / approx_grid >= 8.0 * (double)spec->num_groups;
         if (opts.agg_path == 1) {
             if (!fits) return SJQ_ERR_UNSUPPORTED;
@@ -382,7 +381,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         } else if (opts.agg_path == 2) {
             aggp = AGG_GLOBAL;
         } else {
-            aggp = (small && contended) ? AGG_SMEM : AGG_GLOBAL;
+            aggp = (fits && contended) ? AGG_SMEM : AGG_GLOBAL;
         }
         if (aggp == AGG_SMEM) group_bytes = gb;
     }
