@@ -373,7 +373,7 @@ def main():
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "int64", "data": "synthetic",
                 "config": {"workload": w.name, "rows_per_gpu": n, "referenced_bytes_per_row": ref_bytes,
-                           "step": "plan+build of every dimension table (concurrently, on side streams), then the fused pass"
+                           "step": "plan+build of every dimension table (on side streams; the key-range scans may overlap the previous step's fused pass), then the fused pass"
                                    + (", then all-reduce of the dense result" if world > 1 else ""),
                            "l2": "inputs (%.1f GB) exceed the 126 MB L2; no flush needed" % (n * ref_bytes / 1e9),
                            "parallelism": f"row-sharded x{world}, dimensions replicated", "plan": info.describe()},

@@ -292,8 +292,8 @@ class TableBuilder:
             self.layout = DimLayout()
 
     def begin(self):
-        """Enqueue the key-range scan on the side stream (after everything queued on the current stream)."""
-        self.side.wait_stream(torch.cuda.current_stream(self.device))
+        """Enqueue the key-range scan on the side stream.  It only reads the dimension columns, so it does
+        not wait for work queued on the current stream (a previous run may still be reading the old table)."""
         rc = lib().sjq_dim_plan_begin(self.carr, len(self.names), self.parr, self.npreds, self.key_col, self.pay,
                                       self.npay, self.scratch.data_ptr(), self.stats.data_ptr(),
                                       self.side.cuda_stream)
@@ -310,6 +310,8 @@ class TableBuilder:
         if self.mem is None or self.mem.numel() < self.layout.table_bytes:
             with torch.cuda.device(self.device):
                 self.mem = torch.empty(self.layout.table_bytes, dtype=torch.uint8, device=self.device)
+        # the build overwrites the table memory: it must follow whatever the current stream still runs on it
+        self.side.wait_stream(torch.cuda.current_stream(self.device))
         handle = ctypes.c_void_p()
         rc = lib().sjq_build_dim(self.carr, len(self.names), self.parr, self.npreds, self.key_col, self.pay,
                                  self.npay, ctypes.byref(self.layout), self.mem.data_ptr(), self.mem.numel(),
