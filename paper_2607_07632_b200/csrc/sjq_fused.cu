@@ -34,6 +34,9 @@
 #define SJQ_LB_THREADS 384
 #define SJQ_LB_BLOCKS 2
 #endif
+#ifndef SJQ_HASH_INLINE
+#define SJQ_HASH_INLINE __forceinline__
+#endif
 #ifndef SJQ_PREFETCH_DIST
 #define SJQ_PREFETCH_DIST 2
 #endif
@@ -207,7 +210,7 @@ __device__ __forceinline__ void load_bucket(const int32_t *p, int32_t (&k)[kBuck
 }
 
 template <typename T, int NR, bool WANT>
-__device__ __forceinline__ uint32_t body_hash(const DStage &S, const T (&v)[NR], uint32_t m, uint64_t (&code)[NR])
+__device__ SJQ_HASH_INLINE uint32_t body_hash(const DStage &S, const T (&v)[NR], uint32_t m, uint64_t (&code)[NR])
 {
     constexpr int KPB = sizeof(T) == 4 ? kBucketKeys32 : kBucketKeys64;
     constexpr int CH = 2; // rows advancing together
@@ -272,7 +275,7 @@ __device__ __forceinline__ uint32_t body_hash(const DStage &S, const T (&v)[NR],
     return hit;
 }
 
-template <typename T, int NR, bool WANT>
+template <typename T, int NR, bool WANT, bool HASH>
 __device__ __forceinline__ uint32_t run_stage(const RunParams &P, const DStage &S, const unsigned char *smem,
                                               const T (&v)[NR], uint32_t m, uint64_t (&code)[NR])
 {
@@ -290,7 +293,9 @@ __device__ __forceinline__ uint32_t run_stage(const RunParams &P, const DStage &
     case OP_DIRECT_U64 * 2: return body_direct<T, OP_DIRECT_U64, false, NR, WANT>(S, smem, v, m, code);
     case OP_DIRECT_U64 * 2 + 1: return body_direct<T, OP_DIRECT_U64, true, NR, WANT>(S, smem, v, m, code);
     case OP_HASH32 * 2:
-    case OP_HASH64 * 2: return body_hash<T, NR, WANT>(S, v, m, code);
+    case OP_HASH64 * 2:
+        if (HASH) return body_hash<T, NR, WANT>(S, v, m, code);
+        return 0; // kernels built without the hash probe are never given such a stage
     default: return m; // OP_LOAD
     }
 }
@@ -546,6 +551,7 @@ __device__ __forceinline__ void load_rows(const DStage &S, int64_t base, const u
 }
 
 // One pure filter stage on a batch: returns the mask of rows that pass.
+template <bool HASH>
 __device__ __forceinline__ uint32_t filter_rows(const RunParams &P, const DStage &S, const unsigned char *smem,
                                                 int64_t base, const uint32_t (&off)[kRows], uint32_t valid)
 {
@@ -553,17 +559,17 @@ __device__ __forceinline__ uint32_t filter_rows(const RunParams &P, const DStage
     if (S.is64) {
         int64_t v[kRows];
         load_rows<int64_t, false>(S, base, off, valid, valid, v);
-        return run_stage<int64_t, kRows, false>(P, S, smem, v, valid, unused);
+        return run_stage<int64_t, kRows, false, HASH>(P, S, smem, v, valid, unused);
     }
     int32_t v[kRows];
     load_rows<int32_t, false>(S, base, off, valid, valid, v);
-    return run_stage<int32_t, kRows, false>(P, S, smem, v, valid, unused);
+    return run_stage<int32_t, kRows, false, HASH>(P, S, smem, v, valid, unused);
 }
 
 // Stages [first, nstages) with accumulators, then the terminal.  The column of
 // the next stage is requested before the current stage's probe is resolved, so
 // a stage costs one memory latency, not two.
-template <int AGG, bool MUL, bool CONTIG>
+template <int AGG, bool MUL, bool CONTIG, bool HASH>
 __device__ __forceinline__ void final_rows(const RunParams &P, const DStage *st, unsigned char *smem, int first,
                                            int64_t base, const uint32_t (&off)[kRows], uint32_t valid, int64_t &lsum,
                                            int64_t &lcnt)
@@ -589,7 +595,7 @@ __device__ __forceinline__ void final_rows(const RunParams &P, const DStage *st,
             int64_t v[kRows];
             load_rows<int64_t, CONTIG>(S, base, off, valid, need, v);
             have_next = false;
-            m = run_stage<int64_t, kRows, true>(P, S, smem, v, m, code);
+            m = run_stage<int64_t, kRows, true, HASH>(P, S, smem, v, m, code);
             if (S.acc) accumulate<MUL, int64_t, kRows>(S, v, code, m, key, X, Y);
         } else {
             int32_t v[kRows];
@@ -601,7 +607,7 @@ __device__ __forceinline__ void final_rows(const RunParams &P, const DStage *st,
             }
             have_next = (s + 1 < P.nstages) && !st[s + 1].is64;
             if (have_next) load_rows<int32_t, CONTIG>(st[s + 1], base, off, valid, need, vnext);
-            m = run_stage<int32_t, kRows, true>(P, S, smem, v, m, code);
+            m = run_stage<int32_t, kRows, true, HASH>(P, S, smem, v, m, code);
             if (S.acc) accumulate<MUL, int32_t, kRows>(S, v, code, m, key, X, Y);
         }
     }
@@ -612,7 +618,7 @@ __device__ __forceinline__ void final_rows(const RunParams &P, const DStage *st,
 // One filter stage on the thread's own kSlots groups of four consecutive rows
 // of a tile: the column is loaded for a group only while one of its rows is
 // alive.  FULL: the whole tile lies inside the table (no bounds masks).
-template <typename T, bool FULL>
+template <typename T, bool FULL, bool HASH>
 __device__ __forceinline__ uint32_t dense_stage(const RunParams &P, const DStage &S, const unsigned char *smem,
                                                 int64_t row0, int32_t slot_stride, uint32_t valid, uint32_t alive)
 {
@@ -634,10 +640,10 @@ __device__ __forceinline__ uint32_t dense_stage(const RunParams &P, const DStage
         }
     }
     uint64_t unused[kDenseRows];
-    return run_stage<T, kDenseRows, false>(P, S, smem, v, alive, unused);
+    return run_stage<T, kDenseRows, false, HASH>(P, S, smem, v, alive, unused);
 }
 
-template <bool FULL>
+template <bool FULL, bool HASH>
 __device__ __forceinline__ uint32_t level0(const RunParams &P, const DStage *st, const unsigned char *smem,
                                            int64_t row0, int32_t slot_stride, uint32_t valid)
 {
@@ -645,8 +651,8 @@ __device__ __forceinline__ uint32_t level0(const RunParams &P, const DStage *st,
     for (int s = 0; s < P.nd0; ++s) {
         if (!alive) break;
         const DStage &S = st[s];
-        alive = S.is64 ? dense_stage<int64_t, FULL>(P, S, smem, row0, slot_stride, valid, alive)
-                       : dense_stage<int32_t, FULL>(P, S, smem, row0, slot_stride, valid, alive);
+        alive = S.is64 ? dense_stage<int64_t, FULL, HASH>(P, S, smem, row0, slot_stride, valid, alive)
+                       : dense_stage<int32_t, FULL, HASH>(P, S, smem, row0, slot_stride, valid, alive);
     }
     return alive;
 }
@@ -681,7 +687,7 @@ __device__ __forceinline__ uint32_t queue_base(int l)
     return l == 0 ? 0u : (uint32_t)(kQueue0Cap + (l - 1) * kQueueCap);
 }
 
-template <int AGG, bool MUL>
+template <int AGG, bool MUL, bool HASH>
 __global__ void __launch_bounds__(SJQ_LB_THREADS, SJQ_LB_BLOCKS) fused_kernel(const __grid_constant__ RunParams P)
 {
     extern __shared__ __align__(16) unsigned char smem[];
@@ -725,7 +731,7 @@ __global__ void __launch_bounds__(SJQ_LB_THREADS, SJQ_LB_BLOCKS) fused_kernel(co
             const int64_t base = tile * tile_rows;
             const int64_t rem = P.n - base - 4 * (int64_t)tid;
             const uint32_t valid = rem >= 4 ? 0xFu : (rem > 0 ? ((1u << (int)rem) - 1u) : 0u);
-            final_rows<AGG, MUL, true>(P, st, smem, 0, base, off, valid, lsum, lcnt);
+            final_rows<AGG, MUL, true, HASH>(P, st, smem, 0, base, off, valid, lsum, lcnt);
         }
     } else {
         const int nq = P.nq;
@@ -777,7 +783,7 @@ __global__ void __launch_bounds__(SJQ_LB_THREADS, SJQ_LB_BLOCKS) fused_kernel(co
 #endif
                     uint32_t alive;
                     if (tile_base + tile_rows <= P.n) {
-                        alive = level0<true>(P, st, smem, row0, slot_stride, kDenseRows >= 32 ? 0xFFFFFFFFu : ((1u << kDenseRows) - 1u));
+                        alive = level0<true, HASH>(P, st, smem, row0, slot_stride, kDenseRows >= 32 ? 0xFFFFFFFFu : ((1u << kDenseRows) - 1u));
                     } else {
                         uint32_t valid = 0;
 #pragma unroll
@@ -786,7 +792,7 @@ __global__ void __launch_bounds__(SJQ_LB_THREADS, SJQ_LB_BLOCKS) fused_kernel(co
                             const uint32_t nv = rem >= 4 ? 0xFu : (rem > 0 ? ((1u << (int)rem) - 1u) : 0u);
                             valid |= nv << (4 * k);
                         }
-                        alive = level0<false>(P, st, smem, row0, slot_stride, valid);
+                        alive = level0<false, HASH>(P, st, smem, row0, slot_stride, valid);
                     }
 #if defined(SJQ_EXP_NO_QUEUE)
                     lcnt += __popc(alive);
@@ -845,9 +851,9 @@ __global__ void __launch_bounds__(SJQ_LB_THREADS, SJQ_LB_BLOCKS) fused_kernel(co
                 Q.set_count(l, Q.count(l) - nb);
             }
             if (l + 1 == nq) {
-                final_rows<AGG, MUL, false>(P, st, smem, P.nd0 + l, qbase, off, valid, lsum, lcnt);
+                final_rows<AGG, MUL, false, HASH>(P, st, smem, P.nd0 + l, qbase, off, valid, lsum, lcnt);
             } else {
-                const uint32_t m = filter_rows(P, st[P.nd0 + l], smem, qbase, off, valid);
+                const uint32_t m = filter_rows<HASH>(P, st[P.nd0 + l], smem, qbase, off, valid);
                 const uint32_t mine = (uint32_t)__popc(m);
                 uint32_t incl = mine;
 #pragma unroll
@@ -967,17 +973,25 @@ __global__ void __launch_bounds__(256) compact_kernel(const CompactParams C)
 
 typedef void (*fused_fn)(const RunParams);
 
-fused_fn pick_kernel(int agg, bool mul)
+fused_fn pick_kernel(int agg, bool mul, bool hash)
 {
-    switch (agg * 2 + (mul ? 1 : 0)) {
-    case 0: return fused_kernel<AGG_SCALAR, false>;
-    case 1: return fused_kernel<AGG_SCALAR, true>;
-    case 2: return fused_kernel<AGG_SMEM, false>;
-    case 3: return fused_kernel<AGG_SMEM, true>;
-    case 4: return fused_kernel<AGG_GLOBAL, false>;
-    case 5: return fused_kernel<AGG_GLOBAL, true>;
-    case 6: return fused_kernel<AGG_HASH, false>;
-    default: return fused_kernel<AGG_HASH, true>;
+    switch (agg * 4 + (mul ? 2 : 0) + (hash ? 1 : 0)) {
+    case 0: return fused_kernel<AGG_SCALAR, false, false>;
+    case 1: return fused_kernel<AGG_SCALAR, false, true>;
+    case 2: return fused_kernel<AGG_SCALAR, true, false>;
+    case 3: return fused_kernel<AGG_SCALAR, true, true>;
+    case 4: return fused_kernel<AGG_SMEM, false, false>;
+    case 5: return fused_kernel<AGG_SMEM, false, true>;
+    case 6: return fused_kernel<AGG_SMEM, true, false>;
+    case 7: return fused_kernel<AGG_SMEM, true, true>;
+    case 8: return fused_kernel<AGG_GLOBAL, false, false>;
+    case 9: return fused_kernel<AGG_GLOBAL, false, true>;
+    case 10: return fused_kernel<AGG_GLOBAL, true, false>;
+    case 11: return fused_kernel<AGG_GLOBAL, true, true>;
+    case 12: return fused_kernel<AGG_HASH, false, false>;
+    case 13: return fused_kernel<AGG_HASH, false, true>;
+    case 14: return fused_kernel<AGG_HASH, true, false>;
+    default: return fused_kernel<AGG_HASH, true, true>;
     }
 }
 
@@ -985,9 +999,9 @@ fused_fn pick_kernel(int agg, bool mul)
 
 // ---- launch helpers used by the planner (sjq_run.cu) ----------------------
 
-sjq_status fused_occupancy(int agg, bool mul, int block, size_t smem, int *ctas_per_sm)
+sjq_status fused_occupancy(int agg, bool mul, bool hash, int block, size_t smem, int *ctas_per_sm)
 {
-    fused_fn fn = pick_kernel(agg, mul);
+    fused_fn fn = pick_kernel(agg, mul, hash);
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, fn, block, smem) != cudaSuccess) {
         (void)cudaGetLastError();
@@ -996,9 +1010,10 @@ sjq_status fused_occupancy(int agg, bool mul, int block, size_t smem, int *ctas_
     return SJQ_OK;
 }
 
-sjq_status fused_launch(int agg, bool mul, int grid, int block, size_t smem, const RunParams &P, cudaStream_t stream)
+sjq_status fused_launch(int agg, bool mul, bool hash, int grid, int block, size_t smem, const RunParams &P,
+                        cudaStream_t stream)
 {
-    fused_fn fn = pick_kernel(agg, mul);
+    fused_fn fn = pick_kernel(agg, mul, hash);
     fn<<<grid, block, smem, stream>>>(P);
     if (cudaGetLastError() != cudaSuccess) return SJQ_ERR_CUDA;
     return SJQ_OK;

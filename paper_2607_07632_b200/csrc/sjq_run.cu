@@ -23,8 +23,9 @@
 
 namespace sjq {
 
-sjq_status fused_occupancy(int agg, bool mul, int block, size_t smem, int *ctas_per_sm);
-sjq_status fused_launch(int agg, bool mul, int grid, int block, size_t smem, const RunParams &P, cudaStream_t stream);
+sjq_status fused_occupancy(int agg, bool mul, bool hash, int block, size_t smem, int *ctas_per_sm);
+sjq_status fused_launch(int agg, bool mul, bool hash, int grid, int block, size_t smem, const RunParams &P,
+                        cudaStream_t stream);
 sjq_status clear_launch(int64_t *sums, int64_t *counts, int64_t cells, int64_t *gkeys, int64_t gslots,
                         int64_t *n_groups, int32_t *status, int sm_count, cudaStream_t stream);
 sjq_status compact_launch(const int64_t *gkeys, const int64_t *gsums, const int64_t *gcounts, int64_t gslots,
@@ -452,9 +453,12 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     P.smem_queue = (uint32_t)(stage_bytes + tables + group_bytes);
     size_t smem = stage_bytes + tables + group_bytes + queue_bytes(block);
 
+    bool has_hash = false; // kernels without the hash probe are leaner; pick by what the stages need
+    for (int s2 = 0; s2 < ns; ++s2) has_hash |= P.st[s2].op == OP_HASH32 || P.st[s2].op == OP_HASH64;
+
     // ------------------------------------------------------------ launch shape
     int per_sm = 0;
-    if ((st = fused_occupancy(aggp, mul, block, smem, &per_sm)) != SJQ_OK) return st;
+    if ((st = fused_occupancy(aggp, mul, has_hash, block, smem, &per_sm)) != SJQ_OK) return st;
     if (per_sm < 1) return SJQ_ERR_UNSUPPORTED;
     if (opts.ctas_per_sm > 0) per_sm = std::min(per_sm, opts.ctas_per_sm);
     const int64_t tile_rows = (int64_t)block * (P.nq ? kDenseRows : kRows);
@@ -478,7 +482,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     if (opts.event_before && cudaEventRecord((cudaEvent_t)opts.event_before, stream) != cudaSuccess)
         return SJQ_ERR_CUDA;
     if (n > 0) {
-        if ((st = fused_launch(aggp, mul, grid, block, smem, P, stream)) != SJQ_OK) return st;
+        if ((st = fused_launch(aggp, mul, has_hash, grid, block, smem, P, stream)) != SJQ_OK) return st;
         ++launches;
     }
     if (opts.event_after && cudaEventRecord((cudaEvent_t)opts.event_after, stream) != cudaSuccess)
