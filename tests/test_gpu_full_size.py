@@ -69,3 +69,35 @@ def test_full_size_config(name):
 @pytest.mark.parametrize("groups", W.C4_GROUPS)
 def test_full_size_sweep_point(sel, groups):
     _check(W.config4(600_000_000, sel, groups), f"c4_s{sel:g}_g{groups}")
+
+
+def test_more_than_2_pow_32_rows_equals_split_runs():
+    """Maximum-size edge: beyond 2^32 rows the survivor queues switch to tile-relative offsets and are
+    drained per tile.  The oracle cannot hold such a table, so the check is the split-and-add property
+    (pinned for the oracle on the CPU): one run over all rows must equal two accumulated runs over
+    halves that each stay below 2^32 rows, and the count must equal the closed form of the generator."""
+    import paper_2607_07632_b200 as sjq
+    from datagen import UNIFORM_I32, fill_device
+    from datagen.workloads import AggExpr, KeyExpr, Pred, Term
+
+    n = (1 << 32) + 4099
+    free, _ = torch.cuda.mem_get_info()
+    if free < n * 4 + (2 << 30):
+        pytest.skip("not enough device memory for a 17 GB column")
+    p = fill_device(UNIFORM_I32, 20260707, 901, 0, n, 0, 9999)
+    fact = {"p": p}
+    half = 1 << 31
+    parts = ({"p": p[:half]}, {"p": p[half:]})
+    for kw in (dict(mode="SCALAR", key=None),
+               dict(mode="DENSE", key=KeyExpr((Term("FACT", "p"),), modulo=7), num_groups=7)):
+        agg = AggExpr("COL", Term("FACT", "p"))
+        preds = (Pred("p", "LT", 2500),)
+        whole = sjq.run(fact, preds, (), agg=agg, **kw)
+        acc = sjq.run(parts[0], preds, (), agg=agg, **kw)
+        acc = sjq.run(parts[1], preds, (), agg=agg, opts=sjq.RunOpts(accumulate=True), result=acc, **kw)
+        torch.cuda.synchronize()
+        assert whole.status() == 0 and acc.status() == 0
+        assert torch.equal(whole.sums, acc.sums) and torch.equal(whole.counts, acc.counts)
+        assert int(whole.counts.sum().item()) == int((p < 2500).sum().item())
+    del p, fact, parts
+    torch.cuda.empty_cache()
