@@ -799,6 +799,11 @@ __global__ void __launch_bounds__(SJQ_LB_THREADS, SJQ_LB_BLOCKS) fused_kernel(co
                     tile += gridDim.x;
                     continue;
 #endif
+                    if (!__any_sync(0xffffffffu, alive != 0)) { // a very selective first stage: nothing to push
+                        tile += gridDim.x;
+                        if (wide) flushing = true;
+                        continue;
+                    }
                     // compact the warp's survivors into queue 0
                     const uint32_t mine = (uint32_t)__popc(alive);
                     uint32_t incl = mine;
