@@ -29,8 +29,8 @@ METRIC = "fact_rows_per_s"
 UNIT = "rows/s"
 CONTRACT_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes per fact row of the fused kernel from the ncu capture summarised in
-# profiles/fused_kernel_c3_100m.md (a 100 M-row case of the same workload; traffic grows with the rows)
+# DRAM bytes per fact row of the fused kernel, from an ncu capture of a 100 M-row case of the same workload
+# (dram__bytes_read.sum + dram__bytes_write.sum; traffic grows in proportion to the rows)
 NCU_DRAM_BYTES_PER_ROW = {"c3": 15.6}
 
 
@@ -171,8 +171,8 @@ def run_reference(args):
     dims = oracle.build_dims(w, hd)
     t = oracle.run(w, fact, dims)["seconds"]
     per_row = max(t / probe, 1e-9)
-    budget_s = 90.0
-    sample = int(min(w.n_rows, max(100_000, budget_s / per_row / (args.steps + args.warmup))))
+    wall_s = 90.0  # total CPU time the reference arm may take
+    sample = int(min(w.n_rows, max(100_000, wall_s / per_row / (args.steps + args.warmup))))
     times = []
     for i in range(args.warmup + args.steps):
         row0 = (i * sample) % max(1, w.n_rows - sample + 1)
