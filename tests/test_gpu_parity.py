@@ -265,3 +265,33 @@ def test_prepared_builders_rebuild_identical_tables():
     for k in tabs:
         assert tabs[k].layout.entries == tables[k].layout.entries and tabs[k].layout.kind == tables[k].layout.kind
     compare(w, r, exp)
+
+
+def test_open_addressing_tables_give_the_same_result():
+    for w in (W.config3(1_200_007), W.config2(900_001)):
+        fact = W.host_fact(w)
+        hd = {d.name: W.host_dim(w, d) for d in w.dims}
+        dev = {k: to_dev(v) for k, v in hd.items()}
+        tables = {d.name: sjq.build_dim(dev[d.name], d.key, d.preds, d.payloads, force_kind=sjq.sjq.FORCE_HASH)
+                  for d in w.dims}
+        assert all(t.layout.kind_name.startswith("HASH") and t.status() == 0 for t in tables.values())
+        res, exp, _ = run_both(w, fact, hd, tables=tables)
+        assert res.status() == 0
+        compare(w, res, exp)
+        for opts in (sjq.RunOpts(compaction=1), sjq.RunOpts(compaction=2), sjq.RunOpts(eager_loads=True)):
+            res, _, _ = run_both(w, fact, hd, opts=opts, tables=tables)
+            compare(w, res, exp)
+
+
+def test_stale_layout_is_reported_not_followed():
+    # plan on one key range, then the data changes before the build: the build must flag it, never write outside
+    cols = {"k": torch.arange(1, 1001, dtype=torch.int32, device="cuda"),
+            "p": torch.arange(0, 1000, dtype=torch.int32, device="cuda") % 50}
+    b = sjq.TableBuilder(cols, "k", (), ("p",))
+    b.begin()
+    b.side.synchronize()
+    cols["k"][7] = 5_000_000       # far outside the planned span
+    cols["p"][9] = 100_000         # outside the planned payload range
+    t = b.finish()
+    torch.cuda.synchronize()
+    assert t.status() == 21
