@@ -588,6 +588,23 @@ __device__ __forceinline__ void final_rows(const RunParams &P, const DStage *st,
         const DStage &S = st[s];
         const uint32_t need = P.eager ? valid : m;
         if (!need) break;
+        const uint32_t simple = S.simple;
+        if (simple) { // a plain int32 column feeding one accumulator: no probe, no recipe to interpret
+            int32_t v[kRows];
+            if (have_next) {
+#pragma unroll
+                for (int k = 0; k < kRows; ++k) v[k] = vnext[k];
+            } else {
+                load_rows<int32_t, CONTIG>(S, base, off, valid, need, v);
+            }
+            have_next = (s + 1 < P.nstages) && !st[s + 1].is64;
+            if (have_next) load_rows<int32_t, CONTIG>(st[s + 1], base, off, valid, need, vnext);
+            const int32_t mult = S.mult32[simple - 1];
+            if (simple == 2) add_scaled32<kRows>(X, mult, v, m);
+            else if (simple == 1) add_scaled32<kRows>(key, mult, v, m);
+            else if (MUL) add_scaled32<kRows>(Y, mult, v, m);
+            continue;
+        }
         uint64_t code[kRows];
 #pragma unroll
         for (int k = 0; k < kRows; ++k) code[k] = 0;

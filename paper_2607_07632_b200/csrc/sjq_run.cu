@@ -357,6 +357,9 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
             }
         }
         S.acc32 = ok ? 1 : 0;
+        S.simple = 0;
+        if (ok && S.op == OP_LOAD && (S.acc == 1u || S.acc == 2u || S.acc == 4u))
+            S.simple = (uint8_t)(1 + (S.acc == 1u ? 0 : S.acc == 2u ? 1 : 2));
     }
     P.nstages = ns;
     P.eager = opts.eager_loads ? 1 : 0;

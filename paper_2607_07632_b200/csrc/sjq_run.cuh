@@ -66,6 +66,8 @@ struct DStage {
     uint32_t tab_bytes; // bytes to stage
     uint16_t acc;
     uint8_t op, is64, neg, never, nset, set_idx, pbits0, code_bits, in_smem, kind;
+    uint8_t simple; // 1 + destination (0 key, 1 X, 2 Y): plain int32 load feeding one accumulator through mult32
+    uint8_t pad[7];
 };
 
 struct RunParams {
