@@ -147,6 +147,8 @@ typedef struct sjq_dim_layout {
     int64_t pay_max[SJQ_MAX_PAYLOADS];
     int32_t pay_bits[SJQ_MAX_PAYLOADS];
     int64_t slots;      /* direct: kmax-kmin+1; hash: power-of-two slot count */
+    int64_t filter_bits; /* hash: size (power of two, 0 = none) of the presence bitmap indexed by the key's hash,
+                            probed before the table so that most absent keys never touch it */
     size_t table_bytes; /* device bytes sjq_build_dim needs at table_mem */
 } sjq_dim_layout;
 

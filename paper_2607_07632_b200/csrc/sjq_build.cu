@@ -117,6 +117,8 @@ struct BuildParams {
     int32_t pay_bits[SJQ_MAX_PAYLOADS];
     void *slots;
     void *codes;
+    unsigned int *filter; // hash: presence bitmap words
+    uint32_t fmask;       // hash: filter bits - 1
     unsigned long long *header; // [0] rows inserted, [1] slots occupied
     int32_t *status;
 };
@@ -182,6 +184,10 @@ __global__ void __launch_bounds__(256) build_kernel(const __grid_constant__ Buil
                 continue;
             }
             unsigned long long *keys = static_cast<unsigned long long *>(B.slots);
+            if (B.filter) {
+                const uint32_t fb = filter_hash((uint64_t)k) & B.fmask;
+                atomicOr(B.filter + (fb >> 5), 1u << (fb & 31));
+            }
             uint64_t slot = (hash64((uint64_t)k) * kBucketKeys64) & B.hmask; // first slot of the home bucket
             bool done = false;
             for (uint64_t it = 0; it <= B.hmask; ++it) {
@@ -206,6 +212,10 @@ __global__ void __launch_bounds__(256) build_kernel(const __grid_constant__ Buil
                 continue;
             }
             int *keys = static_cast<int *>(B.slots);
+            if (B.filter) {
+                const uint32_t fb = filter_hash((uint64_t)(int64_t)k32) & B.fmask;
+                atomicOr(B.filter + (fb >> 5), 1u << (fb & 31));
+            }
             uint64_t slot = (hash64((uint64_t)(int64_t)k32) * kBucketKeys32) & B.hmask; // first slot of the home bucket
             bool done = false;
             for (uint64_t it = 0; it <= B.hmask; ++it) {
@@ -501,7 +511,11 @@ extern "C" sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_c
         L.code_bits = npayload == 0 ? 0 : (code_bits <= 32 ? 32 : 64);
         const size_t kb = (size_t)slots * (L.key_dtype == SJQ_I64 ? 8 : 4);
         const size_t cb = (size_t)slots * (size_t)(L.code_bits / 8);
-        L.table_bytes = kTableHeaderBytes + align_up(kb, 256) + align_up(cb, 256);
+        // presence bitmap: 16 bits per entry (about 6 % false positives), at least 1024 bits, at most 2^32
+        uint64_t fbits = 1024;
+        while (fbits < (uint64_t)L.entries * 16 && fbits < ((uint64_t)1 << 32)) fbits <<= 1;
+        L.filter_bits = (int64_t)fbits;
+        L.table_bytes = kTableHeaderBytes + align_up(kb, 256) + align_up(cb, 256) + align_up((size_t)(fbits / 8), 256);
     }
     *layout = L;
     return SJQ_OK;
@@ -518,6 +532,8 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
     sjq_status st = fill_dim_params(cols, ncols, preds, npreds, key_col, payload_cols, npayload, &B.dim);
     if (st != SJQ_OK) return st;
     const sjq_dim_layout &L = *layout;
+    if (L.filter_bits < 0 || (L.filter_bits & (L.filter_bits - 1)) || L.filter_bits > ((int64_t)1 << 32))
+        return SJQ_ERR_INVALID_ARG;
     if (L.kind < SJQ_TABLE_DIRECT_BITMAP || L.kind > SJQ_TABLE_HASH_I64 || L.npayload != npayload ||
         L.key_dtype != cols[key_col].dtype || L.slots <= 0 || L.dim_rows != B.dim.n)
         return SJQ_ERR_INVALID_ARG;
@@ -532,6 +548,7 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
     T->base = static_cast<char *>(table_mem);
     T->slots = T->base + kTableHeaderBytes;
     T->codes = nullptr;
+    T->filter = nullptr;
     T->magic = kTableMagic;
 
     B.kind = L.kind;
@@ -560,8 +577,15 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
     } else {
         const size_t kb = (size_t)L.slots * (L.key_dtype == SJQ_I64 ? 8 : 4);
         T->slots_bytes = kb;
+        const size_t cb = (size_t)L.slots * (size_t)(L.code_bits / 8);
         if (L.code_bits) T->codes = T->slots + align_up(kb, 256);
         B.codes = T->codes;
+        if (L.filter_bits) {
+            T->filter = T->slots + align_up(kb, 256) + align_up(cb, 256);
+            B.filter = reinterpret_cast<unsigned int *>(T->filter);
+            B.fmask = (uint32_t)(L.filter_bits - 1);
+            ok = ok && cudaMemsetAsync(T->filter, 0, (size_t)(L.filter_bits / 8), stream) == cudaSuccess;
+        }
         const int g = grid_for(L.slots, dev.sm_count);
         if (L.key_dtype == SJQ_I64)
             fill_kernel<int64_t><<<g, 256, 0, stream>>>(reinterpret_cast<int64_t *>(T->slots), kEmptyKey64, (size_t)L.slots);

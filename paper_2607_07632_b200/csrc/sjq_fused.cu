@@ -213,7 +213,10 @@ template <typename T, int NR, bool WANT>
 __device__ SJQ_HASH_INLINE uint32_t body_hash(const DStage &S, const T (&v)[NR], uint32_t m, uint64_t (&code)[NR])
 {
     constexpr int KPB = sizeof(T) == 4 ? kBucketKeys32 : kBucketKeys64;
-    constexpr int CH = 2; // rows advancing together
+#ifndef SJQ_HASH_CH
+#define SJQ_HASH_CH 2
+#endif
+    constexpr int CH = NR < SJQ_HASH_CH ? NR : SJQ_HASH_CH; // rows advancing together
     const T empty = sizeof(T) == 4 ? (T)kEmptyKey32 : (T)kEmptyKey64;
     const T *keys = static_cast<const T *>(S.tab);
     const uint32_t bmask = (uint32_t)(S.hmask / KPB); // buckets - 1
@@ -275,6 +278,26 @@ __device__ SJQ_HASH_INLINE uint32_t body_hash(const DStage &S, const T (&v)[NR],
     return hit;
 }
 
+// Presence bitmap of an open-addressing table: one bit per hash value; a clear bit proves the key
+// absent, a set bit sends the row on to the exact probe.
+template <typename T, int NR>
+__device__ __forceinline__ uint32_t body_hashbits(const DStage &S, const T (&v)[NR], uint32_t m)
+{
+    const uint32_t *bits = static_cast<const uint32_t *>(S.tab);
+    const uint32_t fmask = (uint32_t)S.hmask;
+    uint32_t w[NR], idx[NR];
+#pragma unroll
+    for (int i = 0; i < NR; ++i) {
+        idx[i] = filter_hash((uint64_t)(int64_t)v[i]) & fmask;
+        w[i] = 0;
+        if ((m >> i) & 1u) w[i] = __ldg(bits + (idx[i] >> 5));
+    }
+    uint32_t hit = 0;
+#pragma unroll
+    for (int i = 0; i < NR; ++i) hit |= ((w[i] >> (idx[i] & 31)) & 1u) << i;
+    return m & hit;
+}
+
 template <typename T, int NR, bool WANT, bool HASH>
 __device__ __forceinline__ uint32_t run_stage(const RunParams &P, const DStage &S, const unsigned char *smem,
                                               const T (&v)[NR], uint32_t m, uint64_t (&code)[NR])
@@ -292,6 +315,7 @@ __device__ __forceinline__ uint32_t run_stage(const RunParams &P, const DStage &
     case OP_DIRECT_U32 * 2 + 1: return body_direct<T, OP_DIRECT_U32, true, NR, WANT>(S, smem, v, m, code);
     case OP_DIRECT_U64 * 2: return body_direct<T, OP_DIRECT_U64, false, NR, WANT>(S, smem, v, m, code);
     case OP_DIRECT_U64 * 2 + 1: return body_direct<T, OP_DIRECT_U64, true, NR, WANT>(S, smem, v, m, code);
+    case OP_HASHBITS * 2: return body_hashbits<T, NR>(S, v, m);
     case OP_HASH32 * 2:
     case OP_HASH64 * 2:
         if (HASH) return body_hash<T, NR, WANT>(S, v, m, code);

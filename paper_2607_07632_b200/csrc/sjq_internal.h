@@ -42,6 +42,7 @@ struct sjq_table {
     char *base;          // table_mem
     char *slots;         // direct: code array / bitmap words; hash: key array
     char *codes;         // hash: code array (NULL when no payload)
+    char *filter;        // hash: presence bitmap (NULL when none)
     size_t slots_bytes;  // bytes of the direct array (for shared-memory staging)
     uint32_t magic;
 };
@@ -60,6 +61,14 @@ __host__ __device__ inline uint64_t hash64(uint64_t k)
     k ^= k >> 32;
     k *= 0x9E3779B97F4A7C15ULL;
     return k >> 32;
+}
+
+// A second, independent hash for the presence bitmap in front of an open-addressing table.
+__host__ __device__ inline uint32_t filter_hash(uint64_t k)
+{
+    k ^= k >> 29;
+    k *= 0xD6E8FEB86659FD93ULL;
+    return (uint32_t)(k >> 32);
 }
 
 // first-error-wins store into the status word

@@ -40,6 +40,7 @@ struct StageSpec {
     int col;      // fact column
     double sel;   // estimated fraction of rows passing
     double cost;  // relative cost per row evaluated
+    int prefilter; // 1: only the presence bitmap of a hashed join; 2: the exact probe that follows one
 };
 
 double pred_selectivity(const sjq_pred &p)
@@ -147,7 +148,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     std::vector<StageSpec> specs;
     for (int p = 0; p < npreds; ++p) {
         const double bytes = fact[preds[p].col].dtype == SJQ_I64 ? 2.0 : 1.0;
-        specs.push_back({ST_PRED, p, preds[p].col, pred_selectivity(preds[p]), bytes});
+        specs.push_back({ST_PRED, p, preds[p].col, pred_selectivity(preds[p]), bytes, 0});
     }
     for (int j = 0; j < njoins; ++j) {
         const sjq_table *T = joins[j].table;
@@ -156,21 +157,39 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         double sel = L.dim_rows > 0 ? (double)L.entries / (double)L.dim_rows : 0.0;
         const size_t tb = L.table_bytes;
         double probe = tb <= (size_t)200 << 10 ? 0.3 : tb <= (size_t)32 << 20 ? 1.5 : 4.0;
-        specs.push_back({ST_PROBE, j, joins[j].fk_col, std::min(1.0, sel), bytes + probe});
+        if (L.kind >= SJQ_TABLE_HASH_I32 && T->filter && L.filter_bits > 0) {
+            // a hashed join is two stages: its presence bitmap (cheap, passes the hits and ~1/16 of the
+            // misses) early, the exact probe (expensive) on what is left
+            const double fp = std::min(1.0, (double)L.entries / (double)L.filter_bits);
+            const double pass = std::min(1.0, sel + (1.0 - sel) * fp);
+            specs.push_back({ST_PROBE, j, joins[j].fk_col, pass, bytes + 0.7, 1});
+            specs.push_back({ST_PROBE, j, joins[j].fk_col, pass > 0 ? std::min(1.0, sel / pass) : 1.0,
+                             bytes + probe + 4.0, 2});
+            continue;
+        }
+        specs.push_back({ST_PROBE, j, joins[j].fk_col, std::min(1.0, sel), bytes + probe, 0});
     }
     const int nfilter = (int)specs.size();
-    std::vector<int> order(nfilter);
+    std::vector<int> order;
     if (opts.norder) {
-        std::vector<char> seen(nfilter, 0);
-        for (int i = 0; i < nfilter; ++i) {
+        // the caller orders predicates and joins; a hashed join's bitmap and exact probe stay adjacent
+        std::vector<char> seen(npreds + njoins, 0);
+        for (int i = 0; i < npreds + njoins; ++i) {
             const int o = opts.order[i];
-            if (o < 0 || o >= nfilter || seen[o]) return SJQ_ERR_INVALID_ARG;
+            if (o < 0 || o >= npreds + njoins || seen[o]) return SJQ_ERR_INVALID_ARG;
             seen[o] = 1;
-            order[i] = o;
+            for (int k = 0; k < nfilter; ++k) {
+                const bool match = o < npreds ? (specs[k].kind == ST_PRED && specs[k].index == o)
+                                              : (specs[k].kind == ST_PROBE && specs[k].index == o - npreds);
+                if (match) order.push_back(k);
+            }
         }
     } else {
+        order.resize(nfilter);
         for (int i = 0; i < nfilter; ++i) order[i] = i;
         std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+            // exact probes of prefiltered hashed joins go last: they run at the final level
+            if ((specs[a].prefilter == 2) != (specs[b].prefilter == 2)) return specs[b].prefilter == 2;
             return (1.0 - specs[a].sel) / specs[a].cost > (1.0 - specs[b].sel) / specs[b].cost;
         });
     }
@@ -235,11 +254,16 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
                                                                : OP_HASH64);
             S.tab = T->slots;
             S.codes = T->codes;
+            if (sp.prefilter == 1) {
+                S.op = OP_HASHBITS;
+                S.tab = T->filter;
+                S.codes = nullptr;
+            }
             S.kmin = L.kmin;
             S.last = (uint64_t)L.slots - 1;
             S.kmin32 = (int32_t)L.kmin;
             S.last32 = (uint32_t)std::min<uint64_t>((uint64_t)L.slots - 1, 0xFFFFFFFFull);
-            S.hmask = (uint64_t)L.slots - 1;
+            S.hmask = sp.prefilter == 1 ? (uint64_t)L.filter_bits - 1 : (uint64_t)L.slots - 1;
             S.pmin0 = L.pay_min[0];
             S.pmin1 = L.pay_min[1];
             S.pbits0 = (uint8_t)L.pay_bits[0];
@@ -251,10 +275,11 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     };
     for (int i = 0; i < nfilter; ++i) {
         const StageSpec &sp = specs[order[i]];
+        if (ns >= kMaxStages) return SJQ_ERR_UNSUPPORTED;
         if ((st = fill_stage(P.st[ns], sp)) != SJQ_OK) return st;
-        if (sp.kind == ST_PROBE) stage_of_join[sp.index] = ns;
+        if (sp.kind == ST_PROBE && sp.prefilter != 1) stage_of_join[sp.index] = ns;
         if (stage_of_col[sp.col] < 0) stage_of_col[sp.col] = ns;
-        stage_label.push_back(order[i]);
+        stage_label.push_back(sp.kind == ST_PRED ? sp.index : npreds + sp.index);
         ++ns;
     }
     P.want_count = agg->want_count ? 1 : 0;
@@ -282,9 +307,11 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         nd0 = 1;
         if (opts.compaction != 2) {
             const double dense_reach = opts.reserved[0] > 0 ? opts.reserved[0] / 1000.0 : 0.06;
-            while (nd0 < nfilter && specs[order[nd0]].sel < 0.9 && reach[nd0] > dense_reach) ++nd0;
+            while (nd0 < nfilter && specs[order[nd0]].sel < 0.9 && reach[nd0] > dense_reach &&
+                   specs[order[nd0]].prefilter != 2)
+                ++nd0;
             while (nd0 + nfq < nfilter && nfq < kMaxQueues - 1 && specs[order[nd0 + nfq]].sel < 0.9 &&
-                   reach[nd0 + nfq] > 0.002)
+                   reach[nd0 + nfq] > 0.002 && specs[order[nd0 + nfq]].prefilter != 2)
                 ++nfq;
         }
     }
@@ -301,7 +328,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         if (c.src == SJQ_SRC_FACT) {
             if (stage_of_col[c.a] < 0) { // a column nobody filters on: plain load stage at the end
                 if (ns >= kMaxStages) return SJQ_ERR_UNSUPPORTED;
-                StageSpec sp{ST_LOAD, -1, c.a, 1.0, 1.0};
+                StageSpec sp{ST_LOAD, -1, c.a, 1.0, 1.0, 0};
                 fill_stage(P.st[ns], sp);
                 stage_of_col[c.a] = ns;
                 stage_label.push_back(-1);
@@ -499,7 +526,9 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     if (info) {
         std::memset(info, 0, sizeof(*info));
         info->nstages = ns;
-        for (int s = 0; s < ns; ++s) {
+        const int shown = std::min<int>(ns, (int)(sizeof(info->order) / sizeof(info->order[0])));
+        info->nstages = shown;
+        for (int s = 0; s < shown; ++s) {
             info->order[s] = stage_label[s];
             info->stage_in_smem[s] = P.st[s].in_smem;
         }

@@ -23,7 +23,8 @@ enum : uint8_t {
     OP_DIRECT_U32 = 6,
     OP_DIRECT_U64 = 7,
     OP_HASH32 = 8,
-    OP_HASH64 = 9
+    OP_HASH64 = 9,
+    OP_HASHBITS = 10 // presence bitmap in front of an open-addressing table, indexed by a hash of the key
 };
 
 // which accumulators a stage's values feed: bit = 3 * source + destination,
@@ -31,7 +32,7 @@ enum : uint8_t {
 // destination 0 = group key, 1 = X, 2 = Y.  value = X (or X*Y for a product).
 constexpr int kAccKey = 0, kAccX = 1, kAccY = 2;
 
-constexpr int kMaxStages = SJQ_MAX_PREDS + SJQ_MAX_JOINS + 8 + SJQ_MAX_JOINS + SJQ_MAX_PREDS;
+constexpr int kMaxStages = 72; // predicates + joins (two stages when hashed) + plain loads + gather copies
 
 // Geometry of the fused kernel.
 #ifndef SJQ_SLOTS

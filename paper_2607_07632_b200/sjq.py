@@ -65,7 +65,7 @@ class DimLayout(ctypes.Structure):
                 ("code_bits", ctypes.c_int32), ("dim_rows", ctypes.c_int64), ("entries", ctypes.c_int64),
                 ("kmin", ctypes.c_int64), ("kmax", ctypes.c_int64), ("pay_min", ctypes.c_int64 * MAX_PAYLOADS),
                 ("pay_max", ctypes.c_int64 * MAX_PAYLOADS), ("pay_bits", ctypes.c_int32 * MAX_PAYLOADS),
-                ("slots", ctypes.c_int64), ("table_bytes", ctypes.c_size_t)]
+                ("slots", ctypes.c_int64), ("filter_bits", ctypes.c_int64), ("table_bytes", ctypes.c_size_t)]
 
     @property
     def kind_name(self) -> str:
