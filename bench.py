@@ -224,6 +224,10 @@ def main():
     import torch
     import torch.distributed as dist
 
+    from paper_2607_07632_b200 import build as sjq_build
+
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        sjq_build.build()  # compiles libsjq.so only if it is missing or older than its sources
     import paper_2607_07632_b200 as sjq
     from datagen import workloads as W
     from paper_2607_07632_b200 import shard
@@ -422,6 +426,7 @@ def run_extras(sjq, W, device):
     timed(W.config1())
     timed(W.config2())
     timed(W.config5())
+    timed(W.city_pair())  # beyond the five configurations: many groups, few survivors
     for s in (0.0001, 0.01, 0.1, 0.5, 1.0):
         for g in (1, 1000, 100000, 1000000):
             timed(W.config4(600_000_000, s, g))

@@ -258,6 +258,31 @@ def config5(n: int = 300_000_000, dim_rows: int = 8_000_000) -> Workload:
                     AggExpr("COL", Term("FACT", "measure")), "DENSE", num_groups=4096)
 
 
+def city_pair(n: int = 600_000_000) -> Workload:
+    """Beyond the five benchmark configurations: the paper's city x city shape (Section 3.3: hundreds of
+    thousands of groups, few survivors, global group table).  Customer and supplier each carry a city
+    U[0,249] and a nation = city // 10; both are filtered to one nation; group by (customer city,
+    supplier city, year) = 250 * 250 * 7 = 437,500 dense groups; sum(revenue)."""
+    base = 600
+    fact = (ColSpec("custkey", UNIFORM_I32, base + 0, 1, 3000000),
+            ColSpec("suppkey", UNIFORM_I32, base + 1, 1, 200000),
+            ColSpec("orderdate", DATE_FK_I32, base + 2),
+            ColSpec("revenue", UNIFORM_I32, base + 3, 100000, 10000000))
+    cust = DimSpec("customer", 3000000,
+                   (ColSpec("custkey", SEQ_I32), ColSpec("city", UNIFORM_I32, base + 50, 0, 249),
+                    ColSpec("nation", UNIFORM_DIV_I32, base + 50, 0, 249, div=10)),
+                   key="custkey", preds=(Pred("nation", "EQ", 7),), payloads=("city",))
+    supp = DimSpec("supplier", 200000,
+                   (ColSpec("suppkey", SEQ_I32), ColSpec("city", UNIFORM_I32, base + 60, 0, 249),
+                    ColSpec("nation", UNIFORM_DIV_I32, base + 60, 0, 249, div=10)),
+                   key="suppkey", preds=(Pred("nation", "EQ", 7),), payloads=("city",))
+    date = _date_dim(payloads=("year",))
+    key = KeyExpr((Term("PAYLOAD", 0, 0, 250 * 7), Term("PAYLOAD", 1, 0, 7), Term("PAYLOAD", 2, 0, 1)), offset=-1992)
+    return Workload("city_pair_groupby", n, fact, (cust, supp, date),
+                    (("custkey", "customer"), ("suppkey", "supplier"), ("orderdate", "date")), (), key,
+                    AggExpr("COL", Term("FACT", "revenue")), "DENSE", num_groups=250 * 250 * 7)
+
+
 def with_rows(w: Workload, n: int) -> Workload:
     return replace(w, n_rows=n)
 

@@ -295,3 +295,19 @@ def test_stale_layout_is_reported_not_followed():
     t = b.finish()
     torch.cuda.synchronize()
     assert t.status() == 21
+
+
+def test_city_pair_shape_many_groups_few_survivors():
+    # two gathered payloads plus the year as group key, 437,500 dense groups, global group table
+    w = W.city_pair(3_000_017)
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    res, exp, tables = run_both(w, fact, hd)
+    assert res.status() == 0 and res.info.describe()["agg_path"] == "global"
+    compare(w, res, exp)
+    assert int(res.counts.sum().item()) > 1000
+    # the same query with a hashed result list
+    wh = replace(w, mode="HASHED", capacity=1 << 16)
+    res, exp, _ = run_both(wh, fact, hd, tables=tables)
+    assert res.status() == 0
+    compare(wh, res, exp)
