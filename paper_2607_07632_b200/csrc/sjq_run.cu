@@ -298,7 +298,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     const double survivors = (double)n * reach[nfilter];
     // Level 0 runs, on thread-owned rows, the leading filter stages that still see a fair share of
     // the rows (a dense stage costs about the same per table row whatever survives, a queue-fed
-    // level costs per surviving row, roughly fifteen times more: measured break-even near 6 %).
+    // level costs per surviving row, several times more: measured break-even between 20 % and 30 %).
     // Up to kMaxQueues - 1 later filter stages run as queue-fed levels; the rest at the final level.
     // Eager loading and compaction = never use no queue at all.
     int nd0 = 0, nfq = 0;
@@ -306,7 +306,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     if (!direct) {
         nd0 = 1;
         if (opts.compaction != 2) {
-            const double dense_reach = opts.reserved[0] > 0 ? opts.reserved[0] / 1000.0 : 0.06;
+            const double dense_reach = opts.reserved[0] > 0 ? opts.reserved[0] / 1000.0 : 0.3;
             while (nd0 < nfilter && specs[order[nd0]].sel < 0.9 && reach[nd0] > dense_reach &&
                    specs[order[nd0]].prefilter != 2)
                 ++nd0;
