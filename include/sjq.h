@@ -50,6 +50,8 @@ enum {
     SJQ_ERR_CUDA = 4,         /* a CUDA runtime call failed (no device, launch error) */
     SJQ_ERR_BUFFER_SMALL = 5, /* caller-provided table / workspace memory too small */
     SJQ_ERR_STATIC_LIMIT = 6, /* request exceeds the built-in scratch of a no-allocation entry point */
+    SJQ_ERR_JIT = 7,          /* run-time specialisation asked for but the compiler, the device sources or the
+                                 compiled module are unavailable (sjq_jit_log has the details) */
     /* device-detected (written to the status word) */
     SJQ_ERR_DUP_KEY = 16,        /* two dimension rows passing the filter share a key */
     SJQ_ERR_TABLE_FULL = 17,     /* open-addressing insert found no free slot */
@@ -256,7 +258,13 @@ typedef struct sjq_run_opts {
     int32_t order[SJQ_MAX_PREDS + SJQ_MAX_JOINS]; /* entry < npreds: predicate index; else npreds + join index */
     void *event_before; /* optional cudaEvent_t recorded on `stream` right before the fused kernel */
     void *event_after;  /* optional cudaEvent_t recorded right after it (both or neither) */
-    int32_t reserved[8];
+    int32_t dense_reach_permille; /* experiment knob: level 0 keeps the filter stages that more than this share of
+                                     the rows still reach (0 = default, 300) */
+    int32_t specialise; /* 1 = compile the fused kernel for this query's shape at run time (NVRTC) and cache the
+                           module for later runs of the same shape; 0 = interpret the descriptor (default).  Key
+                           ranges, thresholds, table sizes and pointers stay run-time values, so a compiled module
+                           is reused when only they change.  Same results either way. */
+    int32_t reserved[6];
 } sjq_run_opts;
 
 /* What the planner decided for a run (for reports and tests). */
@@ -364,6 +372,18 @@ sjq_status sjq_run_hashed_static(const sjq_col *fact, int nfact, const sjq_pred 
 
 const char *sjq_strerror(sjq_status status);
 const char *sjq_version(void);
+
+/*
+ * Run-time specialisation (Section 4.2 of the paper fuses a query's operators before it runs; here the fused
+ * kernel is compiled for the query's shape with NVRTC when sjq_run_opts.specialise is set).
+ * sjq_jit_log copies the compiler output of the most recent compilation into `buf` (NUL-terminated, truncated
+ * to `bytes`) and returns its full length.  sjq_jit_selftest compiles one of a few built-in query shapes
+ * (shape_id 0 .. sjq_jit_selftest(-1, ...) - 1) without touching a device: SJQ_OK if the device code
+ * compiles for sm_100a, SJQ_ERR_JIT otherwise, with the compiler output in `log`; shape_id -1 returns the number
+ * of built-in shapes instead of a status.
+ */
+size_t sjq_jit_log(char *buf, size_t bytes);
+int32_t sjq_jit_selftest(int32_t shape_id, char *log, size_t log_bytes);
 
 #ifdef __cplusplus
 }

@@ -633,6 +633,7 @@ extern "C" const char *sjq_strerror(sjq_status s)
     case SJQ_ERR_CUDA: return "CUDA runtime error (no device or launch failure)";
     case SJQ_ERR_BUFFER_SMALL: return "caller-provided buffer too small";
     case SJQ_ERR_STATIC_LIMIT: return "request exceeds the built-in scratch of the no-allocation entry point";
+    case SJQ_ERR_JIT: return "run-time specialisation unavailable (compiler, device sources or module load)";
     case SJQ_ERR_DUP_KEY: return "duplicate dimension key among rows passing the filter";
     case SJQ_ERR_TABLE_FULL: return "hash table full";
     case SJQ_ERR_GROUP_RANGE: return "group key outside [0, num_groups)";

@@ -24,6 +24,9 @@
 namespace sjq {
 
 sjq_status fused_occupancy(int agg, bool mul, bool hash, int block, size_t smem, int *ctas_per_sm);
+sjq_status jit_occupancy(const RunParams &P, int agg, bool mul, bool hash, int block, size_t smem, int *ctas_per_sm);
+sjq_status jit_launch(const RunParams &P, int agg, bool mul, bool hash, int grid, int block, size_t smem,
+                      cudaStream_t stream);
 sjq_status fused_launch(int agg, bool mul, bool hash, int grid, int block, size_t smem, const RunParams &P,
                         cudaStream_t stream);
 sjq_status clear_launch(int64_t *sums, int64_t *counts, int64_t cells, int64_t *gkeys, int64_t gslots,
@@ -306,7 +309,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     if (!direct) {
         nd0 = 1;
         if (opts.compaction != 2) {
-            const double dense_reach = opts.reserved[0] > 0 ? opts.reserved[0] / 1000.0 : 0.3;
+            const double dense_reach = opts.dense_reach_permille > 0 ? opts.dense_reach_permille / 1000.0 : 0.3;
             while (nd0 < nfilter && specs[order[nd0]].sel < 0.9 && reach[nd0] > dense_reach &&
                    specs[order[nd0]].prefilter != 2)
                 ++nd0;
@@ -488,7 +491,10 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
 
     // ------------------------------------------------------------ launch shape
     int per_sm = 0;
-    if ((st = fused_occupancy(aggp, mul, has_hash, block, smem, &per_sm)) != SJQ_OK) return st;
+    const bool jit = opts.specialise != 0;
+    st = jit ? jit_occupancy(P, aggp, mul, has_hash, block, smem, &per_sm)
+             : fused_occupancy(aggp, mul, has_hash, block, smem, &per_sm);
+    if (st != SJQ_OK) return st;
     if (per_sm < 1) return SJQ_ERR_UNSUPPORTED;
     if (opts.ctas_per_sm > 0) per_sm = std::min(per_sm, opts.ctas_per_sm);
     const int64_t tile_rows = (int64_t)block * (P.nq ? kDenseRows : kRows);
@@ -512,7 +518,9 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     if (opts.event_before && cudaEventRecord((cudaEvent_t)opts.event_before, stream) != cudaSuccess)
         return SJQ_ERR_CUDA;
     if (n > 0) {
-        if ((st = fused_launch(aggp, mul, has_hash, grid, block, smem, P, stream)) != SJQ_OK) return st;
+        st = jit ? jit_launch(P, aggp, mul, has_hash, grid, block, smem, stream)
+                 : fused_launch(aggp, mul, has_hash, grid, block, smem, P, stream);
+        if (st != SJQ_OK) return st;
         ++launches;
     }
     if (opts.event_after && cudaEventRecord((cudaEvent_t)opts.event_after, stream) != cudaSuccess)

@@ -91,7 +91,8 @@ class _RunOpts(ctypes.Structure):
                 ("agg_path", ctypes.c_int32), ("smem_tables", ctypes.c_int32), ("compaction", ctypes.c_int32),
                 ("accumulate", ctypes.c_int32), ("norder", ctypes.c_int32),
                 ("order", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS)), ("event_before", ctypes.c_void_p),
-                ("event_after", ctypes.c_void_p), ("reserved", ctypes.c_int32 * 8)]
+                ("event_after", ctypes.c_void_p), ("dense_reach_permille", ctypes.c_int32), ("specialise", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 6)]
 
 
 class RunInfo(ctypes.Structure):
@@ -120,6 +121,7 @@ class RunOpts:
     order: Sequence[int] = ()
     events: Optional[tuple] = None  # (torch.cuda.Event, torch.cuda.Event), both already recorded once
     dense_reach_permille: int = 0  # experiment knob: level 0 keeps stages reached by more than this share of rows
+    specialise: bool = False  # compile the fused kernel for this query's shape at run time (cached per shape)
 
     def to_c(self) -> _RunOpts:
         o = _RunOpts()
@@ -129,7 +131,8 @@ class RunOpts:
         o.norder = len(self.order)
         for i, v in enumerate(self.order):
             o.order[i] = v
-        o.reserved[0] = self.dense_reach_permille
+        o.dense_reach_permille = self.dense_reach_permille
+        o.specialise = int(self.specialise)
         if self.events is not None:
             o.event_before, o.event_after = self.events[0].cuda_event, self.events[1].cuda_event
         return o
