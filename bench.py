@@ -210,6 +210,8 @@ def main():
     ap.add_argument("--groups", type=int, default=1000, help="c4: number of groups")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-sample-rows", type=int, default=100_000_000)
+    ap.add_argument("--interpret", action="store_true",
+                    help="interpret the query descriptor instead of compiling the fused kernel for the query's shape")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--extras", action="store_true", help="also time the other configurations (N = 1 only)")
@@ -263,7 +265,7 @@ def main():
     def step(i=None):
         nonlocal launches, info
         tables = sjq.build_tables(builders)
-        opts = sjq.RunOpts(events=pairs[i]) if i is not None else None
+        opts = sjq.RunOpts(events=pairs[i] if i is not None else None, specialise=not args.interpret)
         r = sjq.run_workload(w, fact, tables, opts, result=res)
         if world > 1 and w.mode != "HASHED":
             shard.merge_dense(res.sums, res.counts)
@@ -307,7 +309,7 @@ def main():
     alg_bpr = algorithmic_bytes_per_row(w, list(info.order[: info.nstages]))
     achieved = n * alg_bpr / (fused_ms / 1000.0) / 1e9
     traffic_bpr = NCU_DRAM_BYTES_PER_ROW.get(args.workload)
-    roofline = {"bound": "hbm", "kernel": "fused_kernel", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": "fused_kernel" if args.interpret else "sjq_jit_kernel", "achieved": achieved, "peak": peak,
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic_bpr * n if traffic_bpr else None,
                 "algorithmic_bytes_per_row": alg_bpr, "kernel_ms": fused_ms,
@@ -327,7 +329,8 @@ def main():
             def e2e_step():
                 nonlocal eres, ehost
                 tabs = sjq.build_tables(builders)
-                eres, ehost = sjq.run_workload_host(w, host_fact, tabs, staging, chunk, result=eres, host=ehost)
+                eres, ehost = sjq.run_workload_host(w, host_fact, tabs, staging, chunk,
+                                                    sjq.RunOpts(specialise=not args.interpret), result=eres, host=ehost)
                 torch.cuda.synchronize()  # the result is on the host when this returns
                 return tabs
 
@@ -364,13 +367,13 @@ def main():
     if args.extras and world == 1 and rank == 0:
         del fact
         torch.cuda.empty_cache()
-        extras = run_extras(sjq, W, device)
+        extras = run_extras(sjq, W, device, not args.interpret)
     ablation = None
     if args.ablation and world == 1 and rank == 0:
         if "fact" in locals():
             del fact
         torch.cuda.empty_cache()
-        ablation = run_ablation(sjq, W, device)
+        ablation = run_ablation(sjq, W, device, not args.interpret)
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -380,7 +383,9 @@ def main():
                            "step": "plan+build of every dimension table (on side streams; the key-range scans may overlap the previous step's fused pass), then the fused pass"
                                    + (", then all-reduce of the dense result" if world > 1 else ""),
                            "l2": "inputs (%.1f GB) exceed the 126 MB L2; no flush needed" % (n * ref_bytes / 1e9),
-                           "parallelism": f"row-sharded x{world}, dimensions replicated", "plan": info.describe()},
+                           "parallelism": f"row-sharded x{world}, dimensions replicated", "plan": info.describe(),
+                           "fused_kernel": "interpreted descriptor" if args.interpret else
+                                           "compiled for the query's shape at run time during warm-up (NVRTC), cached"},
                 "effective_gbs": eff_gbs, "pct_of_8tbs": 100.0 * eff_gbs / world / CONTRACT_HBM_GBS,
                 "pct_of_measured_copy_peak": 100.0 * eff_gbs / world / peak,
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
@@ -395,7 +400,7 @@ def main():
     return 0
 
 
-def run_extras(sjq, W, device):
+def run_extras(sjq, W, device, specialise=True):
     """Run-only timings (tables prebuilt) of the other configurations: min and mean of 10 after a warm-up."""
     import torch
 
@@ -405,13 +410,14 @@ def run_extras(sjq, W, device):
         dims = {d.name: W.device_dim(w, d, device) for d in w.dims}
         tables = sjq.build_workload_tables(w, dims)
         fact = W.device_fact(w, device=device)
-        res = sjq.run_workload(w, fact, tables)
+        opts = sjq.RunOpts(specialise=specialise)
+        res = sjq.run_workload(w, fact, tables, opts)
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ts = []
         for _ in range(10):
             e0.record()
-            sjq.run_workload(w, fact, tables, result=res)
+            sjq.run_workload(w, fact, tables, opts, result=res)
             e1.record()
             torch.cuda.synchronize()
             ts.append(e0.elapsed_time(e1))
@@ -433,7 +439,7 @@ def run_extras(sjq, W, device):
     return out
 
 
-def run_ablation(sjq, W, device):
+def run_ablation(sjq, W, device, specialise=True):
     """The paper's A/B experiments restated on this kernel (run-only, min of 5 after a warm-up):
     lazy vs unconditional column loads (its tile-vs-direct table), survivor queues on/off, packed
     direct-mapped vs open-addressing tables, privatised vs global group-by (its ablation figure)."""
@@ -450,6 +456,10 @@ def run_ablation(sjq, W, device):
                       for d in w.dims}
         if fact is None:
             fact = W.device_fact(w, device=device)
+        if opts is None:
+            opts = sjq.RunOpts()
+        if label != INTERPRETED:
+            opts.specialise = specialise
         res = sjq.run_workload(w, fact, tables, opts)
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -467,10 +477,12 @@ def run_ablation(sjq, W, device):
                     "plan": res.info.describe()})
         return fact, dims
 
+    INTERPRETED = "query descriptor interpreted (no run-time specialisation)"
     for mk in (W.config3, W.config2):
         w = mk()
         fact, dims = timed(w, "default")
-        for label, opts in (("eager loads (every column for every row)", sjq.RunOpts(eager_loads=True)),
+        for label, opts in ((INTERPRETED, sjq.RunOpts()),
+                            ("eager loads (every column for every row)", sjq.RunOpts(eager_loads=True)),
                             ("no survivor queues (thread-owned rows throughout)", sjq.RunOpts(compaction=1)),
                             ("one queue only", sjq.RunOpts(compaction=2)),
                             ("global atomics group-by", sjq.RunOpts(agg_path=2)),

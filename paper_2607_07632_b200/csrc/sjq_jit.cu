@@ -141,12 +141,14 @@ void put(std::ostringstream &o, const char *name, long long v) { o << "#define S
 
 // The shape of a run as a header of constants.  Two runs with the same text
 // use the same compiled module.
-std::string jit_shape_header(const RunParams &P, int agg, bool mul, bool hash)
+std::string jit_shape_header(const RunParams &P, int agg, bool mul, bool hash, int lb_threads, int lb_blocks)
 {
     std::ostringstream o;
     o << "// generated: the shape of one query\n";
     o << "#define SJQ_JIT_AGG " << agg << "\n#define SJQ_JIT_MUL " << (mul ? 1 : 0) << "\n#define SJQ_JIT_HASH "
       << (hash ? 1 : 0) << "\n";
+    o << "#define SJQ_LB_THREADS " << lb_threads << "\n#define SJQ_LB_BLOCKS " << lb_blocks << "\n";
+    if (const char *extra = std::getenv("SJQ_JIT_EXTRA")) o << "// options: " << extra << "\n";
     o << "#define SJQ_JIT_nstages " << P.nstages << "\n#define SJQ_JIT_nd0 " << P.nd0 << "\n#define SJQ_JIT_nq " << P.nq
       << "\n";
     o << "#define SJQ_JIT_want_count " << P.want_count << "\n#define SJQ_JIT_eager " << P.eager
@@ -214,6 +216,13 @@ sjq_status compile(const std::string &shape, std::vector<char> *cubin, std::stri
     std::vector<const char *> opts = {"--gpu-architecture=sm_100a", "-std=c++17", "-lineinfo", "-default-device",
                                       "--disable-warnings"};
     if (std::getenv("SJQ_JIT_VERBOSE")) opts.push_back("--ptxas-options=-v");
+    std::vector<std::string> extra; // experiment switches, e.g. SJQ_JIT_EXTRA="-DSJQ_PREFETCH_DIST=3"
+    if (const char *e = std::getenv("SJQ_JIT_EXTRA")) {
+        std::istringstream is(e);
+        std::string tok;
+        while (is >> tok) extra.push_back(tok);
+    }
+    for (const std::string &t : extra) opts.push_back(t.c_str());
     const int rc = N.CompileProgram(prog, (int)opts.size(), opts.data());
     size_t ls = 0;
     if (N.GetProgramLogSize(prog, &ls) == 0 && ls > 1) {
@@ -259,11 +268,12 @@ sjq_status module_for(const std::string &shape, Module **out)
 
 } // namespace
 
-sjq_status jit_occupancy(const RunParams &P, int agg, bool mul, bool hash, int block, size_t smem, int *ctas_per_sm)
+sjq_status jit_occupancy(const RunParams &P, int agg, bool mul, bool hash, int block, int lb_blocks, size_t smem,
+                         int *ctas_per_sm)
 {
     std::lock_guard<std::mutex> lock(g_mutex);
     Module *M = nullptr;
-    sjq_status st = module_for(jit_shape_header(P, agg, mul, hash), &M);
+    sjq_status st = module_for(jit_shape_header(P, agg, mul, hash, block, lb_blocks), &M);
     if (st != SJQ_OK) return st;
     if ((int)smem > M->smem_set) {
         if (cudaFuncSetAttribute(reinterpret_cast<const void *>(M->kernel), cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -281,14 +291,14 @@ sjq_status jit_occupancy(const RunParams &P, int agg, bool mul, bool hash, int b
     return SJQ_OK;
 }
 
-sjq_status jit_launch(const RunParams &P, int agg, bool mul, bool hash, int grid, int block, size_t smem,
-                      cudaStream_t stream)
+sjq_status jit_launch(const RunParams &P, int agg, bool mul, bool hash, int grid, int block, int lb_blocks,
+                      size_t smem, cudaStream_t stream)
 {
     cudaKernel_t kernel;
     {
         std::lock_guard<std::mutex> lock(g_mutex);
         Module *M = nullptr;
-        sjq_status st = module_for(jit_shape_header(P, agg, mul, hash), &M);
+        sjq_status st = module_for(jit_shape_header(P, agg, mul, hash, block, lb_blocks), &M);
         if (st != SJQ_OK) return st;
         kernel = M->kernel;
     }
@@ -411,7 +421,7 @@ extern "C" int32_t sjq_jit_selftest(int32_t shape_id, char *log, size_t log_byte
     if (!sjq::canned_shape(shape_id, &P, &agg, &mul, &hash)) return SJQ_ERR_INVALID_ARG;
     std::string text;
     size_t cubin = 0;
-    const sjq_status st = sjq::jit_compile_only(sjq::jit_shape_header(P, agg, mul, hash), &text, &cubin);
+    const sjq_status st = sjq::jit_compile_only(sjq::jit_shape_header(P, agg, mul, hash, 384, 2), &text, &cubin);
     if (log && log_bytes) {
         const size_t n = text.size() < log_bytes - 1 ? text.size() : log_bytes - 1;
         std::memcpy(log, text.data(), n);

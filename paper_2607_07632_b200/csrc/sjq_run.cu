@@ -24,9 +24,10 @@
 namespace sjq {
 
 sjq_status fused_occupancy(int agg, bool mul, bool hash, int block, size_t smem, int *ctas_per_sm);
-sjq_status jit_occupancy(const RunParams &P, int agg, bool mul, bool hash, int block, size_t smem, int *ctas_per_sm);
-sjq_status jit_launch(const RunParams &P, int agg, bool mul, bool hash, int grid, int block, size_t smem,
-                      cudaStream_t stream);
+sjq_status jit_occupancy(const RunParams &P, int agg, bool mul, bool hash, int block, int lb_blocks, size_t smem,
+                         int *ctas_per_sm);
+sjq_status jit_launch(const RunParams &P, int agg, bool mul, bool hash, int grid, int block, int lb_blocks,
+                      size_t smem, cudaStream_t stream);
 sjq_status fused_launch(int agg, bool mul, bool hash, int grid, int block, size_t smem, const RunParams &P,
                         cudaStream_t stream);
 sjq_status clear_launch(int64_t *sums, int64_t *counts, int64_t cells, int64_t *gkeys, int64_t gslots,
@@ -138,7 +139,9 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     }
     if (!valid_term(agg->x, nfact, joins, njoins)) return SJQ_ERR_INVALID_ARG;
     if (agg->op != SJQ_AGG_COL && !valid_term(agg->y, nfact, joins, njoins)) return SJQ_ERR_INVALID_ARG;
-    if (opts.block_threads && (opts.block_threads < 128 || opts.block_threads > SJQ_LB_THREADS_MAX || opts.block_threads % 32))
+    // the ahead-of-time kernels are bounded at SJQ_LB_THREADS_MAX; a specialised kernel is compiled for its block size
+    if (opts.block_threads && (opts.block_threads < 128 || opts.block_threads % 32 ||
+                               opts.block_threads > (opts.specialise ? 1024 : SJQ_LB_THREADS_MAX)))
         return SJQ_ERR_INVALID_ARG;
     if (opts.norder && opts.norder != npreds + njoins) return SJQ_ERR_INVALID_ARG;
 
@@ -492,7 +495,8 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     // ------------------------------------------------------------ launch shape
     int per_sm = 0;
     const bool jit = opts.specialise != 0;
-    st = jit ? jit_occupancy(P, aggp, mul, has_hash, block, smem, &per_sm)
+    const int lb_blocks = opts.ctas_per_sm > 0 ? opts.ctas_per_sm : 2; // register budget a specialised kernel is compiled for
+    st = jit ? jit_occupancy(P, aggp, mul, has_hash, block, lb_blocks, smem, &per_sm)
              : fused_occupancy(aggp, mul, has_hash, block, smem, &per_sm);
     if (st != SJQ_OK) return st;
     if (per_sm < 1) return SJQ_ERR_UNSUPPORTED;
@@ -518,7 +522,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     if (opts.event_before && cudaEventRecord((cudaEvent_t)opts.event_before, stream) != cudaSuccess)
         return SJQ_ERR_CUDA;
     if (n > 0) {
-        st = jit ? jit_launch(P, aggp, mul, has_hash, grid, block, smem, stream)
+        st = jit ? jit_launch(P, aggp, mul, has_hash, grid, block, lb_blocks, smem, stream)
                  : fused_launch(aggp, mul, has_hash, grid, block, smem, P, stream);
         if (st != SJQ_OK) return st;
         ++launches;

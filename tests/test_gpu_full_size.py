@@ -1,5 +1,6 @@
-"""Parity at the benchmark's full sizes, in the launch configuration bench.py
-times (default options, inputs generated on the device): the result must equal,
+"""Parity at the benchmark's full sizes, in the launch configurations bench.py
+times (the fused kernel compiled for the query's shape, which is its default,
+and the interpreted descriptor; inputs generated on the device): each result must equal,
 bit for bit, the expected values the CPU oracle wrote to tests/golden/full_*.json
 (tests/golden/make_full_size.py).  Hashed results are compared through the
 SHA-256 of their (key, sum, count) triples in ascending key order."""
@@ -31,20 +32,28 @@ def _run(w):
     dims = {d.name: W.device_dim(w, d) for d in w.dims}
     tables = sjq.build_workload_tables(w, dims)
     fact = W.device_fact(w)
-    res = sjq.run_workload(w, fact, tables)
-    torch.cuda.synchronize()
-    assert res.status() == 0 and all(t.status() == 0 for t in tables.values())
+    results = []
+    for specialise in (True, False):
+        res = sjq.run_workload(w, fact, tables, sjq.RunOpts(specialise=specialise))
+        torch.cuda.synchronize()
+        assert res.status() == 0 and all(t.status() == 0 for t in tables.values())
+        results.append(res)
     entries = {k: t.layout.entries for k, t in tables.items()}
     del fact
     torch.cuda.empty_cache()
-    return res, entries
+    return results, entries
 
 
 def _check(w, tag):
     g = _golden(tag)
     assert g["rows"] == w.n_rows and g["workload"] == w.name
-    res, entries = _run(w)
+    results, entries = _run(w)
     assert entries == g["dim_entries"]
+    for res in results:
+        _compare(w, g, res)
+
+
+def _compare(w, g, res):
     if w.mode == "SCALAR":
         assert int(res.sums[0].item()) == g["sum"] and int(res.counts[0].item()) == g["count"]
     elif w.mode == "DENSE":

@@ -1,0 +1,132 @@
+"""Parity of the run-time specialised fused kernel (sjq_run_opts.specialise)
+with the CPU oracle: the same bits as the interpreted kernel, on the same
+seeded inputs, over query shapes, option switches, ragged sizes and edge cases."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from datagen import workloads as W
+from datagen.workloads import AggExpr, KeyExpr, Pred, Term
+
+pytestmark = pytest.mark.gpu
+
+sjq = pytest.importorskip("paper_2607_07632_b200") if torch.cuda.is_available() else None
+
+from gpuhelpers import compare, run_both, to_dev  # noqa: E402
+from qhelpers import ex1, ex2, ex3, random_query  # noqa: E402
+
+
+def spec(**kw):
+    return sjq.RunOpts(specialise=True, **kw)
+
+
+def test_hand_examples_specialised():
+    for mk in (ex1, ex2, ex3):
+        w, fact, hd, _ = mk()
+        res, exp, _ = run_both(w, fact, hd, opts=spec())
+        assert res.status() == 0
+        compare(w, res, exp)
+
+
+@pytest.mark.parametrize("seed", range(300, 348))
+def test_random_small_queries_specialised(seed):
+    w, fact, hd = random_query(seed, allow_dup=False, wide_keys=True)
+    res, exp, _ = run_both(w, fact, hd, opts=spec(), check=False)
+    assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)
+    compare(w, res, exp)
+
+
+@pytest.mark.parametrize("seed", range(348, 356))
+def test_random_queries_option_matrix_specialised(seed):
+    w, fact, hd = random_query(seed, n_fact=700, allow_dup=False, wide_keys=True)
+    dev_fact = to_dev(fact)
+    tables = None
+    for opts in (spec(eager_loads=True), spec(smem_tables=1), spec(block_threads=128, ctas_per_sm=1),
+                 spec(block_threads=1024, ctas_per_sm=1), spec(block_threads=512, compaction=2, smem_tables=2),
+                 spec(agg_path=2), spec(compaction=1),
+                 spec(order=tuple(reversed(range(len(w.preds) + len(w.joins)))))):
+        res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)
+        assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)
+        compare(w, res, exp)
+
+
+@pytest.mark.parametrize("n", [0, 1, 5, 257, 3071, 3073, 100003])
+@pytest.mark.parametrize("cfg", ["c1", "c2", "c3", "c4d", "c4h", "c5"])
+def test_configs_ragged_sizes_specialised(cfg, n):
+    w = {"c1": lambda: W.config1(n), "c2": lambda: W.config2(n), "c3": lambda: W.config3(n),
+         "c4d": lambda: W.config4(n, 0.5, 1000, dim_rows=50000),
+         "c4h": lambda: W.config4(n, 0.5, 100000, dim_rows=50000),
+         "c5": lambda: W.config5(n, 20000)}[cfg]()
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    res, exp, _ = run_both(w, fact, hd, opts=spec())
+    assert res.status() == 0
+    compare(w, res, exp)
+
+
+@pytest.mark.parametrize("mk", [lambda: W.config1(1_500_007), lambda: W.config2(2_000_003),
+                                lambda: W.config3(2_500_001), lambda: W.config5(1_200_005, 300000),
+                                lambda: W.city_pair(1_000_003)] +
+                         [lambda s=s, g=g: W.config4(1_000_003, s, g) for s in (0.0001, 0.1, 1.0)
+                          for g in (1, 1000, 100000, 1000000)])
+def test_configs_multi_tile_specialised(mk):
+    w = mk()
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    res, exp, tables = run_both(w, fact, hd, opts=spec())
+    assert res.status() == 0
+    compare(w, res, exp)
+    dev_fact = to_dev(fact)
+    for opts in (spec(eager_loads=True, smem_tables=1, compaction=1),
+                 spec(agg_path=2 if w.mode == "DENSE" else 0, block_threads=768, ctas_per_sm=1, compaction=2)):
+        res2, _, _ = run_both(w, fact, hd, opts=opts, dev_fact=dev_fact, tables=tables)
+        compare(w, res2, exp)
+
+
+def test_one_module_serves_runs_that_differ_only_in_data_dependent_values():
+    """Thresholds, key ranges and table contents are kernel parameters, not part of the compiled shape:
+    changing them must not need (or wrongly reuse state of) another module, and the results stay exact."""
+    n = 200_003
+    for t in (1, 100, 5000, 10000):
+        w = W.config4(n, t / 10000.0, 1000, dim_rows=30000 + t)
+        fact = W.host_fact(w)
+        hd = {d.name: W.host_dim(w, d) for d in w.dims}
+        res, exp, _ = run_both(w, fact, hd, opts=spec())
+        assert res.status() == 0
+        compare(w, res, exp)
+
+
+def test_group_range_and_overflow_status_specialised():
+    w, fact, hd, _ = ex2()
+    from dataclasses import replace
+    small = replace(w, num_groups=1500)  # keys 2020 fall outside
+    res, exp, _ = run_both(small, fact, hd, opts=spec(), check=False)
+    assert res.status() == 18 and exp["status"] == oracle.GROUP_RANGE
+    compare(small, res, exp)
+
+
+def test_host_buffer_entry_point_specialised():
+    w = W.config3(300_007)
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    dims = oracle.build_dims(w, hd)
+    exp = oracle.run(w, fact, dims)
+    tables = sjq.build_workload_tables(w, {k: to_dev(v) for k, v in hd.items()})
+    host_fact = {k: torch.from_numpy(np.ascontiguousarray(v)).pin_memory() for k, v in fact.items()}
+    chunk = 65536
+    staging = torch.empty(sjq.staging_bytes(host_fact, chunk), dtype=torch.uint8, device="cuda:0")
+    res, host = sjq.run_workload_host(w, host_fact, tables, staging, chunk, spec())
+    torch.cuda.synchronize()
+    assert np.array_equal(host.sums.numpy(), exp["sums"])
+
+
+def test_compiler_log_is_readable():
+    L = sjq.sjq.lib()
+    L.sjq_jit_log.restype = ctypes.c_size_t
+    L.sjq_jit_log.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
+    buf = ctypes.create_string_buffer(4096)
+    n = L.sjq_jit_log(buf, len(buf))
+    assert n >= 0 and len(buf.value) <= 4095

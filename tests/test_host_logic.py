@@ -65,3 +65,18 @@ def test_product_never_imports_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in text.lower(), f
+
+
+def test_device_source_compiles_for_builtin_query_shapes(libsjq):
+    """Run-time specialisation needs no device to compile: every built-in query shape (scalar with a
+    product aggregate, four joins with a shared-memory group table, 64-bit open addressing with a
+    presence bitmap, no queues with a global group hash table) must compile for sm_100a with NVRTC."""
+    libsjq.sjq_jit_selftest.restype = ctypes.c_int32
+    libsjq.sjq_jit_selftest.argtypes = [ctypes.c_int32, ctypes.c_char_p, ctypes.c_size_t]
+    n = libsjq.sjq_jit_selftest(-1, None, 0)
+    assert n >= 4
+    for i in range(n):
+        log = ctypes.create_string_buffer(1 << 16)
+        rc = libsjq.sjq_jit_selftest(i, log, len(log))
+        assert rc == 0, (i, log.value.decode()[:2000])
+    assert libsjq.sjq_jit_selftest(n, None, 0) == 1  # no such shape: invalid argument
