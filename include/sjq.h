@@ -264,7 +264,9 @@ typedef struct sjq_run_opts {
                            module for later runs of the same shape; 0 = interpret the descriptor (default).  Key
                            ranges, thresholds, table sizes and pointers stay run-time values, so a compiled module
                            is reused when only they change.  Same results either way. */
-    int32_t reserved[6];
+    int32_t rows_per_lane; /* rows a lane handles per batch at the queue-fed levels: 0 = library chooses, 4, or 8
+                              (8 only with specialise: the ahead-of-time kernels are built for 4) */
+    int32_t reserved[5];
 } sjq_run_opts;
 
 /* What the planner decided for a run (for reports and tests). */

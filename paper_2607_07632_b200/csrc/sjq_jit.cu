@@ -144,7 +144,7 @@ void put(std::ostringstream &o, const char *name, long long v) { o << "#define S
 std::string jit_shape_header(const RunParams &P, int agg, bool mul, bool hash, int lb_threads, int lb_blocks)
 {
     std::ostringstream o;
-    o << "// generated: the shape of one query\n";
+    o << "// generated: the shape of one query\n#define SJQ_ROWS " << (P.rows == 8 ? 8 : 4) << "\n//@body\n";
     o << "#define SJQ_JIT_AGG " << agg << "\n#define SJQ_JIT_MUL " << (mul ? 1 : 0) << "\n#define SJQ_JIT_HASH "
       << (hash ? 1 : 0) << "\n";
     o << "#define SJQ_LB_THREADS " << lb_threads << "\n#define SJQ_LB_BLOCKS " << lb_blocks << "\n";
@@ -202,10 +202,15 @@ sjq_status compile(const std::string &shape, std::vector<char> *cubin, std::stri
         *log = S.error;
         return SJQ_ERR_JIT;
     }
-    const char *main_src = "#define SJQ_JIT 1\n#include \"sjq_fused_device.cuh\"\n";
+    // what precedes the //@body line of the shape text must be seen before any other header
+    const size_t cut = shape.find("//@body\n");
+    const std::string main_text = "#define SJQ_JIT 1\n" + shape.substr(0, cut == std::string::npos ? 0 : cut) +
+                                  "#include \"sjq_fused_device.cuh\"\n";
+    const std::string shape_body = cut == std::string::npos ? shape : shape.substr(cut);
+    const char *main_src = main_text.c_str();
     const char *names[] = {"sjq_fused_device.cuh", "sjq_run.cuh", "sjq_internal.h", "sjq.h", "sjq_jit_shape.h",
                            "stdint.h",             "stddef.h",    "cuda_runtime.h"};
-    const char *bodies[] = {S.device.c_str(), S.run.c_str(), S.internal.c_str(), S.api.c_str(), shape.c_str(),
+    const char *bodies[] = {S.device.c_str(), S.run.c_str(), S.internal.c_str(), S.api.c_str(), shape_body.c_str(),
                             kStdint,          kEmptyHeader,  kEmptyHeader};
     nvrtcProgram prog = nullptr;
     if (N.CreateProgram(&prog, main_src, "sjq_jit.cu", 8, bodies, names) != 0) {
@@ -387,6 +392,7 @@ int canned_shape(int id, RunParams *P, int *agg, bool *mul, bool *hash)
         P->st[2] = canned(OP_LOAD, ST_LOAD, false, 2, 0, false);
         P->nstages = 3, P->nd0 = 1, P->nq = 1;
         P->modulo = 4096, P->modmask = 4095, P->mod32 = 1, P->want_count = 1;
+        P->rows = 8;
         *agg = AGG_GLOBAL, *hash = true;
         return 1;
     case 3: // no queues, set predicate, 32-bit open addressing, runtime modulo, global group hash table

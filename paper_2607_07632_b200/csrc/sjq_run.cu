@@ -143,6 +143,8 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     if (opts.block_threads && (opts.block_threads < 128 || opts.block_threads % 32 ||
                                opts.block_threads > (opts.specialise ? 1024 : SJQ_LB_THREADS_MAX)))
         return SJQ_ERR_INVALID_ARG;
+    if (opts.rows_per_lane != 0 && opts.rows_per_lane != 4 && !(opts.rows_per_lane == 8 && opts.specialise))
+        return SJQ_ERR_INVALID_ARG;
     if (opts.norder && opts.norder != npreds + njoins) return SJQ_ERR_INVALID_ARG;
 
     DeviceInfo dev;
@@ -324,6 +326,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     const int ndense = nd0 + nfq; // stages that only filter (no accumulators)
     P.nd0 = nd0;
     P.nq = direct ? 0 : nfq + 1;
+    P.rows = opts.rows_per_lane ? opts.rows_per_lane : 4;
 
     // Sources of the accumulators.  A dense stage cannot feed an accumulator
     // (it only keeps a bit per row), so a value it would supply is gathered
@@ -453,7 +456,17 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     int block = opts.block_threads ? opts.block_threads : SJQ_LB_THREADS;
     const size_t smem_cap = (size_t)dev.max_smem_optin - 1024; // static reduce scratch + slack
     const size_t stage_bytes = align_up((size_t)ns * sizeof(DStage), 16);
-    auto queue_bytes = [&](int threads) { return P.nq ? (size_t)(threads / 32) * (size_t)(kQueue0Cap + (P.nq - 1) * kQueueCap) * 4 : (size_t)0; };
+    auto queue_bytes = [&](int threads) { return P.nq ? (size_t)(threads / 32) * (size_t)(kQueue0Cap + (P.nq - 1) * queue_cap_for(P.rows)) * 4 : (size_t)0; };
+    // Two blocks per SM each carry their own group table and queues; when that would take most of the
+    // SM's shared memory (and with it the L1), a kernel compiled for the query runs as one block of 1024
+    // threads per SM instead (config 5, 64 KB group table: 2.8 -> 1.9 ms).
+    bool single_block = false;
+    if (opts.specialise && !opts.block_threads && !opts.ctas_per_sm &&
+        stage_bytes + group_bytes + queue_bytes(block) > ((size_t)80 << 10) &&
+        stage_bytes + group_bytes + queue_bytes(1024) <= smem_cap) {
+        block = 1024;
+        single_block = true;
+    }
     const size_t fixed = stage_bytes + group_bytes + queue_bytes(block);
     if (fixed > smem_cap) return SJQ_ERR_UNSUPPORTED;
     const size_t table_budget = smem_cap - fixed;
@@ -495,13 +508,14 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     // ------------------------------------------------------------ launch shape
     int per_sm = 0;
     const bool jit = opts.specialise != 0;
-    const int lb_blocks = opts.ctas_per_sm > 0 ? opts.ctas_per_sm : 2; // register budget a specialised kernel is compiled for
+    // register budget a specialised kernel is compiled for
+    const int lb_blocks = single_block ? 1 : opts.ctas_per_sm > 0 ? opts.ctas_per_sm : 2;
     st = jit ? jit_occupancy(P, aggp, mul, has_hash, block, lb_blocks, smem, &per_sm)
              : fused_occupancy(aggp, mul, has_hash, block, smem, &per_sm);
     if (st != SJQ_OK) return st;
     if (per_sm < 1) return SJQ_ERR_UNSUPPORTED;
     if (opts.ctas_per_sm > 0) per_sm = std::min(per_sm, opts.ctas_per_sm);
-    const int64_t tile_rows = (int64_t)block * (P.nq ? kDenseRows : kRows);
+    const int64_t tile_rows = (int64_t)block * (P.nq ? kDenseRows : kDirectRows);
     const int64_t ntiles = (n + tile_rows - 1) / tile_rows;
     if (ntiles >= ((int64_t)1 << 31)) return SJQ_ERR_UNSUPPORTED;
     int grid = (int)std::min<int64_t>((int64_t)dev.sm_count * per_sm, std::max<int64_t>(ntiles, 1));

@@ -40,10 +40,15 @@ constexpr int kMaxStages = 72; // predicates + joins (two stages when hashed) + 
 #endif
 constexpr int kSlots = SJQ_SLOTS;        // level 0: 128-bit loads per thread per tile
 constexpr int kDenseRows = 4 * kSlots;   // rows a thread owns at level 0
-constexpr int kRows = 4;                 // rows a lane handles per batch at the queue-fed levels
+#ifndef SJQ_ROWS
+#define SJQ_ROWS 4 // the ahead-of-time kernels; a kernel compiled for one query may use 8
+#endif
+constexpr int kRows = SJQ_ROWS;          // rows a lane handles per batch at the queue-fed levels
+constexpr int kDirectRows = 4;           // rows a thread owns when there are no queues at all (one 128-bit load)
 constexpr int kBatch = 32 * kRows;       // rows a warp processes at once at those levels
 constexpr int kQueue0Cap = kSlots <= 2 ? 512 : 1024; // first queue of a warp: a batch minus one plus a whole tile fit
-constexpr int kQueueCap = 256;           // its later queues: a batch minus one plus a batch fit
+constexpr int queue_cap_for(int rows) { return 64 * rows; }
+constexpr int kQueueCap = queue_cap_for(kRows); // its later queues: a batch minus one plus a batch fit
 constexpr int kMaxQueues = 3;            // queue-fed levels per warp (the last one is the final level)
 
 struct DStage {
@@ -89,6 +94,7 @@ struct RunParams {
                     // filter thread-owned rows at level 0, stages nd0 .. nd0+nq-2 are queue-fed filters and
                     // stages from nd0+nq-1 on run at the final level
     int32_t nd0;
+    int32_t rows;   // rows per lane and batch at the queue-fed levels: 4, or 8 in a kernel compiled for it
     int32_t want_count;
     int32_t eager;   // load every column for every row
     int32_t has_key; // scalar path of a one-group dense result: key is computed and range-checked

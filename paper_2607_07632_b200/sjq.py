@@ -92,7 +92,7 @@ class _RunOpts(ctypes.Structure):
                 ("accumulate", ctypes.c_int32), ("norder", ctypes.c_int32),
                 ("order", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS)), ("event_before", ctypes.c_void_p),
                 ("event_after", ctypes.c_void_p), ("dense_reach_permille", ctypes.c_int32), ("specialise", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 6)]
+                ("rows_per_lane", ctypes.c_int32), ("reserved", ctypes.c_int32 * 5)]
 
 
 class RunInfo(ctypes.Structure):
@@ -122,6 +122,7 @@ class RunOpts:
     events: Optional[tuple] = None  # (torch.cuda.Event, torch.cuda.Event), both already recorded once
     dense_reach_permille: int = 0  # experiment knob: level 0 keeps stages reached by more than this share of rows
     specialise: bool = False  # compile the fused kernel for this query's shape at run time (cached per shape)
+    rows_per_lane: int = 0  # queue-fed levels: 0 auto, 4, or 8 (8 needs specialise)
 
     def to_c(self) -> _RunOpts:
         o = _RunOpts()
@@ -133,6 +134,7 @@ class RunOpts:
             o.order[i] = v
         o.dense_reach_permille = self.dense_reach_permille
         o.specialise = int(self.specialise)
+        o.rows_per_lane = self.rows_per_lane
         if self.events is not None:
             o.event_before, o.event_after = self.events[0].cuda_event, self.events[1].cuda_event
         return o
