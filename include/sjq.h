@@ -149,7 +149,8 @@ typedef struct sjq_dim_layout {
     int64_t pay_max[SJQ_MAX_PAYLOADS];
     int32_t pay_bits[SJQ_MAX_PAYLOADS];
     int64_t slots;      /* direct: kmax-kmin+1; hash: power-of-two slot count */
-    int64_t filter_bits; /* hash: size (power of two, 0 = none) of the presence bitmap indexed by the key's hash,
+    int64_t filter_bits; /* direct with payloads: bits of the presence bitmap over the slots (a multiple of 128);
+                            hash: size (power of two, 0 = none) of the presence bitmap indexed by the key's hash,
                             probed before the table so that most absent keys never touch it */
     size_t table_bytes; /* device bytes sjq_build_dim needs at table_mem */
 } sjq_dim_layout;
@@ -266,7 +267,9 @@ typedef struct sjq_run_opts {
                            is reused when only they change.  Same results either way. */
     int32_t rows_per_lane; /* rows a lane handles per batch at the queue-fed levels: 0 = library chooses, 4, or 8
                               (8 only with specialise: the ahead-of-time kernels are built for 4) */
-    int32_t reserved[5];
+    int32_t no_filter_bitmap; /* 1 = filter stages probe a direct table's code array even when the table has a
+                                 presence bitmap (ablation) */
+    int32_t reserved[4];
 } sjq_run_opts;
 
 /* What the planner decided for a run (for reports and tests). */

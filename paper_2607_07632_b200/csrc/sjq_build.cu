@@ -117,7 +117,7 @@ struct BuildParams {
     int32_t pay_bits[SJQ_MAX_PAYLOADS];
     void *slots;
     void *codes;
-    unsigned int *filter; // hash: presence bitmap words
+    unsigned int *filter; // presence bitmap words (hash: indexed by a hash of the key; direct with payloads: by slot)
     uint32_t fmask;       // hash: filter bits - 1
     unsigned long long *header; // [0] rows inserted, [1] slots occupied
     int32_t *status;
@@ -177,7 +177,10 @@ __global__ void __launch_bounds__(256) build_kernel(const __grid_constant__ Buil
             }
             if (B.kind == SJQ_TABLE_DIRECT_BITMAP)
                 atomicOr(static_cast<unsigned int *>(B.slots) + (idx >> 5), 1u << (idx & 31));
-            else store_code(B.slots, B.code_bits, idx, code); // race-free: keys are unique
+            else {
+                store_code(B.slots, B.code_bits, idx, code); // race-free: keys are unique
+                if (B.filter) atomicOr(B.filter + (idx >> 5), 1u << (idx & 31));
+            }
         } else if (B.kind == SJQ_TABLE_HASH_I64) {
             if (k == kEmptyKey64) {
                 set_status(B.status, SJQ_ERR_RESERVED_KEY);
@@ -502,6 +505,12 @@ extern "C" sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_c
                  : code_bits == 32 ? SJQ_TABLE_DIRECT_U32
                                    : SJQ_TABLE_DIRECT_U64;
         L.table_bytes = kTableHeaderBytes + align_up(direct_bytes, 256);
+        if (npayload > 0) {
+            // a code array is 8 to 64 times the size of a bitmap over the same slots: keep both, so that a
+            // filter stage probes the bitmap and only the survivors gather their payload from the codes
+            L.filter_bits = (int64_t)((span_m1 + 128) / 128 * 128);
+            L.table_bytes += align_up((size_t)(L.filter_bits / 8), 256);
+        }
     } else {
         uint64_t want = ((uint64_t)L.entries * 100u + (uint64_t)load_pct - 1) / (uint64_t)load_pct;
         uint64_t slots = 16;
@@ -532,7 +541,12 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
     sjq_status st = fill_dim_params(cols, ncols, preds, npreds, key_col, payload_cols, npayload, &B.dim);
     if (st != SJQ_OK) return st;
     const sjq_dim_layout &L = *layout;
-    if (L.filter_bits < 0 || (L.filter_bits & (L.filter_bits - 1)) || L.filter_bits > ((int64_t)1 << 32))
+    if (L.kind < SJQ_TABLE_DIRECT_BITMAP || L.kind > SJQ_TABLE_HASH_I64) return SJQ_ERR_INVALID_ARG;
+    if (L.kind >= SJQ_TABLE_HASH_I32 &&
+        (L.filter_bits < 0 || (L.filter_bits & (L.filter_bits - 1)) || L.filter_bits > ((int64_t)1 << 32)))
+        return SJQ_ERR_INVALID_ARG;
+    if (L.kind <= SJQ_TABLE_DIRECT_U64 && L.filter_bits != 0 &&
+        (L.kind == SJQ_TABLE_DIRECT_BITMAP || L.filter_bits < L.slots || L.filter_bits % 128 != 0))
         return SJQ_ERR_INVALID_ARG;
     if (L.kind < SJQ_TABLE_DIRECT_BITMAP || L.kind > SJQ_TABLE_HASH_I64 || L.npayload != npayload ||
         L.key_dtype != cols[key_col].dtype || L.slots <= 0 || L.dim_rows != B.dim.n)
@@ -574,6 +588,11 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
         bytes = align_up(bytes, 16);
         T->slots_bytes = bytes;
         ok = ok && cudaMemsetAsync(T->slots, L.kind == SJQ_TABLE_DIRECT_BITMAP ? 0 : 0xFF, bytes, stream) == cudaSuccess;
+        if (L.filter_bits) {
+            T->filter = T->slots + align_up(bytes, 256);
+            B.filter = reinterpret_cast<unsigned int *>(T->filter);
+            ok = ok && cudaMemsetAsync(T->filter, 0, (size_t)(L.filter_bits / 8), stream) == cudaSuccess;
+        }
     } else {
         const size_t kb = (size_t)L.slots * (L.key_dtype == SJQ_I64 ? 8 : 4);
         T->slots_bytes = kb;

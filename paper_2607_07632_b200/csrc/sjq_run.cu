@@ -163,8 +163,13 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         const sjq_dim_layout &L = T->layout;
         const double bytes = L.key_dtype == SJQ_I64 ? 2.0 : 1.0;
         double sel = L.dim_rows > 0 ? (double)L.entries / (double)L.dim_rows : 0.0;
-        const size_t tb = L.table_bytes;
-        double probe = tb <= (size_t)200 << 10 ? 0.3 : tb <= (size_t)32 << 20 ? 1.5 : 4.0;
+        // bytes a filter stage on this table touches: the presence bitmap when a direct table has one
+        const size_t tb = (L.kind <= SJQ_TABLE_DIRECT_U64 && L.filter_bits > 0 && T->filter && !opts.no_filter_bitmap)
+                              ? (size_t)(L.filter_bits / 8)
+                              : L.table_bytes;
+        // relative cost of one probe: a table the L1 mostly holds, one the L2 holds (measured on the four-join
+        // workload: the 3 MB map before the 175 KB bitmap when it drops twice as many rows), one in HBM
+        double probe = tb <= (size_t)200 << 10 ? 0.3 : tb <= (size_t)32 << 20 ? 0.6 : 4.0;
         if (L.kind >= SJQ_TABLE_HASH_I32 && T->filter && L.filter_bits > 0) {
             // a hashed join is two stages: its presence bitmap (cheap, passes the hits and ~1/16 of the
             // misses) early, the exact probe (expensive) on what is left
@@ -376,6 +381,22 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
             S.op = OP_LOAD;
         }
     }
+    // A filter stage on a direct table with payloads probes the table's presence bitmap (an eighth to a
+    // sixty-fourth of the code array, so far more of it stays in L1/L2); the payload is gathered from the
+    // codes by the sparse copy, for the survivors only.
+    std::vector<char> via_bitmap(ns, 0);
+    if (!opts.no_filter_bitmap) {
+        for (int s = 0; s < ndense; ++s) {
+            DStage &S = P.st[s];
+            if (S.kind != ST_PROBE || S.op < OP_DIRECT_U8 || S.op > OP_DIRECT_U64) continue;
+            const sjq_table *T = joins[specs[order[s]].index].table;
+            if (!T->filter || T->layout.filter_bits <= 0) continue;
+            S.op = OP_DIRECT_BITMAP;
+            S.tab = T->filter;
+            S.tab_bytes = (uint32_t)std::min<size_t>((size_t)(T->layout.filter_bits / 8), 0xFFFFFFF0u);
+            via_bitmap[s] = 1;
+        }
+    }
     // 32-bit fast path of the accumulators: int32 column, multipliers and payload ranges within int32
     for (int s2 = 0; s2 < ns; ++s2) {
         DStage &S = P.st[s2];
@@ -491,7 +512,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
             S.in_smem = 1;
             S.smem_off = (uint32_t)(stage_bytes + tables);
             tables += tb;
-            if (s < ndense && gather_of_stage[s] >= 0) { // the sparse copy reads the same staged table
+            if (s < ndense && gather_of_stage[s] >= 0 && !via_bitmap[s]) { // the sparse copy reads the same staged table
                 P.st[gather_of_stage[s]].in_smem = 1;
                 P.st[gather_of_stage[s]].smem_off = S.smem_off;
             }

@@ -92,7 +92,8 @@ class _RunOpts(ctypes.Structure):
                 ("accumulate", ctypes.c_int32), ("norder", ctypes.c_int32),
                 ("order", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS)), ("event_before", ctypes.c_void_p),
                 ("event_after", ctypes.c_void_p), ("dense_reach_permille", ctypes.c_int32), ("specialise", ctypes.c_int32),
-                ("rows_per_lane", ctypes.c_int32), ("reserved", ctypes.c_int32 * 5)]
+                ("rows_per_lane", ctypes.c_int32), ("no_filter_bitmap", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 4)]
 
 
 class RunInfo(ctypes.Structure):
@@ -123,6 +124,7 @@ class RunOpts:
     dense_reach_permille: int = 0  # experiment knob: level 0 keeps stages reached by more than this share of rows
     specialise: bool = False  # compile the fused kernel for this query's shape at run time (cached per shape)
     rows_per_lane: int = 0  # queue-fed levels: 0 auto, 4, or 8 (8 needs specialise)
+    no_filter_bitmap: bool = False  # filter stages probe the code array of a direct table, not its bitmap
 
     def to_c(self) -> _RunOpts:
         o = _RunOpts()
@@ -135,6 +137,7 @@ class RunOpts:
         o.dense_reach_permille = self.dense_reach_permille
         o.specialise = int(self.specialise)
         o.rows_per_lane = self.rows_per_lane
+        o.no_filter_bitmap = int(self.no_filter_bitmap)
         if self.events is not None:
             o.event_before, o.event_after = self.events[0].cuda_event, self.events[1].cuda_event
         return o

@@ -113,7 +113,9 @@ def test_table_kinds_and_sizes():
     L = tabs["customer"].layout
     # the key range is taken among the rows passing the filter
     assert L.kind_name == "DIRECT_U8" and 2_999_000 <= L.slots <= 3_000_000 and L.code_bits == 8
-    assert L.slots <= L.table_bytes <= 3_000_000 + 1024
+    # byte-packed codes plus the presence bitmap over the same slots (an eighth of a byte per slot)
+    assert L.filter_bits >= L.slots and L.filter_bits % 128 == 0
+    assert L.slots + L.slots // 8 <= L.table_bytes <= 3_000_000 + 375_000 + 1024
     assert tabs["supplier"].layout.kind_name == "DIRECT_BITMAP" and 199_900 <= tabs["supplier"].layout.slots <= 200_000
     assert tabs["part"].layout.kind_name == "DIRECT_BITMAP"
     d = tabs["date"].layout
