@@ -250,8 +250,8 @@ typedef struct sjq_run_opts {
     int32_t ctas_per_sm;   /* 0 = as many as fit */
     int32_t eager_loads;   /* 1 = load every column for every row (ablation of lazy loading) */
     int32_t agg_path;      /* 0 auto, 1 shared-memory privatised table, 2 global atomics (DENSE) */
-    int32_t smem_tables;   /* 0 auto (direct tables up to 16 KiB are copied into shared memory), 1 never,
-                              2 every direct table that fits */
+    int32_t smem_tables;   /* 0 auto (direct tables and presence bitmaps up to 32 KiB are copied into shared
+                              memory), 1 never, 2 every one that fits, >= 1024: size limit in bytes */
     int32_t compaction;    /* 0 auto; 1 never queue survivors (every stage on thread-owned rows);
                               2 one queue only (first stage dense, everything else at the final level) */
     int32_t accumulate;    /* 1 = add into the result buffers instead of clearing them first */

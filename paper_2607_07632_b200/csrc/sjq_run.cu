@@ -505,7 +505,8 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
             const size_t tb = align_up(S.tab_bytes, 16);
             if (tables + tb > table_budget) continue;
             // larger tables are left to L1/L2: shared memory taken here is L1 capacity lost to every other table
-            if (opts.smem_tables == 0 && tb > (size_t)16 << 10) continue;
+            if (opts.smem_tables == 0 && tb > (size_t)32 << 10) continue;
+            if (opts.smem_tables >= 1024 && tb > (size_t)opts.smem_tables) continue; // experiment: size limit in bytes
             // worth it only if a block probes the table more often than it costs to copy
             const double probes_per_cta = (double)n * reach[s] / approx_grid;
             if (probes_per_cta * 4.0 < (double)tb) continue;
