@@ -478,45 +478,61 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     const size_t smem_cap = (size_t)dev.max_smem_optin - 1024; // static reduce scratch + slack
     const size_t stage_bytes = align_up((size_t)ns * sizeof(DStage), 16);
     auto queue_bytes = [&](int threads) { return P.nq ? (size_t)(threads / 32) * (size_t)(kQueue0Cap + (P.nq - 1) * queue_cap_for(P.rows)) * 4 : (size_t)0; };
-    // Two blocks per SM each carry their own group table and queues; when that would take most of the
-    // SM's shared memory (and with it the L1), a kernel compiled for the query runs as one block of 1024
-    // threads per SM instead (config 5, 64 KB group table: 2.8 -> 1.9 ms).
-    bool single_block = false;
-    if (opts.specialise && !opts.block_threads && !opts.ctas_per_sm &&
-        stage_bytes + group_bytes + queue_bytes(block) > ((size_t)80 << 10) &&
-        stage_bytes + group_bytes + queue_bytes(1024) <= smem_cap) {
-        block = 1024;
-        single_block = true;
-    }
-    const size_t fixed = stage_bytes + group_bytes + queue_bytes(block);
-    if (fixed > smem_cap) return SJQ_ERR_UNSUPPORTED;
-    const size_t table_budget = smem_cap - fixed;
-    size_t tables = 0;
-    if (opts.smem_tables != 1) {
-        std::vector<int> cand;
-        for (int s = 0; s < nfilter; ++s)
-            if (P.st[s].op >= OP_DIRECT_BITMAP && P.st[s].op <= OP_DIRECT_U64) cand.push_back(s);
-        // most probes per staged byte first
-        std::stable_sort(cand.begin(), cand.end(), [&](int a, int b) {
-            return reach[a] / (double)P.st[a].tab_bytes > reach[b] / (double)P.st[b].tab_bytes;
-        });
-        for (int s : cand) {
-            DStage &S = P.st[s];
-            const size_t tb = align_up(S.tab_bytes, 16);
-            if (tables + tb > table_budget) continue;
-            // larger tables are left to L1/L2: shared memory taken here is L1 capacity lost to every other table
-            if (opts.smem_tables == 0 && tb > (size_t)32 << 10) continue;
-            if (opts.smem_tables >= 1024 && tb > (size_t)opts.smem_tables) continue; // experiment: size limit in bytes
-            // worth it only if a block probes the table more often than it costs to copy
-            const double probes_per_cta = (double)n * reach[s] / approx_grid;
-            if (probes_per_cta * 4.0 < (double)tb) continue;
-            S.in_smem = 1;
-            S.smem_off = (uint32_t)(stage_bytes + tables);
-            tables += tb;
-            if (s < ndense && gather_of_stage[s] >= 0 && !via_bitmap[s]) { // the sparse copy reads the same staged table
-                P.st[gather_of_stage[s]].in_smem = 1;
-                P.st[gather_of_stage[s]].smem_off = S.smem_off;
+    // Direct tables (and presence bitmaps) worth a copy in shared memory, most probes per staged byte first.
+    auto stage_tables = [&](int threads, size_t *tables_out) -> bool {
+        for (int s2 = 0; s2 < ns; ++s2) P.st[s2].in_smem = 0, P.st[s2].smem_off = 0;
+        const size_t fixed = stage_bytes + group_bytes + queue_bytes(threads);
+        if (fixed > smem_cap) return false;
+        const size_t table_budget = smem_cap - fixed;
+        size_t tables = 0;
+        if (opts.smem_tables != 1) {
+            std::vector<int> cand;
+            for (int s = 0; s < nfilter; ++s)
+                if (P.st[s].op >= OP_DIRECT_BITMAP && P.st[s].op <= OP_DIRECT_U64) cand.push_back(s);
+            std::stable_sort(cand.begin(), cand.end(), [&](int a, int b) {
+                return reach[a] / (double)P.st[a].tab_bytes > reach[b] / (double)P.st[b].tab_bytes;
+            });
+            for (int s : cand) {
+                DStage &S = P.st[s];
+                const size_t tb = align_up(S.tab_bytes, 16);
+                if (tables + tb > table_budget) continue;
+                // larger tables are left to L1/L2: shared memory taken here is L1 capacity lost to every other table
+                if (opts.smem_tables == 0 && tb > (size_t)32 << 10) continue;
+                if (opts.smem_tables >= 1024 && tb > (size_t)opts.smem_tables) continue; // experiment: size limit in bytes
+                // worth it only if a block probes the table more often than it costs to copy
+                const double probes_per_cta = (double)n * reach[s] / approx_grid;
+                if (probes_per_cta * 4.0 < (double)tb) continue;
+                S.in_smem = 1;
+                S.smem_off = (uint32_t)(stage_bytes + tables);
+                tables += tb;
+                if (s < ndense && gather_of_stage[s] >= 0 && !via_bitmap[s]) { // the sparse copy reads the same staged table
+                    P.st[gather_of_stage[s]].in_smem = 1;
+                    P.st[gather_of_stage[s]].smem_off = S.smem_off;
+                }
             }
+        }
+        *tables_out = tables;
+        return true;
+    };
+    size_t tables = 0;
+    if (!stage_tables(block, &tables)) return SJQ_ERR_UNSUPPORTED;
+    // Two blocks per SM each carry their own copies of the staged tables and the group table, and their
+    // queues.  A kernel compiled for the query can run as one block of 1024 threads per SM instead: one
+    // copy, 32 warps instead of 24.  Measured better whenever the copies are sizeable or shared memory
+    // would crowd out the L1 (config 3: 1.43 -> 1.32 ms, config 5: 2.8 -> 1.8 ms), given enough tiles per
+    // block to even out the tail.
+    bool single_block = false;
+    if (opts.specialise && !opts.block_threads && !opts.ctas_per_sm && P.nq) {
+        const size_t copies = tables + group_bytes;
+        const int64_t tiles_per_block = n / ((int64_t)1024 * kDenseRows) / dev.sm_count;
+        size_t tables1024 = 0;
+        if ((copies >= ((size_t)16 << 10) || stage_bytes + copies + queue_bytes(block) > ((size_t)80 << 10)) &&
+            tiles_per_block >= 128 && stage_tables(1024, &tables1024)) {
+            block = 1024;
+            single_block = true;
+            tables = tables1024;
+        } else if (!stage_tables(block, &tables)) {
+            return SJQ_ERR_UNSUPPORTED;
         }
     }
     P.smem_stages = 0;
