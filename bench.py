@@ -31,7 +31,7 @@ CONTRACT_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per fact row of the fused kernel, from an ncu capture of a 100 M-row case of the same workload
 # (dram__bytes_read.sum + dram__bytes_write.sum; traffic grows in proportion to the rows)
-NCU_DRAM_BYTES_PER_ROW = {"c3": 16.8}
+NCU_DRAM_BYTES_PER_ROW = {"c3": 12.5}
 
 
 def measured_hbm_peak():
@@ -74,10 +74,11 @@ def algorithmic_bytes_per_row(w, order):
     sel = stage_selectivities(w)
     names = [f"pred:{p.col}" for p in w.preds] + [f"join:{d}" for _, d in w.joins]
     cols = [p.col for p in w.preds] + [fk for fk, _ in w.joins]
-    reach, total, seen = 1.0, 0.0, set()
+    reach, total, seen, applied = 1.0, 0.0, set(), set()
     for idx in order:
-        if idx < 0:
+        if idx < 0 or idx in applied:  # a repeated label is the gather copy of a filter stage: nothing new is read
             continue
+        applied.add(idx)
         col = cols[idx]
         width = 8 if w.fact_col(col).is64 else 4
         if col not in seen:
@@ -212,6 +213,9 @@ def main():
     ap.add_argument("--cpu-sample-rows", type=int, default=100_000_000)
     ap.add_argument("--interpret", action="store_true",
                     help="interpret the query descriptor instead of compiling the fused kernel for the query's shape")
+    ap.add_argument("--block-threads", type=int, default=0,
+                    help="force the fused kernel's block size (profiling a small case in the full-size launch shape)")
+    ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--extras", action="store_true", help="also time the other configurations (N = 1 only)")
@@ -265,7 +269,8 @@ def main():
     def step(i=None):
         nonlocal launches, info
         tables = sjq.build_tables(builders)
-        opts = sjq.RunOpts(events=pairs[i] if i is not None else None, specialise=not args.interpret)
+        opts = sjq.RunOpts(events=pairs[i] if i is not None else None, specialise=not args.interpret,
+                           block_threads=args.block_threads, ctas_per_sm=args.ctas_per_sm)
         r = sjq.run_workload(w, fact, tables, opts, result=res)
         if world > 1 and w.mode != "HASHED":
             shard.merge_dense(res.sums, res.counts)
