@@ -182,7 +182,8 @@ namespace {
 struct Module {
     cudaLibrary_t lib = nullptr;
     cudaKernel_t kernel = nullptr;
-    int smem_set = -1; // largest dynamic shared memory size the kernel has been opted in for
+    int smem_set[64];  // per device: largest dynamic shared memory size the kernel has been opted in for
+    Module() { for (int &v : smem_set) v = -1; }
     sjq_status status = SJQ_OK;
 };
 
@@ -280,13 +281,15 @@ sjq_status jit_occupancy(const RunParams &P, int agg, bool mul, bool hash, int b
     Module *M = nullptr;
     sjq_status st = module_for(jit_shape_header(P, agg, mul, hash, block, lb_blocks), &M);
     if (st != SJQ_OK) return st;
-    if ((int)smem > M->smem_set) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SJQ_ERR_CUDA;
+    if ((int)smem > M->smem_set[dev]) {
         if (cudaFuncSetAttribute(reinterpret_cast<const void *>(M->kernel), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem) != cudaSuccess) {
             (void)cudaGetLastError();
             return SJQ_ERR_CUDA;
         }
-        M->smem_set = (int)smem;
+        M->smem_set[dev] = (int)smem;
     }
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, reinterpret_cast<const void *>(M->kernel), block,
                                                       smem) != cudaSuccess) {

@@ -101,12 +101,13 @@ def test_more_than_2_pow_32_rows_equals_split_runs():
                dict(mode="DENSE", key=KeyExpr((Term("FACT", "p"),), modulo=7), num_groups=7)):
         agg = AggExpr("COL", Term("FACT", "p"))
         preds = (Pred("p", "LT", 2500),)
-        whole = sjq.run(fact, preds, (), agg=agg, **kw)
         acc = sjq.run(parts[0], preds, (), agg=agg, **kw)
         acc = sjq.run(parts[1], preds, (), agg=agg, opts=sjq.RunOpts(accumulate=True), result=acc, **kw)
-        torch.cuda.synchronize()
-        assert whole.status() == 0 and acc.status() == 0
-        assert torch.equal(whole.sums, acc.sums) and torch.equal(whole.counts, acc.counts)
-        assert int(whole.counts.sum().item()) == int((p < 2500).sum().item())
+        for specialise in (False, True):
+            whole = sjq.run(fact, preds, (), agg=agg, opts=sjq.RunOpts(specialise=specialise), **kw)
+            torch.cuda.synchronize()
+            assert whole.status() == 0 and acc.status() == 0
+            assert torch.equal(whole.sums, acc.sums) and torch.equal(whole.counts, acc.counts)
+            assert int(whole.counts.sum().item()) == int((p < 2500).sum().item())
     del p, fact, parts
     torch.cuda.empty_cache()

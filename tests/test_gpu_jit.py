@@ -130,3 +130,32 @@ def test_compiler_log_is_readable():
     buf = ctypes.create_string_buffer(4096)
     n = L.sjq_jit_log(buf, len(buf))
     assert n >= 0 and len(buf.value) <= 4095
+
+
+@pytest.mark.parametrize("seed", [900, 901, 902])
+def test_largest_query_shape_both_kernels(seed):
+    """Sixteen predicates and eight joins (the limits of the interface), several with two payloads: the
+    interpreted kernel walks about forty stage descriptors, the specialised one unrolls them all."""
+    from dataclasses import replace
+
+    w, fact, hd = random_query(seed, n_fact=600, n_joins=8, allow_dup=False, wide_keys=True)
+    rng = np.random.default_rng(seed)
+    preds = []
+    for i in range(16):
+        col = f"c{i % 3}"
+        kind = i % 4
+        if kind == 0:
+            preds.append(Pred(col, "BETWEEN", -4, int(rng.integers(8, 12))))
+        elif kind == 1:
+            preds.append(Pred(col, "NE", int(rng.integers(-4, 12))))
+        elif kind == 2:
+            preds.append(Pred(col, "GE", int(rng.integers(-4, -1))))
+        else:
+            preds.append(Pred(col, "IN", values=tuple(range(-4, int(rng.integers(6, 12))))))
+    w = replace(w, preds=tuple(preds))
+    dev_fact = to_dev(fact)
+    tables = None
+    for opts in (sjq.RunOpts(), spec(), spec(compaction=1)):
+        res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)
+        assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)
+        compare(w, res, exp)
