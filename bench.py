@@ -279,6 +279,17 @@ def main():
         info = r.info
         return tables
 
+    if not args.interpret:
+        # the first specialised run compiles the kernel; if the compiler is not available on this machine say so
+        # and time the interpreted kernel (still the library's CUDA path) rather than nothing
+        try:
+            step()
+        except sjq.SjqError as ex:
+            if ex.status != 7:
+                raise
+            print(f"bench.py: run-time specialisation unavailable ({ex}); {sjq.jit_log()[:300]!r}; "
+                  "timing the interpreted kernel", file=sys.stderr, flush=True)
+            args.interpret = True
     for _ in range(args.warmup):
         tables = step()
     torch.cuda.synchronize()

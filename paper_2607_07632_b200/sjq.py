@@ -556,6 +556,17 @@ def run_workload_host(w, fact: dict, tables: dict, staging: torch.Tensor, chunk_
                     w.mode, w.num_groups, w.capacity, opts, result, host)
 
 
+def jit_log() -> str:
+    """Compiler output of the most recent run-time compilation of the fused kernel."""
+    L = lib()
+    L.sjq_jit_log.restype = ctypes.c_size_t
+    L.sjq_jit_log.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
+    n = L.sjq_jit_log(None, 0)
+    buf = ctypes.create_string_buffer(int(n) + 1)
+    L.sjq_jit_log(buf, len(buf))
+    return buf.value.decode(errors="replace")
+
+
 def build_launches(table: "Table") -> int:
     """Kernels enqueued by sjq_dim_plan + sjq_build_dim for this table (cudaMemset calls not counted)."""
     direct = table.layout.kind <= 5
