@@ -1,5 +1,8 @@
 // Ahead-of-time instantiations of the fused probe kernel (the query is a descriptor interpreted at
 // run time), result housekeeping kernels and the launch helpers used by the planner.
+#include <mutex>
+#include <unordered_map>
+
 #include "sjq_fused_device.cuh"
 
 namespace sjq {
@@ -87,14 +90,38 @@ fused_fn pick_kernel(int agg, bool mul, bool hash)
 
 // ---- launch helpers used by the planner (sjq_run.cu) ----------------------
 
+// Shared-memory opt-in and occupancy of a kernel variant; both answers are remembered per device, so a
+// repeated query costs two map look-ups instead of two runtime calls.
 sjq_status fused_occupancy(int agg, bool mul, bool hash, int block, size_t smem, int *ctas_per_sm)
 {
+    static std::mutex mutex;
+    static std::unordered_map<uint64_t, int> occupancy; // (device, variant, block, smem) -> blocks per SM
+    static std::unordered_map<uint32_t, int> opted;     // (device, variant) -> largest smem opted in for
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SJQ_ERR_CUDA;
+    const uint32_t variant = (uint32_t)(agg * 4 + (mul ? 2 : 0) + (hash ? 1 : 0));
+    const uint32_t fkey = (uint32_t)dev * 64u + variant;
+    const uint64_t okey = ((uint64_t)fkey << 40) | ((uint64_t)block << 24) | (uint64_t)(smem & 0xFFFFFF);
+    std::lock_guard<std::mutex> lock(mutex);
     fused_fn fn = pick_kernel(agg, mul, hash);
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, fn, block, smem) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return SJQ_ERR_CUDA;
+    auto o = opted.find(fkey);
+    if (o == opted.end() || o->second < (int)smem) {
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return SJQ_ERR_CUDA;
+        }
+        opted[fkey] = (int)smem;
     }
+    auto it = occupancy.find(okey);
+    if (it == occupancy.end()) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fn, block, smem) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return SJQ_ERR_CUDA;
+        }
+        it = occupancy.emplace(okey, n).first;
+    }
+    *ctas_per_sm = it->second;
     return SJQ_OK;
 }
 

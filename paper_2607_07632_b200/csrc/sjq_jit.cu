@@ -179,10 +179,36 @@ std::string jit_shape_header(const RunParams &P, int agg, bool mul, bool hash, i
 
 namespace {
 
+// Everything jit_shape_header prints, as bytes: cheap to build on every run; the text itself is only
+// generated when the key is new.
+std::string shape_key(const RunParams &P, int agg, bool mul, bool hash, int lb_threads, int lb_blocks)
+{
+    std::string k;
+    k.reserve(64 + (size_t)P.nstages * 128);
+    auto put_raw = [&](const void *p, size_t n) { k.append(static_cast<const char *>(p), n); };
+    const int32_t head[] = {agg, mul ? 1 : 0, hash ? 1 : 0, lb_threads, lb_blocks, P.nstages, P.nd0, P.nq,
+                            P.rows, P.want_count, P.eager, P.has_key, P.mod32};
+    put_raw(head, sizeof(head));
+    put_raw(&P.modulo, sizeof(P.modulo));
+    put_raw(&P.modmask, sizeof(P.modmask));
+    for (int s = 0; s < P.nstages; ++s) {
+        const DStage &S = P.st[s];
+        const uint8_t b[] = {S.op, S.is64, S.neg, S.never, S.nset, S.set_idx, S.in_smem, S.kind, S.simple, S.code_bits};
+        put_raw(b, sizeof(b));
+        put_raw(&S.acc, sizeof(S.acc));
+        put_raw(&S.acc32, sizeof(S.acc32));
+        put_raw(S.mult, sizeof(S.mult));
+        put_raw(S.mult32, sizeof(S.mult32));
+    }
+    if (const char *extra = std::getenv("SJQ_JIT_EXTRA")) k += extra;
+    return k;
+}
+
 struct Module {
     cudaLibrary_t lib = nullptr;
     cudaKernel_t kernel = nullptr;
     int smem_set[64];  // per device: largest dynamic shared memory size the kernel has been opted in for
+    std::unordered_map<uint64_t, int> occupancy; // (device, block, smem) -> blocks per SM
     Module() { for (int &v : smem_set) v = -1; }
     sjq_status status = SJQ_OK;
 };
@@ -248,10 +274,12 @@ sjq_status compile(const std::string &shape, std::vector<char> *cubin, std::stri
 }
 
 // Find or build the module of a shape.  Called with g_mutex held.
-sjq_status module_for(const std::string &shape, Module **out)
+sjq_status module_for(const RunParams &P, int agg, bool mul, bool hash, int lb_threads, int lb_blocks, Module **out)
 {
-    auto it = g_modules.find(shape);
+    const std::string key = shape_key(P, agg, mul, hash, lb_threads, lb_blocks);
+    auto it = g_modules.find(key);
     if (it == g_modules.end()) {
+        const std::string shape = jit_shape_header(P, agg, mul, hash, lb_threads, lb_blocks);
         Module M;
         std::vector<char> cubin;
         std::string log;
@@ -266,7 +294,7 @@ sjq_status module_for(const std::string &shape, Module **out)
                 M.status = SJQ_ERR_JIT;
             }
         }
-        it = g_modules.emplace(shape, M).first;
+        it = g_modules.emplace(key, M).first;
     }
     *out = &it->second;
     return it->second.status;
@@ -279,7 +307,7 @@ sjq_status jit_occupancy(const RunParams &P, int agg, bool mul, bool hash, int b
 {
     std::lock_guard<std::mutex> lock(g_mutex);
     Module *M = nullptr;
-    sjq_status st = module_for(jit_shape_header(P, agg, mul, hash, block, lb_blocks), &M);
+    sjq_status st = module_for(P, agg, mul, hash, block, lb_blocks, &M);
     if (st != SJQ_OK) return st;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SJQ_ERR_CUDA;
@@ -291,11 +319,18 @@ sjq_status jit_occupancy(const RunParams &P, int agg, bool mul, bool hash, int b
         }
         M->smem_set[dev] = (int)smem;
     }
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, reinterpret_cast<const void *>(M->kernel), block,
-                                                      smem) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return SJQ_ERR_CUDA;
+    const uint64_t okey = ((uint64_t)dev << 48) | ((uint64_t)block << 24) | (uint64_t)(smem & 0xFFFFFF);
+    auto o = M->occupancy.find(okey);
+    if (o == M->occupancy.end()) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, reinterpret_cast<const void *>(M->kernel), block, smem) !=
+            cudaSuccess) {
+            (void)cudaGetLastError();
+            return SJQ_ERR_CUDA;
+        }
+        o = M->occupancy.emplace(okey, n).first;
     }
+    *ctas_per_sm = o->second;
     return SJQ_OK;
 }
 
@@ -306,7 +341,7 @@ sjq_status jit_launch(const RunParams &P, int agg, bool mul, bool hash, int grid
     {
         std::lock_guard<std::mutex> lock(g_mutex);
         Module *M = nullptr;
-        sjq_status st = module_for(jit_shape_header(P, agg, mul, hash, block, lb_blocks), &M);
+        sjq_status st = module_for(P, agg, mul, hash, block, lb_blocks, &M);
         if (st != SJQ_OK) return st;
         kernel = M->kernel;
     }

@@ -296,7 +296,12 @@ class TableBuilder:
             self.stats = torch.zeros(8, dtype=torch.int64, pin_memory=True)
             self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
             self.side = torch.cuda.Stream(self.device)
-            self.mem = None
+            # two table buffers used in turn: the build of the next table does not have to wait for the run
+            # that still reads the previous one
+            self.mems = [None, None]
+            self.turn = 0
+            self.guards = [torch.cuda.Event(), torch.cuda.Event()]
+            self.guard_set = [False, False]
             self.layout = DimLayout()
 
     def begin(self):
@@ -315,19 +320,30 @@ class TableBuilder:
                                     self.stats.data_ptr(), ctypes.byref(self.layout))
         if rc != 0:
             raise SjqError(rc, "sjq_dim_plan_end")
-        if self.mem is None or self.mem.numel() < self.layout.table_bytes:
+        i = self.turn
+        self.turn ^= 1
+        main = torch.cuda.current_stream(self.device)
+        if self.mems[i] is None or self.mems[i].numel() < self.layout.table_bytes:
             with torch.cuda.device(self.device):
-                self.mem = torch.empty(self.layout.table_bytes, dtype=torch.uint8, device=self.device)
-        # the build overwrites the table memory: it must follow whatever the current stream still runs on it
-        self.side.wait_stream(torch.cuda.current_stream(self.device))
+                self.mems[i] = torch.empty(self.layout.table_bytes, dtype=torch.uint8, device=self.device)
+            self.side.wait_stream(main)
+        # The build overwrites buffer i, which the table returned two calls ago lives in: it must follow
+        # whatever the current stream had queued by the time of the previous call (the runs on that table),
+        # not the runs on the previous table, which read the other buffer.  A table is therefore valid for
+        # work enqueued on the current stream before the next call of finish().
+        if self.guard_set[i]:
+            self.side.wait_event(self.guards[i])
+        self.guards[i ^ 1].record(main)
+        self.guard_set[i ^ 1] = True
+        mem = self.mems[i]
         handle = ctypes.c_void_p()
         rc = lib().sjq_build_dim(self.carr, len(self.names), self.parr, self.npreds, self.key_col, self.pay,
-                                 self.npay, ctypes.byref(self.layout), self.mem.data_ptr(), self.mem.numel(),
+                                 self.npay, ctypes.byref(self.layout), mem.data_ptr(), mem.numel(),
                                  self.status.data_ptr(), self.side.cuda_stream, ctypes.byref(handle))
         if rc != 0:
             raise SjqError(rc, "sjq_build_dim")
         layout = DimLayout.from_buffer_copy(self.layout)
-        return Table(handle.value, layout, self.mem, self.status)
+        return Table(handle.value, layout, mem, self.status)
 
 
 def workload_builders(w, dims: dict) -> dict:
