@@ -350,7 +350,7 @@ def main():
                 torch.cuda.synchronize()  # the result is on the host when this returns
                 return tabs
 
-            e2e_step()
+            tabs = e2e_step()
             if world > 1:
                 dist.barrier()
             t0 = time.perf_counter()
@@ -363,10 +363,21 @@ def main():
             dt = float(tt[0])
             same = bool(torch.equal(ehost.sums, res.sums.cpu())) if world == 1 else None
             cells = 1 if w.mode == "SCALAR" else w.num_groups if w.mode == "DENSE" else w.capacity
-            e2e = {"value": world * n / dt, "unit": UNIT, "h2d_bytes_per_step": n * ref_bytes,
+            # bytes over the bus: whole columns for the copied ones; for a column the kernel reads in place, the
+            # 32-byte sectors holding a surviving row (estimated from the planner's share of rows reaching it)
+            plan = sjq.host_transfer_plan({c.name: host_fact[c.name] for c in w.fact_cols}, w.preds,
+                                          [(fk, tabs[dn]) for fk, dn in w.joins], w.key, w.agg,
+                                          sjq.RunOpts(specialise=not args.interpret))
+            copied = sum(n * host_fact[k].element_size() for k, (how, _) in plan.items() if how == "copy")
+            in_place = sum(n * host_fact[k].element_size() * (1.0 - (1.0 - sh) ** (32 // host_fact[k].element_size()))
+                           for k, (how, sh) in plan.items() if how == "in place")
+            e2e = {"value": world * n / dt, "unit": UNIT, "h2d_bytes_per_step": int(copied + in_place),
+                   "h2d_copied_bytes": int(copied), "h2d_in_place_bytes_estimate": int(in_place),
+                   "columns": {k: how for k, (how, _) in plan.items()},
                    "d2h_bytes_per_step": cells * 8 * (2 if w.agg.want_count else 1) + 4, "ms_per_step": dt * 1000.0,
                    "steps": args.e2e_steps, "chunk_rows": chunk, "matches_device_run": same,
-                   "api": "sjq_run_host (pinned host columns, chunked double-buffered copies, result copied back)"}
+                   "api": "sjq_run_host (pinned host columns: chunked double-buffered copies of the columns most rows need, "
+                          "in-place reads of the sparse ones, result copied back)"}
             del host_fact, staging
         except Exception as ex:  # e.g. not enough page-locked memory on the box
             e2e = {"value": None, "unit": UNIT, "error": repr(ex)[:200]}

@@ -269,7 +269,10 @@ typedef struct sjq_run_opts {
                               (8 only with specialise: the ahead-of-time kernels are built for 4) */
     int32_t no_filter_bitmap; /* 1 = filter stages probe a direct table's code array even when the table has a
                                  presence bitmap (ablation) */
-    int32_t reserved[4];
+    int32_t host_copy_all; /* sjq_run_host: 1 = copy every referenced column to the device; 0 = columns that only a
+                              few per cent of the rows reach are read by the kernel from the page-locked host
+                              buffer instead */
+    int32_t reserved[3];
 } sjq_run_opts;
 
 /* What the planner decided for a run (for reports and tests). */
@@ -325,9 +328,15 @@ sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *preds, int np
  *                 host destinations (page-locked for an asynchronous copy) of
  *                 the arrays of `out`; NULL = do not copy that one.  HASHED
  *                 results copy `capacity` entries.
- * Every column is copied whole: lazy loading cannot skip bytes that have to
- * cross the bus before the predicates are known.  Enqueues only; the caller
- * synchronises `stream`.  Errors as sjq_run, plus BUFFER_SMALL.
+ * A column that most rows still need when it is first read is copied whole.
+ * A column that at most a few per cent of the rows reach (by the planner's
+ * estimate) is not copied when its buffer is page-locked: the kernel reads it
+ * in place over the bus, for the surviving rows only, which moves far fewer
+ * bytes (opts->host_copy_all = 1 copies it all the same; a pageable buffer is
+ * always copied).  A column the query does not reference is not transferred.
+ * The host buffers must stay valid and unchanged until `stream` has finished.
+ * Enqueues only; the caller synchronises `stream`.  Errors as sjq_run, plus
+ * BUFFER_SMALL.
  */
 sjq_status sjq_run_host(const sjq_col *fact_host, int nfact, const sjq_pred *preds, int npreds,
                         const sjq_join *joins, int njoins, const sjq_key_expr *key, const sjq_agg_expr *agg,
@@ -335,6 +344,17 @@ sjq_status sjq_run_host(const sjq_col *fact_host, int nfact, const sjq_pred *pre
                         void *staging_dev, size_t staging_bytes, int64_t chunk_rows, int64_t *host_sums,
                         int64_t *host_counts, int64_t *host_keys, int64_t *host_n_groups, int32_t *host_status,
                         void *stream);
+
+/*
+ * What sjq_run_host would do with each column of `fact_host` for this query:
+ * how[c] = 0 copied chunk by chunk, 1 read in place from the page-locked host
+ * buffer by the kernel, 2 not transferred (the query does not reference it);
+ * share[c] (optional) = estimated share of the rows the column is first read
+ * for.  Enqueues nothing.
+ */
+sjq_status sjq_host_transfer_plan(const sjq_col *fact_host, int nfact, const sjq_pred *preds, int npreds,
+                                  const sjq_join *joins, int njoins, const sjq_key_expr *key,
+                                  const sjq_agg_expr *agg, const sjq_run_opts *opts, int32_t *how, double *share);
 
 /*
  * Hashed group-by without any workspace from the caller.  (The paper has no

@@ -76,6 +76,69 @@ bool valid_term(const sjq_term &t, int nfact, const sjq_join *joins, int njoins)
     return false;
 }
 
+// The filter stages of a query (its predicates and joins; a hashed join with a presence bitmap is two
+// stages) with estimated selectivities and relative costs, and the order they are evaluated in: the
+// caller's, or by rank (1 - selectivity) / cost.
+sjq_status order_stages(const sjq_col *fact, const sjq_pred *preds, int npreds, const sjq_join *joins, int njoins,
+                        const sjq_run_opts &opts, std::vector<StageSpec> *specs_out, std::vector<int> *order_out)
+{
+    std::vector<StageSpec> &specs = *specs_out;
+    std::vector<int> &order = *order_out;
+    for (int p = 0; p < npreds; ++p) {
+        const double bytes = fact[preds[p].col].dtype == SJQ_I64 ? 2.0 : 1.0;
+        specs.push_back({ST_PRED, p, preds[p].col, pred_selectivity(preds[p]), bytes, 0});
+    }
+    for (int j = 0; j < njoins; ++j) {
+        const sjq_table *T = joins[j].table;
+        const sjq_dim_layout &L = T->layout;
+        const double bytes = L.key_dtype == SJQ_I64 ? 2.0 : 1.0;
+        double sel = L.dim_rows > 0 ? (double)L.entries / (double)L.dim_rows : 0.0;
+        // bytes a filter stage on this table touches: the presence bitmap when a direct table has one
+        const size_t tb = (L.kind <= SJQ_TABLE_DIRECT_U64 && L.filter_bits > 0 && T->filter && !opts.no_filter_bitmap)
+                              ? (size_t)(L.filter_bits / 8)
+                              : L.table_bytes;
+        // relative cost of one probe: a table the L1 mostly holds, one the L2 holds (measured on the four-join
+        // workload: the 3 MB map before the 175 KB bitmap when it drops twice as many rows), one in HBM
+        double probe = tb <= (size_t)200 << 10 ? 0.3 : tb <= (size_t)32 << 20 ? 0.6 : 4.0;
+        if (L.kind >= SJQ_TABLE_HASH_I32 && T->filter && L.filter_bits > 0) {
+            // a hashed join is two stages: its presence bitmap (cheap, passes the hits and ~1/16 of the
+            // misses) early, the exact probe (expensive) on what is left
+            const double fp = std::min(1.0, (double)L.entries / (double)L.filter_bits);
+            const double pass = std::min(1.0, sel + (1.0 - sel) * fp);
+            specs.push_back({ST_PROBE, j, joins[j].fk_col, pass, bytes + 0.7, 1});
+            specs.push_back({ST_PROBE, j, joins[j].fk_col, pass > 0 ? std::min(1.0, sel / pass) : 1.0,
+                             bytes + probe + 4.0, 2});
+            continue;
+        }
+        specs.push_back({ST_PROBE, j, joins[j].fk_col, std::min(1.0, sel), bytes + probe, 0});
+    }
+    const int nfilter = (int)specs.size();
+    if (opts.norder) {
+        // the caller orders predicates and joins; a hashed join's bitmap and exact probe stay adjacent
+        std::vector<char> seen(npreds + njoins, 0);
+        for (int i = 0; i < npreds + njoins; ++i) {
+            const int o = opts.order[i];
+            if (o < 0 || o >= npreds + njoins || seen[o]) return SJQ_ERR_INVALID_ARG;
+            seen[o] = 1;
+            for (int k = 0; k < nfilter; ++k) {
+                const bool match = o < npreds ? (specs[k].kind == ST_PRED && specs[k].index == o)
+                                              : (specs[k].kind == ST_PROBE && specs[k].index == o - npreds);
+                if (match) order.push_back(k);
+            }
+        }
+    } else {
+        order.resize(nfilter);
+        for (int i = 0; i < nfilter; ++i) order[i] = i;
+        std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+            // exact probes of prefiltered hashed joins go last: they run at the final level
+            if ((specs[a].prefilter == 2) != (specs[b].prefilter == 2)) return specs[b].prefilter == 2;
+            return (1.0 - specs[a].sel) / specs[a].cost > (1.0 - specs[b].sel) / specs[b].cost;
+        });
+    }
+
+    return SJQ_OK;
+}
+
 } // namespace
 } // namespace sjq
 
@@ -154,58 +217,9 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
 
     // ------------------------------------------------------------ stage list
     std::vector<StageSpec> specs;
-    for (int p = 0; p < npreds; ++p) {
-        const double bytes = fact[preds[p].col].dtype == SJQ_I64 ? 2.0 : 1.0;
-        specs.push_back({ST_PRED, p, preds[p].col, pred_selectivity(preds[p]), bytes, 0});
-    }
-    for (int j = 0; j < njoins; ++j) {
-        const sjq_table *T = joins[j].table;
-        const sjq_dim_layout &L = T->layout;
-        const double bytes = L.key_dtype == SJQ_I64 ? 2.0 : 1.0;
-        double sel = L.dim_rows > 0 ? (double)L.entries / (double)L.dim_rows : 0.0;
-        // bytes a filter stage on this table touches: the presence bitmap when a direct table has one
-        const size_t tb = (L.kind <= SJQ_TABLE_DIRECT_U64 && L.filter_bits > 0 && T->filter && !opts.no_filter_bitmap)
-                              ? (size_t)(L.filter_bits / 8)
-                              : L.table_bytes;
-        // relative cost of one probe: a table the L1 mostly holds, one the L2 holds (measured on the four-join
-        // workload: the 3 MB map before the 175 KB bitmap when it drops twice as many rows), one in HBM
-        double probe = tb <= (size_t)200 << 10 ? 0.3 : tb <= (size_t)32 << 20 ? 0.6 : 4.0;
-        if (L.kind >= SJQ_TABLE_HASH_I32 && T->filter && L.filter_bits > 0) {
-            // a hashed join is two stages: its presence bitmap (cheap, passes the hits and ~1/16 of the
-            // misses) early, the exact probe (expensive) on what is left
-            const double fp = std::min(1.0, (double)L.entries / (double)L.filter_bits);
-            const double pass = std::min(1.0, sel + (1.0 - sel) * fp);
-            specs.push_back({ST_PROBE, j, joins[j].fk_col, pass, bytes + 0.7, 1});
-            specs.push_back({ST_PROBE, j, joins[j].fk_col, pass > 0 ? std::min(1.0, sel / pass) : 1.0,
-                             bytes + probe + 4.0, 2});
-            continue;
-        }
-        specs.push_back({ST_PROBE, j, joins[j].fk_col, std::min(1.0, sel), bytes + probe, 0});
-    }
-    const int nfilter = (int)specs.size();
     std::vector<int> order;
-    if (opts.norder) {
-        // the caller orders predicates and joins; a hashed join's bitmap and exact probe stay adjacent
-        std::vector<char> seen(npreds + njoins, 0);
-        for (int i = 0; i < npreds + njoins; ++i) {
-            const int o = opts.order[i];
-            if (o < 0 || o >= npreds + njoins || seen[o]) return SJQ_ERR_INVALID_ARG;
-            seen[o] = 1;
-            for (int k = 0; k < nfilter; ++k) {
-                const bool match = o < npreds ? (specs[k].kind == ST_PRED && specs[k].index == o)
-                                              : (specs[k].kind == ST_PROBE && specs[k].index == o - npreds);
-                if (match) order.push_back(k);
-            }
-        }
-    } else {
-        order.resize(nfilter);
-        for (int i = 0; i < nfilter; ++i) order[i] = i;
-        std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
-            // exact probes of prefiltered hashed joins go last: they run at the final level
-            if ((specs[a].prefilter == 2) != (specs[b].prefilter == 2)) return specs[b].prefilter == 2;
-            return (1.0 - specs[a].sel) / specs[a].cost > (1.0 - specs[b].sel) / specs[b].cost;
-        });
-    }
+    if ((st = order_stages(fact, preds, npreds, joins, njoins, opts, &specs, &order)) != SJQ_OK) return st;
+    const int nfilter = (int)specs.size();
 
     // ------------------------------------------------------------ accumulators
     // Every term adds mult * value to one accumulator; fold the expressions
@@ -547,7 +561,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     int per_sm = 0;
     const bool jit = opts.specialise != 0;
     // register budget a specialised kernel is compiled for
-    const int lb_blocks = single_block ? 1 : opts.ctas_per_sm > 0 ? opts.ctas_per_sm : 2;
+    const int lb_blocks = single_block ? 1 : opts.ctas_per_sm > 0 ? opts.ctas_per_sm : block > 512 ? 1 : 2;
     st = jit ? jit_occupancy(P, aggp, mul, has_hash, block, lb_blocks, smem, &per_sm)
              : fused_occupancy(aggp, mul, has_hash, block, smem, &per_sm);
     if (st != SJQ_OK) return st;
@@ -640,6 +654,93 @@ HostPipe *host_pipe()
 
 } // namespace
 
+namespace {
+
+enum { HOST_COPY = 0, HOST_IN_PLACE = 1, HOST_SKIP = 2 };
+
+// How each host-resident column reaches the kernel.  A column most rows still need is copied chunk by
+// chunk; one that only a few per cent of the rows reach (lazy loading: it is read for survivors only) is
+// read by the kernel straight from the page-locked host buffer, 32 bytes per touched sector, which moves
+// far fewer bytes over the bus than the whole column (measured on the four-join workload, 600 M rows:
+// revenue and supplycost 16 ms instead of 87 ms of copies; break-even near 5 % of the rows); a column the
+// query never references is not transferred at all.  `need`: share of the rows each column is first read
+// for (< 0: never).  Invalid queries get "copy everything" and are rejected later by sjq_run.
+void host_transfer_plan(const sjq_col *fact_host, int nfact, const sjq_pred *preds, int npreds,
+                        const sjq_join *joins, int njoins, const sjq_key_expr *key, const sjq_agg_expr *agg,
+                        const sjq_run_opts &opts, std::vector<int> *how_out, std::vector<const char *> *base_out,
+                        std::vector<double> *need_out)
+{
+    std::vector<int> &how = *how_out;
+    std::vector<const char *> &direct_base = *base_out;
+    how.assign(nfact, HOST_COPY);
+    direct_base.assign(nfact, nullptr);
+    need_out->assign(nfact, 1.0);
+    const int64_t n = fact_host[0].n;
+    bool ok = npreds >= 0 && npreds <= SJQ_MAX_PREDS && njoins >= 0 && njoins <= SJQ_MAX_JOINS &&
+              (!npreds || preds) && (!njoins || joins) && n > 0 && agg;
+    for (int p = 0; ok && p < npreds; ++p) ok = preds[p].col >= 0 && preds[p].col < nfact;
+    for (int j = 0; ok && j < njoins; ++j)
+        ok = joins[j].table && joins[j].table->magic == kTableMagic && joins[j].fk_col >= 0 && joins[j].fk_col < nfact;
+    auto term_ok = [&](const sjq_term &t) { return t.src != SJQ_SRC_FACT || (t.a >= 0 && t.a < nfact); };
+    if (ok && key) {
+        ok = key->nterms >= 0 && key->nterms <= SJQ_MAX_KEY_TERMS;
+        for (int t = 0; ok && t < key->nterms; ++t) ok = term_ok(key->t[t]);
+    }
+    ok = ok && term_ok(agg->x) && (agg->op == SJQ_AGG_COL || term_ok(agg->y));
+    std::vector<StageSpec> specs;
+    std::vector<int> order;
+    if (!ok || order_stages(fact_host, preds, npreds, joins, njoins, opts, &specs, &order) != SJQ_OK) return;
+    std::vector<double> &need = *need_out;
+    need.assign(nfact, -1.0);
+    double reach = 1.0;
+    for (int i : order) {
+        if (need[specs[i].col] < 0) need[specs[i].col] = reach;
+        reach *= specs[i].sel;
+    }
+    auto use = [&](const sjq_term &t) {
+        if (t.src == SJQ_SRC_FACT && need[t.a] < 0) need[t.a] = reach;
+    };
+    if (key)
+        for (int t = 0; t < key->nterms; ++t) use(key->t[t]);
+    use(agg->x);
+    if (agg->op != SJQ_AGG_COL) use(agg->y);
+    for (int c = 0; c < nfact; ++c) {
+        if (need[c] < 0) {
+            how[c] = HOST_SKIP;
+        } else if (need[c] <= 0.04 && !opts.eager_loads && !opts.host_copy_all) {
+            cudaPointerAttributes attr;
+            if (cudaPointerGetAttributes(&attr, fact_host[c].data) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
+                attr.devicePointer && aligned16(attr.devicePointer)) {
+                how[c] = HOST_IN_PLACE;
+                direct_base[c] = static_cast<const char *>(attr.devicePointer);
+            } else {
+                (void)cudaGetLastError(); // pageable memory: copy it
+            }
+        }
+    }
+}
+
+} // namespace
+
+extern "C" sjq_status sjq_host_transfer_plan(const sjq_col *fact_host, int nfact, const sjq_pred *preds, int npreds,
+                                             const sjq_join *joins, int njoins, const sjq_key_expr *key,
+                                             const sjq_agg_expr *agg, const sjq_run_opts *opts_, int32_t *how,
+                                             double *share)
+{
+    if (!fact_host || nfact <= 0 || nfact > 64 || !agg || !how) return SJQ_ERR_INVALID_ARG;
+    sjq_run_opts opts{};
+    if (opts_) opts = *opts_;
+    std::vector<int> h;
+    std::vector<const char *> base;
+    std::vector<double> need;
+    host_transfer_plan(fact_host, nfact, preds, npreds, joins, njoins, key, agg, opts, &h, &base, &need);
+    for (int c = 0; c < nfact; ++c) {
+        how[c] = h[c];
+        if (share) share[c] = need[c] < 0 ? 0.0 : need[c];
+    }
+    return SJQ_OK;
+}
+
 extern "C" sjq_status sjq_run_host(const sjq_col *fact_host, int nfact, const sjq_pred *preds, int npreds,
                                    const sjq_join *joins, int njoins, const sjq_key_expr *key,
                                    const sjq_agg_expr *agg, const sjq_result_spec *spec, const sjq_result *out,
@@ -670,6 +771,11 @@ extern "C" sjq_status sjq_run_host(const sjq_col *fact_host, int nfact, const sj
     if (opts_) opts = *opts_;
     opts.event_before = opts.event_after = nullptr;
 
+    std::vector<int> how;
+    std::vector<const char *> direct_base;
+    std::vector<double> need_share;
+    host_transfer_plan(fact_host, nfact, preds, npreds, joins, njoins, key, agg, opts, &how, &direct_base, &need_share);
+
     // internal streams start after whatever is already queued on the caller's stream
     if (cudaEventRecord(hp->start, stream) != cudaSuccess) return SJQ_ERR_CUDA;
     for (int b = 0; b < 2; ++b)
@@ -686,6 +792,11 @@ extern "C" sjq_status sjq_run_host(const sjq_col *fact_host, int nfact, const sj
         for (int c = 0; c < nfact; ++c) {
             const size_t w = fact_host[c].dtype == SJQ_I64 ? 8 : 4;
             dev_cols[c] = sjq_col{base + col_off[c], fact_host[c].dtype, rows};
+            if (how[c] == HOST_SKIP) continue; // never dereferenced
+            if (how[c] == HOST_IN_PLACE) {
+                dev_cols[c].data = direct_base[c] + (size_t)r0 * w;
+                continue;
+            }
             if (rows > 0 &&
                 cudaMemcpyAsync(base + col_off[c], static_cast<const char *>(fact_host[c].data) + (size_t)r0 * w,
                                 (size_t)rows * w, cudaMemcpyHostToDevice, hp->s[b]) != cudaSuccess)

@@ -93,7 +93,7 @@ class _RunOpts(ctypes.Structure):
                 ("order", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS)), ("event_before", ctypes.c_void_p),
                 ("event_after", ctypes.c_void_p), ("dense_reach_permille", ctypes.c_int32), ("specialise", ctypes.c_int32),
                 ("rows_per_lane", ctypes.c_int32), ("no_filter_bitmap", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 4)]
+                ("host_copy_all", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3)]
 
 
 class RunInfo(ctypes.Structure):
@@ -125,6 +125,7 @@ class RunOpts:
     specialise: bool = False  # compile the fused kernel for this query's shape at run time (cached per shape)
     rows_per_lane: int = 0  # queue-fed levels: 0 auto, 4, or 8 (8 needs specialise)
     no_filter_bitmap: bool = False  # filter stages probe the code array of a direct table, not its bitmap
+    host_copy_all: bool = False  # run_host: copy every referenced column instead of reading sparse ones in place
 
     def to_c(self) -> _RunOpts:
         o = _RunOpts()
@@ -138,6 +139,7 @@ class RunOpts:
         o.specialise = int(self.specialise)
         o.rows_per_lane = self.rows_per_lane
         o.no_filter_bitmap = int(self.no_filter_bitmap)
+        o.host_copy_all = int(self.host_copy_all)
         if self.events is not None:
             o.event_before, o.event_after = self.events[0].cuda_event, self.events[1].cuda_event
         return o
@@ -509,6 +511,39 @@ def staging_bytes(fact: dict, chunk_rows: int) -> int:
     for t in fact.values():
         per += (chunk_rows * t.element_size() + 255) // 256 * 256
     return 2 * per
+
+
+def host_transfer_plan(fact: dict, preds=(), joins=(), key=None, agg=None, opts: Optional[RunOpts] = None) -> dict:
+    """sjq_host_transfer_plan: for each host column, ("copy" | "in place" | "not transferred", estimated
+    share of the rows it is first read for) as run_host would treat it."""
+    names = list(fact.keys())
+    tensors = [fact[n] for n in names]
+    carr = (_Col * len(tensors))()
+    for i, t in enumerate(tensors):
+        carr[i] = _Col(t.data_ptr(), 1 if t.dtype == torch.int64 else 0, t.numel())
+    parr, keep = _preds(preds, names)
+    jarr = (_Join * max(1, len(joins)))()
+    for j, (fk, table) in enumerate(joins):
+        jarr[j] = _Join(names.index(fk), table.handle)
+    kexpr = None
+    if key is not None:
+        kexpr = _KeyExpr()
+        for i, t in enumerate(key.terms):
+            kexpr.t[i] = _term(t, names)
+        kexpr.nterms, kexpr.offset, kexpr.modulo = len(key.terms), key.offset, key.modulo
+    aexpr = _AggExpr(AGGS[agg.op], _term(agg.x, names), _term(agg.y, names), int(agg.want_count))
+    copts = (opts or RunOpts()).to_c()
+    how = (ctypes.c_int32 * len(names))()
+    share = (ctypes.c_double * len(names))()
+    L = lib()
+    L.sjq_host_transfer_plan.restype = ctypes.c_int32
+    rc = L.sjq_host_transfer_plan(carr, len(names), parr, len(preds), jarr, len(joins),
+                                  ctypes.byref(kexpr) if kexpr is not None else None, ctypes.byref(aexpr),
+                                  ctypes.byref(copts), how, share)
+    if rc != 0:
+        raise SjqError(rc, "sjq_host_transfer_plan")
+    label = ("copy", "in place", "not transferred")
+    return {n: (label[how[i]], share[i]) for i, n in enumerate(names)}
 
 
 def run_host(fact: dict, staging: torch.Tensor, chunk_rows: int, preds=(), joins=(), key=None, agg=None,

@@ -313,3 +313,33 @@ def test_city_pair_shape_many_groups_few_survivors():
     res, exp, _ = run_both(wh, fact, hd, tables=tables)
     assert res.status() == 0
     compare(wh, res, exp)
+
+
+def test_host_path_reads_sparse_columns_in_place_and_matches_copies():
+    """sjq_run_host leaves a column that few rows reach in page-locked host memory and lets the kernel read
+    it there; copying everything (host_copy_all), pageable buffers (always copied) and the device-resident
+    run must all give the oracle's bits.  The transfer plan names what happens to each column."""
+    w = W.config3(700_003)
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    exp = oracle.run(w, fact, oracle.build_dims(w, hd))
+    tables = sjq.build_workload_tables(w, {k: to_dev(v) for k, v in hd.items()})
+    pinned = {k: torch.from_numpy(np.ascontiguousarray(v)).pin_memory() for k, v in fact.items()}
+    pinned["unused"] = torch.zeros(w.n_rows, dtype=torch.int32).pin_memory()  # not referenced by the query
+    pageable = {k: torch.from_numpy(np.ascontiguousarray(v)) for k, v in fact.items()}
+    joins = [(fk, tables[dn]) for fk, dn in w.joins]
+    plan = sjq.host_transfer_plan(pinned, w.preds, joins, w.key, w.agg)
+    assert plan["suppkey"][0] == "copy" and plan["orderdate"][0] == "copy"
+    assert plan["revenue"][0] == "in place" and plan["supplycost"][0] == "in place"
+    assert plan["unused"] == ("not transferred", 0.0)
+    assert all(how == "copy" or name == "unused" for name, (how, _) in
+               sjq.host_transfer_plan(pinned, w.preds, joins, w.key, w.agg, sjq.RunOpts(host_copy_all=True)).items())
+    chunk = 131072
+    for cols, opts in ((pinned, None), (pinned, sjq.RunOpts(host_copy_all=True)), (pageable, None),
+                       (pinned, sjq.RunOpts(specialise=True))):
+        staging = torch.empty(sjq.staging_bytes(cols, chunk), dtype=torch.uint8, device="cuda:0")
+        res, host = sjq.run_host(cols, staging, chunk, w.preds, joins, w.key, w.agg, w.mode, w.num_groups,
+                                 w.capacity, opts)
+        torch.cuda.synchronize()
+        assert int(host.status[0]) == 0
+        assert np.array_equal(host.sums.numpy(), exp["sums"]) and np.array_equal(host.counts.numpy(), exp["counts"])
