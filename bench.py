@@ -515,7 +515,9 @@ def run_ablation(sjq, W, device, specialise=True):
                             ("global atomics group-by", sjq.RunOpts(agg_path=2)),
                             ("shared-memory privatised group-by", sjq.RunOpts(agg_path=1)),
                             ("every direct table in shared memory that fits", sjq.RunOpts(smem_tables=2)),
-                            ("no table in shared memory", sjq.RunOpts(smem_tables=1))):
+                            ("no table in shared memory", sjq.RunOpts(smem_tables=1)),
+                            ("filter stages probe the packed code arrays, not their presence bitmaps",
+                             sjq.RunOpts(no_filter_bitmap=True))):
             try:
                 timed(w, label, opts, fact=fact, dims=dims)
             except sjq.SjqError as e:
