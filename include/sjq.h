@@ -401,6 +401,8 @@ const char *sjq_version(void);
 /*
  * Run-time specialisation (Section 4.2 of the paper fuses a query's operators before it runs; here the fused
  * kernel is compiled for the query's shape with NVRTC when sjq_run_opts.specialise is set).
+ * Compiled modules are cached per process; when the environment variable SJQ_JIT_CACHE_DIR names a writable
+ * directory they are also kept there as files, so that a later process loads instead of compiling.
  * sjq_jit_log copies the compiler output of the most recent compilation into `buf` (NUL-terminated, truncated
  * to `bytes`) and returns its full length.  sjq_jit_selftest compiles one of a few built-in query shapes
  * (shape_id 0 .. sjq_jit_selftest(-1, ...) - 1) without touching a device: SJQ_OK if the device code

@@ -17,6 +17,7 @@
 // run that asks for specialisation fails with SJQ_ERR_JIT; it never falls back
 // silently.
 #include <dlfcn.h>
+#include <unistd.h>
 
 #include <cstdio>
 #include <cstdlib>
@@ -45,6 +46,7 @@ struct Nvrtc {
     int (*GetProgramLogSize)(nvrtcProgram, size_t *);
     int (*GetProgramLog)(nvrtcProgram, char *);
     int (*DestroyProgram)(nvrtcProgram *);
+    int (*Version)(int *, int *) = nullptr;
     bool ok = false;
 };
 
@@ -72,6 +74,7 @@ Nvrtc &nvrtc()
         N.GetProgramLog = reinterpret_cast<decltype(N.GetProgramLog)>(sym("nvrtcGetProgramLog"));
         N.DestroyProgram = reinterpret_cast<decltype(N.DestroyProgram)>(sym("nvrtcDestroyProgram"));
         N.ok = all;
+        N.Version = reinterpret_cast<decltype(N.Version)>(dlsym(N.handle, "nvrtcVersion"));
     });
     return N;
 }
@@ -217,6 +220,32 @@ std::mutex g_mutex;
 std::unordered_map<std::string, Module> g_modules;
 std::string g_last_log;
 
+// Optional cache of compiled modules on disk (SJQ_JIT_CACHE_DIR): a process that meets a shape some
+// earlier process compiled loads the cubin instead of compiling.  The file name is a hash of everything
+// the cubin depends on: the shape text, the device sources, the compiler's version and the options.
+uint64_t fnv1a(uint64_t h, const std::string &s)
+{
+    for (unsigned char c : s) h = (h ^ c) * 0x100000001B3ULL;
+    return h;
+}
+
+std::string cache_path(const std::string &shape, const Sources &S, int nvrtc_major, int nvrtc_minor)
+{
+    const char *dir = std::getenv("SJQ_JIT_CACHE_DIR");
+    if (!dir || !*dir) return std::string();
+    uint64_t h = 0xCBF29CE484222325ULL;
+    h = fnv1a(h, shape);
+    h = fnv1a(h, S.device);
+    h = fnv1a(h, S.run);
+    h = fnv1a(h, S.internal);
+    h = fnv1a(h, S.api);
+    if (const char *e = std::getenv("SJQ_JIT_EXTRA")) h = fnv1a(h, e);
+    char name[96];
+    std::snprintf(name, sizeof(name), "/sjq_%016llx_nvrtc%d.%d_sm100a.cubin", (unsigned long long)h, nvrtc_major,
+                  nvrtc_minor);
+    return std::string(dir) + name;
+}
+
 sjq_status compile(const std::string &shape, std::vector<char> *cubin, std::string *log)
 {
     Nvrtc &N = nvrtc();
@@ -228,6 +257,17 @@ sjq_status compile(const std::string &shape, std::vector<char> *cubin, std::stri
     if (!S.ok) {
         *log = S.error;
         return SJQ_ERR_JIT;
+    }
+    int vmaj = 0, vmin = 0;
+    if (N.Version) N.Version(&vmaj, &vmin);
+    const std::string cached = cache_path(shape, S, vmaj, vmin);
+    if (!cached.empty()) {
+        std::string bytes;
+        if (read_file(cached, &bytes) && bytes.size() > 64) {
+            cubin->assign(bytes.begin(), bytes.end());
+            *log = "loaded from " + cached;
+            return SJQ_OK;
+        }
     }
     // what precedes the //@body line of the shape text must be seen before any other header
     const size_t cut = shape.find("//@body\n");
@@ -268,6 +308,15 @@ sjq_status compile(const std::string &shape, std::vector<char> *cubin, std::stri
     } else {
         cubin->resize(cs);
         if (N.GetCUBIN(prog, cubin->data()) != 0) st = SJQ_ERR_JIT;
+        if (st == SJQ_OK && !cached.empty()) { // write beside, then rename: readers never see a partial file
+            const std::string tmp = cached + ".tmp" + std::to_string((long long)getpid());
+            std::ofstream f(tmp, std::ios::binary);
+            if (f && f.write(cubin->data(), (std::streamsize)cubin->size()) && (f.close(), true)) {
+                if (std::rename(tmp.c_str(), cached.c_str()) != 0) std::remove(tmp.c_str());
+            } else {
+                std::remove(tmp.c_str());
+            }
+        }
     }
     N.DestroyProgram(&prog);
     return st;
