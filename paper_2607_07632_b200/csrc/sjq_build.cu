@@ -484,7 +484,8 @@ extern "C" sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_c
     size_t direct_bytes = 0;
     if (direct_ok) {
         const uint64_t span = span_m1 + 1;
-        direct_bytes = npayload == 0 ? (size_t)((span + 31) / 32 * 4) : (size_t)(span * (uint64_t)(code_bits / 8));
+        // one spare entry after the last slot, never set: a probe clamps its index there instead of testing the range
+        direct_bytes = npayload == 0 ? (size_t)((span + 32) / 32 * 4) : (size_t)((span + 1) * (uint64_t)(code_bits / 8));
         direct_bytes = align_up(direct_bytes, 16);
     }
     bool use_direct;
@@ -508,7 +509,7 @@ extern "C" sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_c
         if (npayload > 0) {
             // a code array is 8 to 64 times the size of a bitmap over the same slots: keep both, so that a
             // filter stage probes the bitmap and only the survivors gather their payload from the codes
-            L.filter_bits = (int64_t)((span_m1 + 128) / 128 * 128);
+            L.filter_bits = (int64_t)((span_m1 + 129) / 128 * 128); // at least one spare bit after the last slot
             L.table_bytes += align_up((size_t)(L.filter_bits / 8), 256);
         }
     } else {
@@ -546,7 +547,7 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
         (L.filter_bits < 0 || (L.filter_bits & (L.filter_bits - 1)) || L.filter_bits > ((int64_t)1 << 32)))
         return SJQ_ERR_INVALID_ARG;
     if (L.kind <= SJQ_TABLE_DIRECT_U64 && L.filter_bits != 0 &&
-        (L.kind == SJQ_TABLE_DIRECT_BITMAP || L.filter_bits < L.slots || L.filter_bits % 128 != 0))
+        (L.kind == SJQ_TABLE_DIRECT_BITMAP || L.filter_bits <= L.slots || L.filter_bits % 128 != 0))
         return SJQ_ERR_INVALID_ARG;
     if (L.kind < SJQ_TABLE_DIRECT_BITMAP || L.kind > SJQ_TABLE_HASH_I64 || L.npayload != npayload ||
         L.key_dtype != cols[key_col].dtype || L.slots <= 0 || L.dim_rows != B.dim.n)
@@ -583,8 +584,8 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
     const bool direct = L.kind <= SJQ_TABLE_DIRECT_U64;
     if (direct) {
         const uint64_t span = (uint64_t)L.slots;
-        size_t bytes = L.kind == SJQ_TABLE_DIRECT_BITMAP ? (size_t)((span + 31) / 32 * 4)
-                                                         : (size_t)(span * (uint64_t)(L.code_bits / 8));
+        size_t bytes = L.kind == SJQ_TABLE_DIRECT_BITMAP ? (size_t)((span + 32) / 32 * 4)
+                                                         : (size_t)((span + 1) * (uint64_t)(L.code_bits / 8));
         bytes = align_up(bytes, 16);
         T->slots_bytes = bytes;
         ok = ok && cudaMemsetAsync(T->slots, L.kind == SJQ_TABLE_DIRECT_BITMAP ? 0 : 0xFF, bytes, stream) == cudaSuccess;

@@ -290,6 +290,8 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
             S.last = (uint64_t)L.slots - 1;
             S.kmin32 = (int32_t)L.kmin;
             S.last32 = (uint32_t)std::min<uint64_t>((uint64_t)L.slots - 1, 0xFFFFFFFFull);
+            // with 2^32 slots or more every 32-bit index is in range and nothing is clamped
+            S.clamp32 = (uint32_t)std::min<uint64_t>((uint64_t)L.slots, 0xFFFFFFFFull);
             S.hmask = sp.prefilter == 1 ? (uint64_t)L.filter_bits - 1 : (uint64_t)L.slots - 1;
             S.pmin0 = L.pay_min[0];
             S.pmin1 = L.pay_min[1];
@@ -561,7 +563,13 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     int per_sm = 0;
     const bool jit = opts.specialise != 0;
     // register budget a specialised kernel is compiled for
-    const int lb_blocks = single_block ? 1 : opts.ctas_per_sm > 0 ? opts.ctas_per_sm : block > 512 ? 1 : 2;
+    // (three blocks of 384 threads when their shared memory leaves the L1 alone: 56 registers are enough for the
+    // short pipelines that have so little state, and 36 warps hide more latency than 24)
+    const int lb_blocks = single_block ? 1
+                          : opts.ctas_per_sm > 0 ? opts.ctas_per_sm
+                          : block > 512 ? 1
+                          : (block <= 384 && smem <= ((size_t)48 << 10)) ? 3
+                                                                        : 2;
     st = jit ? jit_occupancy(P, aggp, mul, has_hash, block, lb_blocks, smem, &per_sm)
              : fused_occupancy(aggp, mul, has_hash, block, smem, &per_sm);
     if (st != SJQ_OK) return st;

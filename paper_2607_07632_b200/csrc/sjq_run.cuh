@@ -66,15 +66,17 @@ struct DStage {
     int32_t acc32;     // every multiplier, raw value and payload of this stage fits in 32 bits
     int32_t lo32;      // 32-bit predicate: pass iff (uint32)(v - lo32) <= width32
     uint32_t width32;
-    int32_t kmin32;    // 32-bit direct probe: idx = (uint32)v - (uint32)kmin32, hit range idx <= last32
+    int32_t kmin32;    // 32-bit direct probe: idx = min((uint32)v - (uint32)kmin32, clamp32)
     uint32_t last32;
+    uint32_t clamp32;  // index of the spare, never set entry after the last slot (every key outside the range lands there)
     uint32_t smem_off;  // byte offset of the staged copy in dynamic shared memory
     uint32_t tab_bytes; // bytes to stage
     uint16_t acc;
     uint8_t op, is64, neg, never, nset, set_idx, pbits0, code_bits, in_smem, kind;
     uint8_t simple; // 1 + destination (0 key, 1 X, 2 Y): plain int32 load feeding one accumulator through mult32
-    uint8_t pad[7];
+    uint8_t pad[3];
 };
+static_assert(sizeof(DStage) % 8 == 0, "stage descriptors are copied as 64-bit words");
 
 struct RunParams {
     DStage st[kMaxStages];
