@@ -348,6 +348,8 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     P.nd0 = nd0;
     P.nq = direct ? 0 : nfq + 1;
     P.rows = opts.rows_per_lane ? opts.rows_per_lane : 4;
+    // a third or more of the rows reaching the first queue: pushes are dense enough for bank conflicts to matter
+    P.qfold = (opts.specialise && P.nq && reach[nd0] >= 0.3) ? 7u : 0u;
 
     // Sources of the accumulators.  A dense stage cannot feed an accumulator
     // (it only keeps a bit per row), so a value it would supply is gathered

@@ -97,6 +97,7 @@ struct RunParams {
                     // stages from nd0+nq-1 on run at the final level
     int32_t nd0;
     int32_t rows;   // rows per lane and batch at the queue-fed levels: 4, or 8 in a kernel compiled for it
+    uint32_t qfold; // 7: queue slots are swizzled (dense survivors), 0: ring positions are used as they are
     int32_t want_count;
     int32_t eager;   // load every column for every row
     int32_t has_key; // scalar path of a one-group dense result: key is computed and range-checked
