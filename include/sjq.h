@@ -381,6 +381,9 @@ sjq_status sjq_host_transfer_plan(const sjq_col *fact_host, int nfact, const sjq
  *   - `opts->accumulate` is ignored: the table is cleared at the start of
  *     every call, because it is shared by all calls and still holds the
  *     previous call's groups.
+ *   - `opts->specialise` is ignored: loading a module compiled at run time
+ *     allocates device memory, so this entry point always runs the interpreted
+ *     kernel.
  *   - Calls whose kernels could overlap on the GPU (different streams, several
  *     host threads) race on the one table; run them one after another.
  *   - The first call on a device looks the array's device address up once; make

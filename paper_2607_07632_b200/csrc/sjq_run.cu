@@ -881,5 +881,6 @@ extern "C" sjq_status sjq_run_hashed_static(const sjq_col *fact, int nfact, cons
     sjq_run_opts opts{};
     if (opts_) opts = *opts_;
     opts.accumulate = 0; // the shared table holds the last call's groups: always start from a cleared table
+    opts.specialise = 0; // loading a compiled module allocates device memory: this entry point only interprets
     return sjq_run(fact, nfact, preds, npreds, joins, njoins, key, agg, &spec, &r, &opts, stream, info);
 }
