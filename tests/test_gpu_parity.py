@@ -49,7 +49,7 @@ def test_random_queries_option_matrix(seed):
     tables = None
     for opts in (sjq.RunOpts(), sjq.RunOpts(eager_loads=True), sjq.RunOpts(smem_tables=1),
                  sjq.RunOpts(block_threads=128, ctas_per_sm=1), sjq.RunOpts(block_threads=256, compaction=2, smem_tables=1), sjq.RunOpts(agg_path=2),
-                 sjq.RunOpts(compaction=2), sjq.RunOpts(compaction=1),
+                 sjq.RunOpts(compaction=2), sjq.RunOpts(compaction=1), sjq.RunOpts(no_filter_bitmap=True),
                  sjq.RunOpts(order=tuple(reversed(range(len(w.preds) + len(w.joins)))))):
         res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)
         assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)
@@ -343,3 +343,13 @@ def test_host_path_reads_sparse_columns_in_place_and_matches_copies():
         torch.cuda.synchronize()
         assert int(host.status[0]) == 0
         assert np.array_equal(host.sums.numpy(), exp["sums"]) and np.array_equal(host.counts.numpy(), exp["counts"])
+
+
+def test_rows_per_lane_eight_needs_the_specialised_kernel():
+    w, fact, hd, _ = ex1()
+    tables = sjq.build_workload_tables(w, {k: to_dev(v) for k, v in hd.items()})
+    with pytest.raises(sjq.SjqError) as e:
+        sjq.run_workload(w, to_dev(fact), tables, sjq.RunOpts(rows_per_lane=8))
+    assert e.value.status == 1
+    with pytest.raises(sjq.SjqError):
+        sjq.run_workload(w, to_dev(fact), tables, sjq.RunOpts(rows_per_lane=5, specialise=True))
