@@ -417,6 +417,33 @@ def alloc_result(mode: str, num_groups: int, capacity: int, want_count: bool, de
     return Result(mode, sums, counts, keys, n_groups, status, ws)
 
 
+def _query(names: Sequence[str], preds, joins, key, agg):
+    """Marshal the query part of a call: (predicates, joins, key expression or None, aggregate expression,
+    objects that must outlive the call)."""
+    parr, keep = _preds(preds, names)
+    jarr = (_Join * max(1, len(joins)))()
+    for j, (fk, table) in enumerate(joins):
+        jarr[j] = _Join(names.index(fk), table.handle)
+    kexpr = None
+    if key is not None:
+        if len(key.terms) > MAX_KEY_TERMS:
+            raise ValueError("too many key terms")
+        kexpr = _KeyExpr()
+        for i, t in enumerate(key.terms):
+            kexpr.t[i] = _term(t, names)
+        kexpr.nterms, kexpr.offset, kexpr.modulo = len(key.terms), key.offset, key.modulo
+    aexpr = _AggExpr(AGGS[agg.op], _term(agg.x, names), _term(agg.y, names), int(agg.want_count))
+    return parr, jarr, kexpr, aexpr, keep
+
+
+def _result_struct(res: "Result") -> _Result:
+    return _Result(res.sums.data_ptr(), res.counts.data_ptr() if res.counts is not None else None,
+                   res.keys.data_ptr() if res.keys is not None else None,
+                   res.n_groups.data_ptr() if res.n_groups is not None else None, res.status_dev.data_ptr(),
+                   res.workspace.data_ptr() if res.workspace is not None else None,
+                   res.workspace.numel() if res.workspace is not None else 0)
+
+
 def run(fact: dict, preds=(), joins=(), key=None, agg=None, mode: str = "SCALAR", num_groups: int = 1,
         capacity: int = 0, opts: Optional[RunOpts] = None, result: Optional[Result] = None) -> Result:
     """sjq_run over a dict of CUDA tensors.  joins: sequence of (fk column name, Table)."""
@@ -425,26 +452,10 @@ def run(fact: dict, preds=(), joins=(), key=None, agg=None, mode: str = "SCALAR"
     device = tensors[0].device
     with torch.cuda.device(device):
         carr = _cols(tensors)
-        parr, keep = _preds(preds, names)
-        jarr = (_Join * max(1, len(joins)))()
-        for j, (fk, table) in enumerate(joins):
-            jarr[j] = _Join(names.index(fk), table.handle)
-        kexpr = None
-        if key is not None:
-            kexpr = _KeyExpr()
-            if len(key.terms) > MAX_KEY_TERMS:
-                raise ValueError("too many key terms")
-            for i, t in enumerate(key.terms):
-                kexpr.t[i] = _term(t, names)
-            kexpr.nterms, kexpr.offset, kexpr.modulo = len(key.terms), key.offset, key.modulo
-        aexpr = _AggExpr(AGGS[agg.op], _term(agg.x, names), _term(agg.y, names), int(agg.want_count))
+        parr, jarr, kexpr, aexpr, keep = _query(names, preds, joins, key, agg)
         spec = _ResultSpec(MODES[mode], num_groups, capacity)
         res = result if result is not None else alloc_result(mode, num_groups, capacity, agg.want_count, device)
-        cres = _Result(res.sums.data_ptr(), res.counts.data_ptr() if res.counts is not None else None,
-                       res.keys.data_ptr() if res.keys is not None else None,
-                       res.n_groups.data_ptr() if res.n_groups is not None else None, res.status_dev.data_ptr(),
-                       res.workspace.data_ptr() if res.workspace is not None else None,
-                       res.workspace.numel() if res.workspace is not None else 0)
+        cres = _result_struct(res)
         copts = (opts or RunOpts()).to_c()
         rc = lib().sjq_run(carr, len(names), parr, len(preds), jarr, len(joins),
                            ctypes.byref(kexpr) if kexpr is not None else None, ctypes.byref(aexpr),
@@ -469,15 +480,7 @@ def run_hashed_static(fact: dict, preds=(), joins=(), key=None, agg=None, capaci
     device = tensors[0].device
     with torch.cuda.device(device):
         carr = _cols(tensors)
-        parr, keep = _preds(preds, names)
-        jarr = (_Join * max(1, len(joins)))()
-        for j, (fk, table) in enumerate(joins):
-            jarr[j] = _Join(names.index(fk), table.handle)
-        kexpr = _KeyExpr()
-        for i, t in enumerate(key.terms):
-            kexpr.t[i] = _term(t, names)
-        kexpr.nterms, kexpr.offset, kexpr.modulo = len(key.terms), key.offset, key.modulo
-        aexpr = _AggExpr(AGGS[agg.op], _term(agg.x, names), _term(agg.y, names), int(agg.want_count))
+        parr, jarr, kexpr, aexpr, keep = _query(names, preds, joins, key, agg)
         if result is None:
             n = max(1, capacity)
             result = Result("HASHED", torch.empty(n, dtype=torch.int64, device=device),
@@ -521,17 +524,7 @@ def host_transfer_plan(fact: dict, preds=(), joins=(), key=None, agg=None, opts:
     carr = (_Col * len(tensors))()
     for i, t in enumerate(tensors):
         carr[i] = _Col(t.data_ptr(), 1 if t.dtype == torch.int64 else 0, t.numel())
-    parr, keep = _preds(preds, names)
-    jarr = (_Join * max(1, len(joins)))()
-    for j, (fk, table) in enumerate(joins):
-        jarr[j] = _Join(names.index(fk), table.handle)
-    kexpr = None
-    if key is not None:
-        kexpr = _KeyExpr()
-        for i, t in enumerate(key.terms):
-            kexpr.t[i] = _term(t, names)
-        kexpr.nterms, kexpr.offset, kexpr.modulo = len(key.terms), key.offset, key.modulo
-    aexpr = _AggExpr(AGGS[agg.op], _term(agg.x, names), _term(agg.y, names), int(agg.want_count))
+    parr, jarr, kexpr, aexpr, keep = _query(names, preds, joins, key, agg)
     copts = (opts or RunOpts()).to_c()
     how = (ctypes.c_int32 * len(names))()
     share = (ctypes.c_double * len(names))()
@@ -561,17 +554,7 @@ def run_host(fact: dict, staging: torch.Tensor, chunk_rows: int, preds=(), joins
             if t.is_cuda or t.dtype not in (torch.int32, torch.int64) or not t.is_contiguous():
                 raise ValueError("run_host takes contiguous int32/int64 host tensors")
             carr[i] = _Col(t.data_ptr(), 1 if t.dtype == torch.int64 else 0, t.numel())
-        parr, keep = _preds(preds, names)
-        jarr = (_Join * max(1, len(joins)))()
-        for j, (fk, table) in enumerate(joins):
-            jarr[j] = _Join(names.index(fk), table.handle)
-        kexpr = None
-        if key is not None:
-            kexpr = _KeyExpr()
-            for i, t in enumerate(key.terms):
-                kexpr.t[i] = _term(t, names)
-            kexpr.nterms, kexpr.offset, kexpr.modulo = len(key.terms), key.offset, key.modulo
-        aexpr = _AggExpr(AGGS[agg.op], _term(agg.x, names), _term(agg.y, names), int(agg.want_count))
+        parr, jarr, kexpr, aexpr, keep = _query(names, preds, joins, key, agg)
         spec = _ResultSpec(MODES[mode], num_groups, capacity)
         res = result if result is not None else alloc_result(mode, num_groups, capacity, agg.want_count, device)
         if host is None:
@@ -581,11 +564,7 @@ def run_host(fact: dict, staging: torch.Tensor, chunk_rows: int, preds=(), joins
                               torch.empty_like(res.keys, device="cpu", **pin) if res.keys is not None else None,
                               torch.zeros(1, dtype=torch.int64, **pin) if res.n_groups is not None else None,
                               torch.zeros(1, dtype=torch.int32, **pin))
-        cres = _Result(res.sums.data_ptr(), res.counts.data_ptr() if res.counts is not None else None,
-                       res.keys.data_ptr() if res.keys is not None else None,
-                       res.n_groups.data_ptr() if res.n_groups is not None else None, res.status_dev.data_ptr(),
-                       res.workspace.data_ptr() if res.workspace is not None else None,
-                       res.workspace.numel() if res.workspace is not None else 0)
+        cres = _result_struct(res)
         copts = (opts or RunOpts()).to_c()
         rc = lib().sjq_run_host(carr, len(names), parr, len(preds), jarr, len(joins),
                                 ctypes.byref(kexpr) if kexpr is not None else None, ctypes.byref(aexpr),
