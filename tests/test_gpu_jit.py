@@ -161,3 +161,17 @@ def test_largest_query_shape_both_kernels(seed):
         res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)
         assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)
         compare(w, res, exp)
+
+
+@pytest.mark.parametrize("seed", range(400, 430))
+def test_random_queries_over_many_tiles_both_kernels(seed):
+    """Random query shapes over a fact table of several tiles with a ragged tail (the hand-sized random
+    queries fit one tile): queues fill, drain and wrap for shapes no configuration has."""
+    n = 20_000 + 37 * (seed % 7) + (seed % 4)
+    w, fact, hd = random_query(seed, n_fact=n, max_dim=40, allow_dup=False, wide_keys=True)
+    dev_fact = to_dev(fact)
+    tables = None
+    for opts in (sjq.RunOpts(), spec(), spec(block_threads=128, ctas_per_sm=4), sjq.RunOpts(compaction=2)):
+        res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)
+        assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)
+        compare(w, res, exp)
