@@ -167,7 +167,8 @@ std::string jit_shape_header(const RunParams &P, int agg, bool mul, bool hash, i
         o << "    case " << s << ":\n        S.op = " << (int)S.op << "; S.is64 = " << (int)S.is64 << "; S.neg = " << (int)S.neg
           << "; S.never = " << (int)S.never << "; S.nset = " << (int)S.nset << "; S.set_idx = " << (int)S.set_idx
           << "; S.in_smem = " << (int)S.in_smem << "; S.kind = " << (int)S.kind << "; S.simple = " << (int)S.simple
-          << "; S.acc = " << (int)S.acc << "; S.acc32 = " << S.acc32 << "; S.code_bits = " << (int)S.code_bits << ";\n";
+          << "; S.acc = " << (int)S.acc << "; S.acc32 = " << S.acc32 << "; S.code_bits = " << (int)S.code_bits
+          << "; S.issue_after = " << (int)S.issue_after << ";\n";
         for (int i = 0; i < 9; ++i) {
             // INT64_MIN cannot be written as a literal
             if (S.mult[i] == INT64_MIN) o << "        S.mult[" << i << "] = (-9223372036854775807LL - 1);";
@@ -197,7 +198,8 @@ std::string shape_key(const RunParams &P, int agg, bool mul, bool hash, int lb_t
     put_raw(&P.modmask, sizeof(P.modmask));
     for (int s = 0; s < P.nstages; ++s) {
         const DStage &S = P.st[s];
-        const uint8_t b[] = {S.op, S.is64, S.neg, S.never, S.nset, S.set_idx, S.in_smem, S.kind, S.simple, S.code_bits};
+        const uint8_t b[] = {S.op, S.is64, S.neg, S.never, S.nset, S.set_idx, S.in_smem, S.kind, S.simple, S.code_bits,
+                             (uint8_t)S.issue_after};
         put_raw(b, sizeof(b));
         put_raw(&S.acc, sizeof(S.acc));
         put_raw(&S.acc32, sizeof(S.acc32));
@@ -500,6 +502,18 @@ int canned_shape(int id, RunParams *P, int *agg, bool *mul, bool *hash)
 } // namespace
 } // namespace sjq
 
+namespace sjq {
+namespace {
+// the load schedule the planner would give a final level none of whose stages drops rows
+void canned_schedule(RunParams *P)
+{
+    if (!P->nq) return;
+    const int first = P->nd0 + P->nq - 1;
+    for (int t = first; t < P->nstages; ++t) P->st[t].issue_after = (int8_t)(t - 3 > first - 1 ? t - 3 : first - 1);
+}
+} // namespace
+} // namespace sjq
+
 extern "C" int32_t sjq_jit_selftest(int32_t shape_id, char *log, size_t log_bytes)
 {
     static sjq::RunParams P; // large: keep it off the stack
@@ -513,6 +527,7 @@ extern "C" int32_t sjq_jit_selftest(int32_t shape_id, char *log, size_t log_byte
         return n;
     }
     if (!sjq::canned_shape(shape_id, &P, &agg, &mul, &hash)) return SJQ_ERR_INVALID_ARG;
+    sjq::canned_schedule(&P);
     std::string text;
     size_t cubin = 0;
     const sjq_status st = sjq::jit_compile_only(sjq::jit_shape_header(P, agg, mul, hash, 384, 2), &text, &cubin);

@@ -438,6 +438,18 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     }
     P.nstages = ns;
     P.eager = opts.eager_loads ? 1 : 0;
+    // Load schedule of the final level (used by kernels compiled for the query): a column is requested
+    // once the last stage before it that is expected to drop rows has produced its mask, and at most
+    // three columns ahead of the stage being processed.
+    if (P.nq) {
+        const int first = ndense;
+        int last_barrier = first - 1;
+        for (int t = first; t < ns; ++t) {
+            P.st[t].issue_after = (int8_t)std::max(std::max(last_barrier, t - 3), first - 1);
+            const bool drops = t < nfilter && specs[order[t]].sel < 0.9;
+            if (drops) last_barrier = t;
+        }
+    }
 
     // ------------------------------------------------------------ aggregation path
     int aggp;

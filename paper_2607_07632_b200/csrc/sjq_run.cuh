@@ -74,7 +74,9 @@ struct DStage {
     uint16_t acc;
     uint8_t op, is64, neg, never, nset, set_idx, pbits0, code_bits, in_smem, kind;
     uint8_t simple; // 1 + destination (0 key, 1 X, 2 Y): plain int32 load feeding one accumulator through mult32
-    uint8_t pad[3];
+    int8_t issue_after; // final level of a compiled kernel: the column is requested once this stage's mask is known
+                        // (a stage before the level's first one = on entry)
+    uint8_t pad[2];
 };
 static_assert(sizeof(DStage) % 8 == 0, "stage descriptors are copied as 64-bit words");
 
