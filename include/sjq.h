@@ -17,8 +17,11 @@
  *     Descriptor structs (columns, predicates, expressions, options) are HOST
  *     memory and are copied during the call.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
- *   - The library allocates no device memory.  All kernels are enqueued on
- *     the given stream; calls return after enqueueing unless stated otherwise.
+ *   - The library allocates no device memory for data.  (A run that asks for
+ *     run-time specialisation loads a compiled module the first time it meets
+ *     a query shape; the CUDA driver places the module's code on the device.)
+ *     All kernels are enqueued on the given stream; calls return after
+ *     enqueueing unless stated otherwise.
  *   - Functions return 0 (SJQ_OK) or a host-detected error code.  Errors only
  *     the device can see are written to the caller's int32 status word (first
  *     error wins); kernels never trap and never spin without a bound.  Results
