@@ -416,6 +416,9 @@ const char *sjq_version(void);
  * of built-in shapes instead of a status.
  */
 size_t sjq_jit_log(char *buf, size_t bytes);
+/* Unload every module compiled at run time in this process and forget them (the next specialised run of a shape
+ * compiles or loads it again); returns how many were unloaded.  No kernel of such a module may still be running. */
+int32_t sjq_jit_cache_clear(void);
 int32_t sjq_jit_selftest(int32_t shape_id, char *log, size_t log_bytes);
 
 #ifdef __cplusplus

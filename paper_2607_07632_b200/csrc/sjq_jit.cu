@@ -418,6 +418,20 @@ sjq_status jit_compile_only(const std::string &shape, std::string *log, size_t *
 } // namespace sjq
 
 // ---------------------------------------------------------------- C ABI
+extern "C" int32_t sjq_jit_cache_clear(void)
+{
+    std::lock_guard<std::mutex> lock(sjq::g_mutex);
+    int32_t n = 0;
+    for (auto &kv : sjq::g_modules) {
+        if (kv.second.lib) {
+            if (cudaLibraryUnload(kv.second.lib) != cudaSuccess) (void)cudaGetLastError();
+            ++n;
+        }
+    }
+    sjq::g_modules.clear();
+    return n;
+}
+
 extern "C" size_t sjq_jit_log(char *buf, size_t bytes)
 {
     std::lock_guard<std::mutex> lock(sjq::g_mutex);

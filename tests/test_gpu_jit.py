@@ -175,3 +175,16 @@ def test_random_queries_over_many_tiles_both_kernels(seed):
         res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)
         assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)
         compare(w, res, exp)
+
+
+def test_clearing_the_module_cache_recompiles_and_gives_the_same_bits():
+    w, fact, hd, _ = ex2()
+    res, exp, tables = run_both(w, fact, hd, opts=spec())
+    compare(w, res, exp)
+    torch.cuda.synchronize()
+    L = sjq.sjq.lib()
+    L.sjq_jit_cache_clear.restype = ctypes.c_int32
+    assert L.sjq_jit_cache_clear() >= 1
+    assert L.sjq_jit_cache_clear() == 0
+    res2, _, _ = run_both(w, fact, hd, opts=spec(), tables=tables)
+    compare(w, res2, exp)
