@@ -275,7 +275,9 @@ typedef struct sjq_run_opts {
     int32_t host_copy_all; /* sjq_run_host: 1 = copy every referenced column to the device; 0 = columns that only a
                               few per cent of the rows reach are read by the kernel from the page-locked host
                               buffer instead */
-    int32_t reserved[3];
+    int32_t dense_slots; /* level 0: groups of four consecutive rows a thread owns per tile: 0 = library chooses, 2,
+                            or 4 (4 only with specialise) */
+    int32_t reserved[2];
 } sjq_run_opts;
 
 /* What the planner decided for a run (for reports and tests). */

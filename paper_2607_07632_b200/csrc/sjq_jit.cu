@@ -147,7 +147,8 @@ void put(std::ostringstream &o, const char *name, long long v) { o << "#define S
 std::string jit_shape_header(const RunParams &P, int agg, bool mul, bool hash, int lb_threads, int lb_blocks)
 {
     std::ostringstream o;
-    o << "// generated: the shape of one query\n#define SJQ_ROWS " << (P.rows == 8 ? 8 : 4) << "\n//@body\n";
+    o << "// generated: the shape of one query\n#define SJQ_ROWS " << (P.rows == 8 ? 8 : 4) << "\n#define SJQ_SLOTS "
+      << (P.slots == 4 ? 4 : 2) << "\n//@body\n";
     o << "#define SJQ_JIT_AGG " << agg << "\n#define SJQ_JIT_MUL " << (mul ? 1 : 0) << "\n#define SJQ_JIT_HASH "
       << (hash ? 1 : 0) << "\n";
     o << "#define SJQ_LB_THREADS " << lb_threads << "\n#define SJQ_LB_BLOCKS " << lb_blocks << "\n";
@@ -192,7 +193,7 @@ std::string shape_key(const RunParams &P, int agg, bool mul, bool hash, int lb_t
     k.reserve(64 + (size_t)P.nstages * 128);
     auto put_raw = [&](const void *p, size_t n) { k.append(static_cast<const char *>(p), n); };
     const int32_t head[] = {agg, mul ? 1 : 0, hash ? 1 : 0, lb_threads, lb_blocks, P.nstages, P.nd0, P.nq,
-                            P.rows, P.want_count, P.eager, P.has_key, P.mod32, (int32_t)P.qfold};
+                            P.rows, P.want_count, P.eager, P.has_key, P.mod32, (int32_t)P.qfold, P.slots};
     put_raw(head, sizeof(head));
     put_raw(&P.modulo, sizeof(P.modulo));
     put_raw(&P.modmask, sizeof(P.modmask));

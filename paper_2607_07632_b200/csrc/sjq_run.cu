@@ -208,6 +208,8 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         return SJQ_ERR_INVALID_ARG;
     if (opts.rows_per_lane != 0 && opts.rows_per_lane != 4 && !(opts.rows_per_lane == 8 && opts.specialise))
         return SJQ_ERR_INVALID_ARG;
+    if (opts.dense_slots != 0 && opts.dense_slots != 2 && !(opts.dense_slots == 4 && opts.specialise))
+        return SJQ_ERR_INVALID_ARG;
     if (opts.norder && opts.norder != npreds + njoins) return SJQ_ERR_INVALID_ARG;
 
     DeviceInfo dev;
@@ -348,6 +350,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     P.nd0 = nd0;
     P.nq = direct ? 0 : nfq + 1;
     P.rows = opts.rows_per_lane ? opts.rows_per_lane : 4;
+    P.slots = (opts.specialise && opts.dense_slots == 4) ? 4 : 2;
     // a third or more of the rows reaching the first queue: pushes are dense enough for bank conflicts to matter
     P.qfold = (opts.specialise && P.nq && reach[nd0] >= 0.3) ? 7u : 0u;
 
@@ -507,7 +510,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     int block = opts.block_threads ? opts.block_threads : SJQ_LB_THREADS;
     const size_t smem_cap = (size_t)dev.max_smem_optin - 1024; // static reduce scratch + slack
     const size_t stage_bytes = align_up((size_t)ns * sizeof(DStage), 16);
-    auto queue_bytes = [&](int threads) { return P.nq ? (size_t)(threads / 32) * (size_t)(kQueue0Cap + (P.nq - 1) * queue_cap_for(P.rows)) * 4 : (size_t)0; };
+    auto queue_bytes = [&](int threads) { return P.nq ? (size_t)(threads / 32) * (size_t)(queue0_cap_for(P.slots) + (P.nq - 1) * queue_cap_for(P.rows)) * 4 : (size_t)0; };
     // Direct tables (and presence bitmaps) worth a copy in shared memory, most probes per staged byte first.
     auto stage_tables = [&](int threads, size_t *tables_out) -> bool {
         for (int s2 = 0; s2 < ns; ++s2) P.st[s2].in_smem = 0, P.st[s2].smem_off = 0;
@@ -554,7 +557,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     bool single_block = false;
     if (opts.specialise && !opts.block_threads && !opts.ctas_per_sm && P.nq) {
         const size_t copies = tables + group_bytes;
-        const int64_t tiles_per_block = n / ((int64_t)1024 * kDenseRows) / dev.sm_count;
+        const int64_t tiles_per_block = n / ((int64_t)1024 * 4 * P.slots) / dev.sm_count;
         size_t tables1024 = 0;
         if ((copies >= ((size_t)16 << 10) || stage_bytes + copies + queue_bytes(block) > ((size_t)80 << 10)) &&
             tiles_per_block >= 128 && stage_tables(1024, &tables1024)) {
@@ -589,7 +592,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     if (st != SJQ_OK) return st;
     if (per_sm < 1) return SJQ_ERR_UNSUPPORTED;
     if (opts.ctas_per_sm > 0) per_sm = std::min(per_sm, opts.ctas_per_sm);
-    const int64_t tile_rows = (int64_t)block * (P.nq ? kDenseRows : kDirectRows);
+    const int64_t tile_rows = (int64_t)block * (P.nq ? 4 * P.slots : kDirectRows);
     const int64_t ntiles = (n + tile_rows - 1) / tile_rows;
     if (ntiles >= ((int64_t)1 << 31)) return SJQ_ERR_UNSUPPORTED;
     int grid = (int)std::min<int64_t>((int64_t)dev.sm_count * per_sm, std::max<int64_t>(ntiles, 1));

@@ -46,7 +46,8 @@ constexpr int kDenseRows = 4 * kSlots;   // rows a thread owns at level 0
 constexpr int kRows = SJQ_ROWS;          // rows a lane handles per batch at the queue-fed levels
 constexpr int kDirectRows = 4;           // rows a thread owns when there are no queues at all (one 128-bit load)
 constexpr int kBatch = 32 * kRows;       // rows a warp processes at once at those levels
-constexpr int kQueue0Cap = kSlots <= 2 ? 512 : 1024; // first queue of a warp: a batch minus one plus a whole tile fit
+constexpr int queue0_cap_for(int slots) { return slots <= 2 ? 512 : 1024; }
+constexpr int kQueue0Cap = queue0_cap_for(kSlots); // first queue of a warp: a batch minus one plus a whole tile fit
 constexpr int queue_cap_for(int rows) { return 64 * rows; }
 constexpr int kQueueCap = queue_cap_for(kRows); // its later queues: a batch minus one plus a batch fit
 constexpr int kMaxQueues = 3;            // queue-fed levels per warp (the last one is the final level)
@@ -99,6 +100,7 @@ struct RunParams {
                     // stages from nd0+nq-1 on run at the final level
     int32_t nd0;
     int32_t rows;   // rows per lane and batch at the queue-fed levels: 4, or 8 in a kernel compiled for it
+    int32_t slots;  // level 0: groups of four rows a thread owns per tile: 2, or 4 in a kernel compiled for it
     uint32_t qfold; // 7: queue slots are swizzled (dense survivors), 0: ring positions are used as they are
     int32_t want_count;
     int32_t eager;   // load every column for every row

@@ -93,7 +93,8 @@ class _RunOpts(ctypes.Structure):
                 ("order", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS)), ("event_before", ctypes.c_void_p),
                 ("event_after", ctypes.c_void_p), ("dense_reach_permille", ctypes.c_int32), ("specialise", ctypes.c_int32),
                 ("rows_per_lane", ctypes.c_int32), ("no_filter_bitmap", ctypes.c_int32),
-                ("host_copy_all", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3)]
+                ("host_copy_all", ctypes.c_int32), ("dense_slots", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 2)]
 
 
 class RunInfo(ctypes.Structure):
@@ -126,6 +127,7 @@ class RunOpts:
     rows_per_lane: int = 0  # queue-fed levels: 0 auto, 4, or 8 (8 needs specialise)
     no_filter_bitmap: bool = False  # filter stages probe the code array of a direct table, not its bitmap
     host_copy_all: bool = False  # run_host: copy every referenced column instead of reading sparse ones in place
+    dense_slots: int = 0  # level 0: 0 auto, 2, or 4 groups of four rows per thread (4 needs specialise)
 
     def to_c(self) -> _RunOpts:
         o = _RunOpts()
@@ -140,6 +142,7 @@ class RunOpts:
         o.rows_per_lane = self.rows_per_lane
         o.no_filter_bitmap = int(self.no_filter_bitmap)
         o.host_copy_all = int(self.host_copy_all)
+        o.dense_slots = self.dense_slots
         if self.events is not None:
             o.event_before, o.event_after = self.events[0].cuda_event, self.events[1].cuda_event
         return o
