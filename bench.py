@@ -31,7 +31,7 @@ CONTRACT_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per fact row of the fused kernel, from an ncu capture of a 100 M-row case of the same workload
 # (dram__bytes_read.sum + dram__bytes_write.sum; traffic grows in proportion to the rows)
-NCU_DRAM_BYTES_PER_ROW = {"c3": 12.5}
+NCU_DRAM_BYTES_PER_ROW = {"c3": 12.2}
 
 
 def measured_hbm_peak():
