@@ -15,11 +15,11 @@
 
 #include "sjq_run.cuh"
 
+// Block size the ahead-of-time kernels are built for (their launch bound); a build for experiments may set another.
 #ifndef SJQ_LB_THREADS
-#define SJQ_LB_THREADS_MAX 384
-#else
-#define SJQ_LB_THREADS_MAX SJQ_LB_THREADS
+#define SJQ_LB_THREADS 384
 #endif
+#define SJQ_LB_THREADS_MAX SJQ_LB_THREADS
 
 namespace sjq {
 
@@ -504,9 +504,6 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
 
     // ------------------------------------------------------------ shared memory layout
     // [stage descriptors][staged tables][group table][per-warp survivor queues]
-    #ifndef SJQ_LB_THREADS
-#define SJQ_LB_THREADS 384
-#endif
     int block = opts.block_threads ? opts.block_threads : SJQ_LB_THREADS;
     const size_t smem_cap = (size_t)dev.max_smem_optin - 1024; // static reduce scratch + slack
     const size_t stage_bytes = align_up((size_t)ns * sizeof(DStage), 16);
