@@ -463,6 +463,11 @@ def run_extras(sjq, W, device, specialise=True):
     for s in (0.0001, 0.01, 0.1, 0.5, 1.0):
         for g in (1, 1000, 100000, 1000000):
             timed(W.config4(600_000_000, s, g))
+    # the large group counts as DENSE results too (global atomics, no key look-up), for comparison with the
+    # hashed form the configuration asks for
+    for s in (0.1, 1.0):
+        for g in (100000, 1000000):
+            timed(W.config4(600_000_000, s, g, hashed=False))
     return out
 
 
