@@ -530,6 +530,13 @@ def run_ablation(sjq, W, device, specialise=True):
         timed(w, "open-addressing tables instead of packed direct maps", None, force_hash=True, fact=fact, dims=dims)
         del fact, dims
         torch.cuda.empty_cache()
+    # hashed result over a million groups: the table indexed by the key (what a modulo key allows) vs the hash table
+    w = W.config4(600_000_000, 0.1, 1000000)
+    fact, dims = timed(w, "default")
+    timed(w, "group hash table instead of the direct-indexed group table", sjq.RunOpts(group_hash_always=True),
+          fact=fact, dims=dims)
+    del fact, dims
+    torch.cuda.empty_cache()
     return out
 
 

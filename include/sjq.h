@@ -231,7 +231,9 @@ typedef struct sjq_result_spec {
  *   SCALAR: sums[0], counts[0].
  *   DENSE : sums[num_groups], counts[num_groups] (absent groups are zero).
  *   HASHED: keys/sums/counts[capacity] hold *n_groups entries in no particular
- *           order; `workspace` is the group hash table (scratch).
+ *           order; `workspace` is the group table (scratch): an
+ *           open-addressing hash table, or, when the key is taken modulo M and
+ *           2M - 1 cells fit, a table indexed by the key itself.
  * `counts` may be NULL when want_count is 0 (SCALAR and DENSE only).
  * `n_groups` is required for HASHED.  `status` is always required. */
 typedef struct sjq_result {
@@ -277,7 +279,10 @@ typedef struct sjq_run_opts {
                               buffer instead */
     int32_t dense_slots; /* level 0: groups of four consecutive rows a thread owns per tile: 0 = library chooses, 2,
                             or 4 (4 only with specialise) */
-    int32_t reserved[2];
+    int32_t group_hash_always; /* HASHED results: 1 = always use the group hash table; 0 = a key taken modulo M whose
+                                  2M - 1 possible values fit the workspace is aggregated in a table indexed by the
+                                  key itself */
+    int32_t reserved[1];
 } sjq_run_opts;
 
 /* What the planner decided for a run (for reports and tests). */

@@ -35,7 +35,8 @@ __global__ void __launch_bounds__(256) clear_kernel(const ClearParams C)
 
 struct CompactParams {
     const int64_t *gkeys, *gsums, *gcounts;
-    int64_t gslots; // regular slots; the side slot follows
+    int64_t dense_base; // >= 0: the table is indexed by key + dense_base and has no key array
+    int64_t gslots; // regular slots; the side slot follows (direct-indexed: cells - 1)
     int64_t *keys, *sums, *counts;
     int64_t capacity;
     int64_t *n_groups;
@@ -47,9 +48,10 @@ __global__ void __launch_bounds__(256) compact_kernel(const CompactParams C)
 {
     const int64_t stride = (int64_t)blockDim.x * gridDim.x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i <= C.gslots; i += stride) {
-        const bool side = i == C.gslots;
-        const int64_t k = side ? kEmptyKey64 : C.gkeys[i];
-        const bool used = side ? (C.gcounts[i] != 0) : (k != kEmptyKey64);
+        const bool direct = C.dense_base >= 0;
+        const bool side = !direct && i == C.gslots;
+        const int64_t k = direct ? i - C.dense_base : side ? kEmptyKey64 : C.gkeys[i];
+        const bool used = (direct || side) ? (C.gcounts[i] != 0) : (k != kEmptyKey64);
         if (!used) continue;
         const int64_t pos = (int64_t)atomicAdd(reinterpret_cast<unsigned long long *>(C.n_groups), 1ull);
         if (pos < C.capacity) {
@@ -147,10 +149,10 @@ sjq_status clear_launch(int64_t *sums, int64_t *counts, int64_t cells, int64_t *
 }
 
 sjq_status compact_launch(const int64_t *gkeys, const int64_t *gsums, const int64_t *gcounts, int64_t gslots,
-                          int64_t *keys, int64_t *sums, int64_t *counts, int64_t capacity, int64_t *n_groups,
-                          int32_t *status, int sm_count, cudaStream_t stream)
+                          int64_t dense_base, int64_t *keys, int64_t *sums, int64_t *counts, int64_t capacity,
+                          int64_t *n_groups, int32_t *status, int sm_count, cudaStream_t stream)
 {
-    CompactParams C{gkeys, gsums, gcounts, gslots, keys, sums, counts, capacity, n_groups, status};
+    CompactParams C{gkeys, gsums, gcounts, dense_base, gslots, keys, sums, counts, capacity, n_groups, status};
     int64_t blocks = (gslots + 256) / 256;
     if (blocks > (int64_t)sm_count * 8) blocks = (int64_t)sm_count * 8;
     compact_kernel<<<(int)blocks, 256, 0, stream>>>(C);

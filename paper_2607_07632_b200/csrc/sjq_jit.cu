@@ -159,6 +159,7 @@ std::string jit_shape_header(const RunParams &P, int agg, bool mul, bool hash, i
     o << "#define SJQ_JIT_want_count " << P.want_count << "\n#define SJQ_JIT_eager " << P.eager
       << "\n#define SJQ_JIT_has_key " << P.has_key << "\n#define SJQ_JIT_mod32 " << P.mod32 << "\n";
     put(o, "modulo", P.modulo);
+    put(o, "post_offset", P.post_offset);
     o << "#define SJQ_JIT_modmask " << P.modmask << "ULL\n";
     o << "namespace sjq {\nnamespace {\n"
          "__device__ __forceinline__ DStage jit_stage(const RunParams &P, int s)\n{\n"
@@ -196,6 +197,7 @@ std::string shape_key(const RunParams &P, int agg, bool mul, bool hash, int lb_t
                             P.rows, P.want_count, P.eager, P.has_key, P.mod32, (int32_t)P.qfold, P.slots};
     put_raw(head, sizeof(head));
     put_raw(&P.modulo, sizeof(P.modulo));
+    put_raw(&P.post_offset, sizeof(P.post_offset));
     put_raw(&P.modmask, sizeof(P.modmask));
     for (int s = 0; s < P.nstages; ++s) {
         const DStage &S = P.st[s];

@@ -33,8 +33,8 @@ sjq_status fused_launch(int agg, bool mul, bool hash, int grid, int block, size_
 sjq_status clear_launch(int64_t *sums, int64_t *counts, int64_t cells, int64_t *gkeys, int64_t gslots,
                         int64_t *n_groups, int32_t *status, int sm_count, cudaStream_t stream);
 sjq_status compact_launch(const int64_t *gkeys, const int64_t *gsums, const int64_t *gcounts, int64_t gslots,
-                          int64_t *keys, int64_t *sums, int64_t *counts, int64_t capacity, int64_t *n_groups,
-                          int32_t *status, int sm_count, cudaStream_t stream);
+                          int64_t dense_base, int64_t *keys, int64_t *sums, int64_t *counts, int64_t capacity,
+                          int64_t *n_groups, int32_t *status, int sm_count, cudaStream_t stream);
 
 namespace {
 
@@ -454,21 +454,33 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         }
     }
 
+    // A hashed result whose key is taken modulo M can only hold keys in (-M, M): when 2M - 1 cells fit the
+    // workspace arrays the group table is indexed directly by key + M - 1 (no key array, no hashing, no claim:
+    // two atomics per row instead of a look-up and two atomics; every dense aggregation path applies) and the
+    // compaction recovers the keys from the cell numbers (config 4, G = 10^6 at 10 %: 3.2 -> 1.6 ms).
+    const uint64_t gslots_all = spec->mode == SJQ_HASHED ? hashed_slots(spec->capacity) : 0;
+    const bool direct_groups = spec->mode == SJQ_HASHED && key && key->modulo > 0 && !opts.group_hash_always &&
+                               (uint64_t)key->modulo <= (gslots_all + 1) / 2;
+    const int64_t table_groups = direct_groups ? 2 * key->modulo - 1 : spec->num_groups;
+    if (direct_groups) {
+        P.post_offset = key->modulo - 1;
+        P.want_count = 1; // the counts tell which cells hold a group
+    }
     // ------------------------------------------------------------ aggregation path
     int aggp;
     size_t group_bytes = 0;
     const int approx_grid = dev.sm_count * 2;
     if (spec->mode == SJQ_SCALAR) {
         aggp = AGG_SCALAR;
-    } else if (spec->mode == SJQ_HASHED) {
+    } else if (spec->mode == SJQ_HASHED && !direct_groups) {
         aggp = AGG_HASH;
-    } else if (spec->num_groups == 1) {
+    } else if (spec->mode == SJQ_DENSE && spec->num_groups == 1) {
         aggp = AGG_SCALAR; // a single group: register accumulation, key only range-checked
         P.has_key = 1;
     } else {
-        const size_t gb = (size_t)spec->num_groups * 8 * (P.want_count ? 2 : 1);
+        const size_t gb = (size_t)table_groups * 8 * (P.want_count ? 2 : 1);
         const bool fits = gb <= (size_t)64 << 10;
-        bool contended = survivors / approx_grid >= 8.0 * (double)spec->num_groups;
+        bool contended = survivors / approx_grid >= 8.0 * (double)table_groups;
         if (opts.agg_path == 1) {
             if (!fits) return SJQ_ERR_UNSUPPORTED;
             aggp = AGG_SMEM;
@@ -479,7 +491,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         }
         if (aggp == AGG_SMEM) group_bytes = gb;
     }
-    P.num_groups = spec->mode == SJQ_DENSE ? spec->num_groups : 0;
+    P.num_groups = spec->mode == SJQ_DENSE ? spec->num_groups : direct_groups ? table_groups : 0;
 
     // ------------------------------------------------------------ result buffers
     int64_t *gkeys = nullptr, *gsums = nullptr, *gcounts = nullptr;
@@ -494,7 +506,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         gsums = reinterpret_cast<int64_t *>(static_cast<char *>(out->workspace) + arr);
         gcounts = reinterpret_cast<int64_t *>(static_cast<char *>(out->workspace) + 2 * arr);
         P.gmask = gslots - 1;
-        P.gkeys = gkeys;
+        P.gkeys = direct_groups ? nullptr : gkeys;
         P.sums = gsums;
         P.counts = gcounts;
     } else {
@@ -597,10 +609,13 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     // ------------------------------------------------------------ launches
     int launches = 0;
     if (!opts.accumulate) {
-        int64_t cells = spec->mode == SJQ_SCALAR ? 1 : spec->mode == SJQ_DENSE ? spec->num_groups : (int64_t)gslots + 1;
+        int64_t cells = spec->mode == SJQ_SCALAR ? 1
+                        : spec->mode == SJQ_DENSE ? spec->num_groups
+                        : direct_groups           ? table_groups
+                                                  : (int64_t)gslots + 1;
         st = clear_launch(P.sums, spec->mode == SJQ_HASHED ? gcounts : out->counts, cells, gkeys,
-                          spec->mode == SJQ_HASHED ? (int64_t)gslots + 1 : 0, out->n_groups, out->status,
-                          dev.sm_count, stream);
+                          (spec->mode == SJQ_HASHED && !direct_groups) ? (int64_t)gslots + 1 : 0, out->n_groups,
+                          out->status, dev.sm_count, stream);
         if (st != SJQ_OK) return st;
         ++launches;
     } else if (spec->mode == SJQ_HASHED) {
@@ -618,7 +633,8 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     if (opts.event_after && cudaEventRecord((cudaEvent_t)opts.event_after, stream) != cudaSuccess)
         return SJQ_ERR_CUDA;
     if (spec->mode == SJQ_HASHED) {
-        st = compact_launch(gkeys, gsums, gcounts, (int64_t)gslots, out->keys, out->sums, out->counts, spec->capacity,
+        st = compact_launch(gkeys, gsums, gcounts, direct_groups ? table_groups - 1 : (int64_t)gslots,
+                            direct_groups ? P.post_offset : -1, out->keys, out->sums, out->counts, spec->capacity,
                             out->n_groups, out->status, dev.sm_count, stream);
         if (st != SJQ_OK) return st;
         ++launches;

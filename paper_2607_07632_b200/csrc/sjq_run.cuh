@@ -87,6 +87,7 @@ struct RunParams {
     int64_t n;
     int64_t key_offset;
     int64_t modulo;   // 0 = none
+    int64_t post_offset; // added to the key after the modulo (a hashed result kept as a direct-indexed table)
     uint64_t modmask; // modulo - 1 when modulo is a power of two, else 0
     int64_t num_groups;
     uint64_t gmask; // hashed: group-table slots - 1

@@ -94,7 +94,7 @@ class _RunOpts(ctypes.Structure):
                 ("event_after", ctypes.c_void_p), ("dense_reach_permille", ctypes.c_int32), ("specialise", ctypes.c_int32),
                 ("rows_per_lane", ctypes.c_int32), ("no_filter_bitmap", ctypes.c_int32),
                 ("host_copy_all", ctypes.c_int32), ("dense_slots", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 2)]
+                ("group_hash_always", ctypes.c_int32), ("reserved", ctypes.c_int32 * 1)]
 
 
 class RunInfo(ctypes.Structure):
@@ -128,6 +128,7 @@ class RunOpts:
     no_filter_bitmap: bool = False  # filter stages probe the code array of a direct table, not its bitmap
     host_copy_all: bool = False  # run_host: copy every referenced column instead of reading sparse ones in place
     dense_slots: int = 0  # level 0: 0 auto, 2, or 4 groups of four rows per thread (4 needs specialise)
+    group_hash_always: bool = False  # HASHED: keep the group hash table even when the key domain is small
 
     def to_c(self) -> _RunOpts:
         o = _RunOpts()
@@ -143,6 +144,7 @@ class RunOpts:
         o.no_filter_bitmap = int(self.no_filter_bitmap)
         o.host_copy_all = int(self.host_copy_all)
         o.dense_slots = self.dense_slots
+        o.group_hash_always = int(self.group_hash_always)
         if self.events is not None:
             o.event_before, o.event_after = self.events[0].cuda_event, self.events[1].cuda_event
         return o

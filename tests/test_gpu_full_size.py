@@ -33,8 +33,11 @@ def _run(w):
     tables = sjq.build_workload_tables(w, dims)
     fact = W.device_fact(w)
     results = []
-    for specialise in (True, False):
-        res = sjq.run_workload(w, fact, tables, sjq.RunOpts(specialise=specialise))
+    variants = [sjq.RunOpts(specialise=True), sjq.RunOpts(specialise=False)]
+    if w.mode == "HASHED":  # the group hash table as well as the direct-indexed table a modulo key allows
+        variants.append(sjq.RunOpts(specialise=True, group_hash_always=True))
+    for opts in variants:
+        res = sjq.run_workload(w, fact, tables, opts)
         torch.cuda.synchronize()
         assert res.status() == 0 and all(t.status() == 0 for t in tables.values())
         results.append(res)

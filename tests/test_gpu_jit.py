@@ -47,7 +47,7 @@ def test_random_queries_option_matrix_specialised(seed):
     for opts in (spec(eager_loads=True), spec(smem_tables=1), spec(block_threads=128, ctas_per_sm=1),
                  spec(block_threads=1024, ctas_per_sm=1), spec(block_threads=512, compaction=2, smem_tables=2),
                  spec(agg_path=2), spec(compaction=1), spec(rows_per_lane=8), spec(rows_per_lane=8, compaction=2),
-                 spec(no_filter_bitmap=True), spec(dense_slots=4), spec(dense_slots=4, block_threads=768, ctas_per_sm=1),
+                 spec(no_filter_bitmap=True), spec(group_hash_always=True), spec(dense_slots=4), spec(dense_slots=4, block_threads=768, ctas_per_sm=1),
                  spec(order=tuple(reversed(range(len(w.preds) + len(w.joins)))))):
         res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)
         assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)

@@ -50,6 +50,7 @@ def test_random_queries_option_matrix(seed):
     for opts in (sjq.RunOpts(), sjq.RunOpts(eager_loads=True), sjq.RunOpts(smem_tables=1),
                  sjq.RunOpts(block_threads=128, ctas_per_sm=1), sjq.RunOpts(block_threads=256, compaction=2, smem_tables=1), sjq.RunOpts(agg_path=2),
                  sjq.RunOpts(compaction=2), sjq.RunOpts(compaction=1), sjq.RunOpts(no_filter_bitmap=True),
+                 sjq.RunOpts(group_hash_always=True),
                  sjq.RunOpts(order=tuple(reversed(range(len(w.preds) + len(w.joins)))))):
         res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)
         assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)
@@ -353,3 +354,29 @@ def test_rows_per_lane_eight_needs_the_specialised_kernel():
     assert e.value.status == 1
     with pytest.raises(sjq.SjqError):
         sjq.run_workload(w, to_dev(fact), tables, sjq.RunOpts(rows_per_lane=5, specialise=True))
+
+
+def test_hashed_result_with_a_modulo_key_uses_a_direct_table_when_it_fits():
+    """Keys taken modulo M lie in (-M, M): with room for 2M - 1 cells the group table is indexed by the key
+    (negative keys included), otherwise and on request the hash table is used; same list either way."""
+    rng = np.random.default_rng(77)
+    n = 50_000
+    fact = {"a": rng.integers(-500, 500, n).astype(np.int32), "v": rng.integers(-1000, 1000, n).astype(np.int32)}
+    from qhelpers import adhoc
+    for modulo, capacity, expect in ((37, 200, "direct"), (37, 20, "hash"), (1, 8, "direct"), (0, 2000, "hash")):
+        w = adhoc("modkey", fact, [], [], [Pred("v", "NE", 0)], KeyExpr((Term("FACT", "a", 0, 3),), offset=-7, modulo=modulo),
+                  AggExpr("COL", Term("FACT", "v")), "HASHED", capacity=capacity)
+        exp = oracle.run(w, fact, oracle.build_dims(w, {}), check=False)
+        for opts in (sjq.RunOpts(), sjq.RunOpts(specialise=True), sjq.RunOpts(group_hash_always=True)):
+            res = sjq.run_workload(w, to_dev(fact), {}, opts)
+            torch.cuda.synchronize()
+            if len(exp["keys"]) > capacity:
+                assert res.status() == 19
+                continue
+            assert res.status() == 0
+            compare(w, res, exp)
+            path = res.info.describe()["agg_path"]
+            if expect == "direct" and not opts.group_hash_always:
+                assert path in ("global", "shared")
+            else:
+                assert path == "hash"
