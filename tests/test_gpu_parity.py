@@ -380,3 +380,29 @@ def test_hashed_result_with_a_modulo_key_uses_a_direct_table_when_it_fits():
                 assert path in ("global", "shared")
             else:
                 assert path == "hash"
+
+
+@pytest.mark.parametrize("groups", [1000, 100000])
+def test_hashed_accumulate_and_host_path_equal_whole(groups):
+    """A hashed result accumulated over two calls, and over the chunks of the host-buffer entry point, equals the
+    single run (both forms of the group table: indexed by the modulo key, and the hash table)."""
+    w = W.config4(400_003, 0.5, groups, hashed=True, dim_rows=50000)
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    for opts_kw in ({}, {"group_hash_always": True}, {"specialise": True}):
+        res, exp, tables = run_both(w, fact, hd, opts=sjq.RunOpts(**opts_kw))
+        compare(w, res, exp)
+        k = 150_001
+        a = to_dev({c: v[:k] for c, v in fact.items()})
+        b = to_dev({c: v[k:].copy() for c, v in fact.items()})
+        r = sjq.run_workload(replace(w, n_rows=k), a, tables, sjq.RunOpts(**opts_kw))
+        r = sjq.run_workload(replace(w, n_rows=w.n_rows - k), b, tables, sjq.RunOpts(accumulate=True, **opts_kw), result=r)
+        torch.cuda.synchronize()
+        compare(w, r, exp)
+        pinned = {c: torch.from_numpy(np.ascontiguousarray(v)).pin_memory() for c, v in fact.items()}
+        chunk = 65536
+        staging = torch.empty(sjq.staging_bytes(pinned, chunk), dtype=torch.uint8, device="cuda:0")
+        rh, host = sjq.run_workload_host(w, pinned, tables, staging, chunk, sjq.RunOpts(**opts_kw))
+        torch.cuda.synchronize()
+        assert int(host.status[0]) == 0
+        compare(w, rh, exp)
