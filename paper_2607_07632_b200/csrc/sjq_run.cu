@@ -231,7 +231,8 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     auto add_term = [&](const sjq_term &t, int dest, int64_t sign) {
         contrib.push_back({t.src, t.a, t.b, dest, (int64_t)((uint64_t)t.mult * (uint64_t)sign)});
     };
-    if (key)
+    // a key taken modulo 1 is 0 whatever its terms are: they are neither loaded nor gathered
+    if (key && key->modulo != 1)
         for (int t = 0; t < key->nterms; ++t) add_term(key->t[t], kAccKey, 1);
     const bool mul = agg->op == SJQ_AGG_MUL;
     add_term(agg->x, kAccX, 1);
@@ -738,7 +739,7 @@ void host_transfer_plan(const sjq_col *fact_host, int nfact, const sjq_pred *pre
     auto use = [&](const sjq_term &t) {
         if (t.src == SJQ_SRC_FACT && need[t.a] < 0) need[t.a] = reach;
     };
-    if (key)
+    if (key && key->modulo != 1) // (modulo 1: the planner drops the key's terms)
         for (int t = 0; t < key->nterms; ++t) use(key->t[t]);
     use(agg->x);
     if (agg->op != SJQ_AGG_COL) use(agg->y);

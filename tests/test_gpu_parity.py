@@ -406,3 +406,24 @@ def test_hashed_accumulate_and_host_path_equal_whole(groups):
         torch.cuda.synchronize()
         assert int(host.status[0]) == 0
         compare(w, rh, exp)
+
+
+def test_key_modulo_one_ignores_its_terms():
+    """x % 1 is 0 for every x: the key's columns are not read, the result is the one group 0 (dense or hashed),
+    and a column that only the key names is not transferred by the host path."""
+    from qhelpers import adhoc
+    rng = np.random.default_rng(5)
+    n = 30_000
+    fact = {"g": rng.integers(-(1 << 30), 1 << 30, n).astype(np.int32), "v": rng.integers(-50, 50, n).astype(np.int32)}
+    for mode, kw in (("DENSE", dict(num_groups=1)), ("HASHED", dict(capacity=4))):
+        w = adhoc("mod1", fact, [], [], [Pred("v", "GT", -40)], KeyExpr((Term("FACT", "g"),), offset=5, modulo=1),
+                  AggExpr("COL", Term("FACT", "v")), mode, **kw)
+        exp = oracle.run(w, fact, oracle.build_dims(w, {}))
+        for opts in (sjq.RunOpts(), sjq.RunOpts(specialise=True)):
+            res = sjq.run_workload(w, to_dev(fact), {}, opts)
+            torch.cuda.synchronize()
+            assert res.status() == 0
+            compare(w, res, exp)
+        pinned = {k: torch.from_numpy(v).pin_memory() for k, v in fact.items()}
+        plan = sjq.host_transfer_plan(pinned, w.preds, [], w.key, w.agg)
+        assert plan["g"][0] == "not transferred" and plan["v"][0] == "copy"
