@@ -93,36 +93,50 @@ def algorithmic_bytes_per_row(w, order):
 
 
 class ClockSampler(threading.Thread):
-    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs.  NVML is
+    initialised before the thread starts, so that a short timed region is covered from its first milliseconds
+    (an NVML query takes milliseconds: it must not sit in the timing loop itself)."""
 
     def __init__(self, index: int):
         super().__init__(daemon=True)
         self.index, self.stop_flag, self.samples, self.reasons, self.max_mhz = index, False, [], set(), None
         self.error = None
-
-    def run(self):
+        self.nv = self.handle = None
+        self.names = {}
         try:
             import pynvml as nv
 
             nv.nvmlInit()
-            h = nv.nvmlDeviceGetHandleByIndex(self.index)
-            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
-            names = {nv.nvmlClocksEventReasonHwSlowdown: "hw_slowdown",
-                     nv.nvmlClocksEventReasonHwThermalSlowdown: "hw_thermal_slowdown",
-                     nv.nvmlClocksEventReasonSwThermalSlowdown: "sw_thermal_slowdown",
-                     nv.nvmlClocksEventReasonSwPowerCap: "sw_power_cap"}
-            while not self.stop_flag:
-                self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
-                try:
-                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
-                except Exception:
-                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
-                for bit, nm in names.items():
-                    if r & bit:
-                        self.reasons.add(nm)
-                time.sleep(0.01)
+            self.nv = nv
+            self.handle = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(self.handle, nv.NVML_CLOCK_SM)
+            self.names = {nv.nvmlClocksEventReasonHwSlowdown: "hw_slowdown",
+                          nv.nvmlClocksEventReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                          nv.nvmlClocksEventReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                          nv.nvmlClocksEventReasonSwPowerCap: "sw_power_cap"}
         except Exception as e:  # pragma: no cover - depends on the box
             self.error = repr(e)
+
+    def sample(self):
+        if self.handle is None:
+            return
+        try:
+            nv = self.nv
+            self.samples.append(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
+            try:
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+            except Exception:
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle)
+            for bit, nm in self.names.items():
+                if r & bit:
+                    self.reasons.add(nm)
+        except Exception as e:  # pragma: no cover
+            self.error = repr(e)
+
+    def run(self):
+        while not self.stop_flag:
+            self.sample()
+            time.sleep(0.01)
 
     def summary(self):
         if not self.samples:
