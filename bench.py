@@ -6,11 +6,17 @@
 
 A step is one whole query: plan and build every dimension table from the
 filtered dimension columns, then one fused pass over the fact table (and, for
-N > 1, an all-reduce of the dense result).  The workload is the four-join
+N > 1, the merge of the per-rank results: one all-reduce, or for a hashed
+result one all-gather and a merge kernel).  The workload is the four-join
 group-by over 600 M fact rows (14.4 GB of referenced fact columns, far larger
 than the 126 MB L2, so no L2 flush is needed between steps); every rank holds
 its own 600 M-row shard of the row space and a replica of the dimensions
-(weak scaling).  Rank 0 prints ONE JSON line.
+(weak scaling; `--scaling strong` cuts one 1.2 B-row table over the ranks
+instead).  Rank 0 prints ONE JSON line.  At N = 1 the line also carries
+`points`: every other configuration (config 1, 2, 5, the 20 points of the
+selectivity x cardinality sweep, the two high-cardinality shapes), each run
+ten times or more with its own roofline figures, clock record and a bit-exact
+comparison with the oracle-written expected values under tests/golden/.
 """
 from __future__ import annotations
 
@@ -30,8 +36,27 @@ UNIT = "rows/s"
 CONTRACT_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per fact row of the fused kernel, from an ncu capture of a 100 M-row case of the same workload
-# (dram__bytes_read.sum + dram__bytes_write.sum; traffic grows in proportion to the rows)
-NCU_DRAM_BYTES_PER_ROW = {"c3": 12.2}
+# (dram__bytes_read.sum + dram__bytes_write.sum; traffic grows in proportion to the rows), each with the plan
+# it was captured under: the figure is reported only while the running plan is that one.
+NCU_PROFILED = {
+    "c3_four_join_groupby": {"dram_bytes_per_row": 12.2, "kernel": "sjq_jit_kernel",
+                             "order": [1, 3, 0, 2, 3, 0, -1, -1], "block": 1024, "queue_levels": 3,
+                             "summary": "profiles/fused_kernel_c3_100m.md"},
+}
+
+
+def profiled_traffic(w, info, kernel, rows):
+    """(bytes per launch, note): the ncu DRAM traffic scaled to `rows`, or None when the plan that ran is not
+    the plan the capture was taken under."""
+    p = NCU_PROFILED.get(w.name)
+    if p is None:
+        return None, "no capture of this workload"
+    plan = info.describe()
+    same = (plan["order"] == p["order"] and plan["block"] == p["block"] and plan["queue_levels"] == p["queue_levels"]
+            and kernel == p["kernel"])
+    if not same:
+        return None, f"the plan that ran differs from the one captured in {p['summary']}"
+    return p["dram_bytes_per_row"] * rows, p["summary"]
 
 
 def measured_hbm_peak():
@@ -47,32 +72,71 @@ def make_workload(name: str, rows: int | None, sel: float, groups: int):
 
     if name == "c4":
         return W.config4(rows or 600_000_000, sel, groups)
-    return W.CONFIGS[name](rows) if rows else W.CONFIGS[name]()
+    mk = W.CONFIGS.get(name) or W.EXTRA_SHAPES[name]
+    return mk(rows) if rows else mk()
 
 
-def stage_selectivities(w):
-    """Exact pass fractions of the workload's filters, from its definition (uniform draws)."""
-    from datagen import DATE_ROWS
+def _uniform_pred_fraction(c, p):
+    """Exact share of U[a, b] that passes predicate p (None when the column is not a plain uniform draw)."""
+    from datagen import UNIFORM_I32
 
-    sel = {}
-    if w.name.startswith("c1"):
-        sel = {"pred:discount": 3 / 11, "pred:quantity": 29 / 50, "join:date": 365 / DATE_ROWS}
-    elif w.name.startswith("c2"):
-        sel = {"join:part": 1 / 25, "join:supplier": 1 / 5, "join:date": 1.0}
-    elif w.name.startswith("c3"):
-        sel = {"join:customer": 1 / 5, "join:supplier": 1 / 5, "join:part": 2 / 5, "join:date": 729 / DATE_ROWS}
-    elif w.name.startswith("c4"):
-        sel = {"pred:p": w.preds[0].lo / 10000.0, "join:dim": 1.0}
-    elif w.name.startswith("c5"):
-        sel = {"join:dim": 0.25}
-    return sel
+    if c.kind != UNIFORM_I32:
+        return None
+    a, b = c.a, c.b
+    n = b - a + 1
+
+    def below(x):  # values of [a, b] that are < x
+        return min(max(x - a, 0), n)
+
+    if p.op == "EQ":
+        k = 1 if a <= p.lo <= b else 0
+    elif p.op == "NE":
+        k = n - (1 if a <= p.lo <= b else 0)
+    elif p.op == "LT":
+        k = below(p.lo)
+    elif p.op == "LE":
+        k = below(p.lo + 1)
+    elif p.op == "GT":
+        k = n - below(p.lo + 1)
+    elif p.op == "GE":
+        k = n - below(p.lo)
+    elif p.op == "BETWEEN":
+        k = max(0, min(b, p.hi) - max(a, p.lo) + 1)
+    else:
+        k = len({v for v in p.values if a <= v <= b})
+    return k / n
 
 
-def algorithmic_bytes_per_row(w, order):
+def stage_pass_fractions(w, tables, survivors=None):
+    """Pass fraction of every filter of the workload, label -> fraction, labels as in the plan's `order`
+    (predicate index, then number of predicates + join index).  Predicates on uniform columns and joins whose
+    foreign key is drawn uniformly over the dimension's rows are exact by construction (rows passing the
+    dimension filter / rows of the dimension, as the built table reports them); one remaining unknown (the
+    Zipf-distributed key of config 5) is solved from the survivor count of the run."""
+    from datagen import DATE_FK_I32, SEQ_I32, DATE_KEY_I32, UNIFORM_I32
+
+    frac = {}
+    for i, p in enumerate(w.preds):
+        frac[i] = _uniform_pred_fraction(w.fact_col(p.col), p)
+    for j, (fk, dn) in enumerate(w.joins):
+        c, d, L = w.fact_col(fk), w.dim(dn), tables[dn].layout
+        key_kind = next(x.kind for x in d.cols if x.name == d.key)
+        uniform = (c.kind == UNIFORM_I32 and key_kind == SEQ_I32 and c.a == 1 and c.b == d.rows) or \
+                  (c.kind == DATE_FK_I32 and key_kind == DATE_KEY_I32)
+        frac[len(w.preds) + j] = (L.entries / L.dim_rows) if (uniform and L.dim_rows) else None
+    unknown = [k for k, v in frac.items() if v is None]
+    if len(unknown) == 1 and survivors is not None and w.n_rows:
+        known = 1.0
+        for v in frac.values():
+            known *= v if v is not None else 1.0
+        frac[unknown[0]] = min(1.0, survivors / w.n_rows / known) if known > 0 else 1.0
+    return {k: (1.0 if v is None else v) for k, v in frac.items()}
+
+
+def algorithmic_bytes_per_row(w, order, frac):
     """Sector model: the first column is read whole; a later column is read for a 32-byte sector
-    iff at least one of its rows survived everything evaluated before it."""
-    sel = stage_selectivities(w)
-    names = [f"pred:{p.col}" for p in w.preds] + [f"join:{d}" for _, d in w.joins]
+    iff at least one of its rows survived everything evaluated before it.  `order`: the stage labels of
+    the plan that ran; `frac`: pass fraction per label."""
     cols = [p.col for p in w.preds] + [fk for fk, _ in w.joins]
     reach, total, seen, applied = 1.0, 0.0, set(), set()
     for idx in order:
@@ -84,9 +148,11 @@ def algorithmic_bytes_per_row(w, order):
         if col not in seen:
             total += width * (1.0 - (1.0 - reach) ** (32 // width))
             seen.add(col)
-        reach *= sel.get(names[idx], 1.0)
+        reach *= frac.get(idx, 1.0)
+    referenced = set(cols) | {t.a for t in ((w.key.terms if w.key and w.key.modulo != 1 else ()) + (w.agg.x,) +
+                                            ((w.agg.y,) if w.agg.y is not None else ())) if t.src == "FACT"}
     for c in w.fact_cols:  # columns only the key or the aggregate reads
-        if c.name not in seen:
+        if c.name not in seen and c.name in referenced:
             width = 8 if c.is64 else 4
             total += width * (1.0 - (1.0 - reach) ** (32 // width))
     return total
@@ -213,14 +279,182 @@ def run_reference(args):
     return 0
 
 
+def golden_for(w):
+    """Expected result written by the CPU oracle for this workload at this size (tests/golden/full_*.json), or None."""
+    from datagen import workloads as W
+
+    if w.name.startswith("c4_sweep"):
+        sel = next(s for s, t in W.C4_THRESHOLDS.items() if t == w.preds[0].lo)
+        tag = f"c4_s{sel:g}_g{w.key.modulo}"
+    else:
+        tag = {"c1_filter_agg": "c1", "c2_two_join_groupby": "c2", "c3_four_join_groupby": "c3",
+               "c5_skewed_sparse": "c5", "city_pair_groupby": "city_pair", "city_brand_groupby": "city_brand",
+               "city_brand_groupby_dense": "city_brand"}.get(w.name)
+    path = os.path.join(ROOT, "tests", "golden", f"full_{tag}.json")
+    if tag is None or not os.path.exists(path):
+        return None
+    with open(path) as f:
+        g = json.load(f)
+    return g if g["rows"] == w.n_rows else None
+
+
+def matches_golden(w, res, g):
+    """True iff the device result equals the stored expected values bit for bit (None: nothing stored)."""
+    import hashlib
+
+    import numpy as np
+
+    if g is None:
+        return None
+    if w.mode == "SCALAR":
+        return int(res.sums[0].item()) == g["sum"] and int(res.counts[0].item()) == g["count"]
+
+    def digest(*arrays):
+        h = hashlib.sha256()
+        for a in arrays:
+            h.update(np.ascontiguousarray(a, dtype="<i8").tobytes())
+        return h.hexdigest()
+
+    if w.mode == "DENSE":
+        s, c = res.sums.cpu().numpy(), res.counts.cpu().numpy()
+        if "sums" in g:
+            return s.tolist() == g["sums"] and c.tolist() == g["counts"]
+        if g.get("mode") == "HASHED":  # stored as a list: compare the non-empty groups of the dense array
+            keys = np.nonzero(c)[0]
+            return keys.size == g["groups"] and digest(keys, s[keys], c[keys]) == g["sha256"]
+        return digest(s, c) == g["dense_sha256"]
+    k, s, c = (t.cpu().numpy() for t in res.hashed_sorted())
+    if "sha256" in g:
+        return k.size == g["groups"] and digest(k, s, c) == g["sha256"]
+    # stored as a dense array: scatter the list
+    full_s, full_c = np.zeros(w.num_groups, np.int64), np.zeros(w.num_groups, np.int64)
+    full_s[k], full_c[k] = s, c
+    return digest(full_s, full_c) == g["dense_sha256"]
+
+
+def measure_point(sjq, torch, w, fact, tables, specialise, gpu_index, peak, extra_opts=None, min_runs=10,
+                  min_busy_ms=60.0):
+    """Run-only measurement of one workload (tables prebuilt): at least `min_runs` calls of sjq_run enqueued
+    back to back (more, until the GPU has been busy for `min_busy_ms`, so that the clock sampler sees the
+    point under load), each timed with its own CUDA events: the whole call (clear + fused kernel + compaction)
+    and the fused kernel alone."""
+    kw = dict(extra_opts or {})
+    res = sjq.run_workload(w, fact, tables, sjq.RunOpts(specialise=specialise, **kw))
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    sjq.run_workload(w, fact, tables, sjq.RunOpts(specialise=specialise, **kw), result=res)
+    e1.record()
+    torch.cuda.synchronize()
+    runs = int(min(200, max(min_runs, min_busy_ms / max(e0.elapsed_time(e1), 1e-3))))
+    ref_bytes = w.referenced_bytes_per_row()
+    small = w.n_rows * ref_bytes < (512 << 20)  # may sit in the 126 MB L2: evict it between runs
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=res.sums.device) if small else None
+    outer = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(runs)]
+    inner = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(runs)]
+    for a, b in inner:
+        a.record()
+        b.record()
+    sampler = ClockSampler(gpu_index)
+    torch.cuda.synchronize()
+    sampler.sample()
+    sampler.start()
+    for i in range(runs):
+        if flush is not None:
+            flush.zero_()
+        outer[i][0].record()
+        sjq.run_workload(w, fact, tables, sjq.RunOpts(specialise=specialise, events=inner[i], **kw), result=res)
+        outer[i][1].record()
+    torch.cuda.synchronize()
+    sampler.sample()
+    sampler.stop_flag = True
+    sampler.join(timeout=2.0)
+    ms = [a.elapsed_time(b) for a, b in outer]
+    kms = [a.elapsed_time(b) for a, b in inner]
+    status = res.status()
+    info = res.info
+    if w.mode == "HASHED":
+        survivors = int(res.counts[: int(res.n_groups.item())].sum().item())
+    else:
+        survivors = int(res.counts.sum().item()) if res.counts is not None else None
+    frac = stage_pass_fractions(w, tables, survivors)
+    plan = info.describe()
+    alg = algorithmic_bytes_per_row(w, plan["order"], frac)
+    ms_mean, k_mean = sum(ms) / runs, sum(kms) / runs
+    achieved = w.n_rows * alg / (k_mean / 1000.0) / 1e9
+    eff = w.n_rows * ref_bytes / (k_mean / 1000.0) / 1e9
+    out = {"workload": w.name, "rows": w.n_rows, "runs": runs, "ms_min": min(ms), "ms_mean": ms_mean,
+           "kernel_ms_min": min(kms), "kernel_ms_mean": k_mean, "rows_per_s": w.n_rows / (ms_mean / 1000.0),
+           "algorithmic_bytes_per_row": alg, "achieved_gbs": achieved, "frac": achieved / peak,
+           "referenced_bytes_per_row": ref_bytes, "effective_gbs_kernel": eff,
+           "pct_of_8tbs": 100.0 * eff / CONTRACT_HBM_GBS, "survivors": survivors,
+           "pass_fractions": {str(k): round(v, 6) for k, v in frac.items()},
+           "l2": "256 MB written between runs" if small else "inputs exceed the L2",
+           "status": status, "parity": matches_golden(w, res, golden_for(w)) if status == 0 else False,
+           "plan": plan, "table_kinds": {k: t.layout.kind_name for k, t in tables.items()},
+           "clocks": sampler.summary()}
+    if plan["agg_path"] in ("global", "hash") and survivors is not None:
+        # one 64-bit atomic add per survivor for the sum and one for the count where counts are kept
+        per_row = 2 if (w.agg.want_count or w.mode == "HASHED") else 1
+        out["atomic_adds_per_s"] = survivors * per_row / (k_mean / 1000.0)
+    return out
+
+
+def run_points(sjq, torch, W, device, specialise, gpu_index, peak, c3_inputs=None, extras=False):
+    """Every configuration besides the headline one, run-only, each with its own figures and parity."""
+    out = []
+
+    def inputs(w):
+        dims = {d.name: W.device_dim(w, d, device) for d in w.dims}
+        return W.device_fact(w, device=device), sjq.build_workload_tables(w, dims)
+
+    def point(w, fact=None, tables=None, **kw):
+        if fact is None:
+            fact, tables = inputs(w)
+        try:
+            out.append(measure_point(sjq, torch, w, fact, tables, specialise, gpu_index, peak, **kw))
+        except Exception as ex:  # one failing point must not hide the others
+            out.append({"workload": w.name, "rows": w.n_rows, "error": repr(ex)[:300], "parity": False})
+        return fact, tables
+
+    if c3_inputs is not None:
+        point(*c3_inputs)
+        c3_inputs[1].clear()  # the caller's columns are not needed any more: free them
+        torch.cuda.empty_cache()
+    for mk in (W.config1, W.config2, W.config5, W.city_pair, W.city_brand):
+        point(mk())
+        torch.cuda.empty_cache()
+    if extras:
+        point(W.city_brand(hashed=False))  # the same query asked for as the dense array of all 1.75 M groups
+        torch.cuda.empty_cache()
+    # the sweep: its four fact columns and its dimension do not depend on the threshold or the group count
+    fact = tables = None
+    for s in W.C4_THRESHOLDS:
+        for g in W.C4_GROUPS:
+            fact, tables = point(W.config4(600_000_000, s, g), fact, tables)
+    if extras:
+        # the large group counts as DENSE results too (no key list), and through the group hash table
+        for s in (0.1, 1.0):
+            for g in (100000, 1000000):
+                point(W.config4(600_000_000, s, g, hashed=False), fact, tables)
+                point(W.config4(600_000_000, s, g), fact, tables, extra_opts={"group_hash_always": True})
+    del fact, tables
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4", "c5"])
-    ap.add_argument("--rows", type=int, default=None, help="override the fact rows per GPU (debugging)")
+    ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4", "c5", "city_pair", "city_brand"])
+    ap.add_argument("--rows", type=int, default=None,
+                    help="fact rows per GPU (weak scaling) or of the whole table (strong scaling); default: the "
+                         "configuration's size, 1.2 B rows for --scaling strong")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="weak: every rank owns its own rows; strong: one table cut into contiguous row ranges")
     ap.add_argument("--sel", type=float, default=0.1, help="c4: fact predicate selectivity")
     ap.add_argument("--groups", type=int, default=1000, help="c4: number of groups")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -232,9 +466,11 @@ def main():
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--extras", action="store_true", help="also time the other configurations (N = 1 only)")
+    ap.add_argument("--no-points", action="store_true", help="skip the other configurations (N = 1 runs them by default)")
+    ap.add_argument("--extras", action="store_true", help="more points: large group counts as dense arrays and through the hash table")
     ap.add_argument("--ablation", action="store_true",
-                    help="also run the A/B switches (lazy vs eager loads, queues, table forms, group-by paths)")
+                    help="also run the A/B switches (lazy vs eager loads, queues, table forms, group-by paths, "
+                         "operator-at-a-time)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -263,10 +499,13 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=device)
 
-    w = make_workload(args.workload, args.rows, args.sel, args.groups)
-    n = w.n_rows
+    rows = args.rows if args.rows else (1_200_000_000 if args.scaling == "strong" else None)
+    w = make_workload(args.workload, rows, args.sel, args.groups)
+    row0, n = shard.rank_rows(rank, world, w.n_rows, args.scaling)  # this rank's part of the row space
+    total_rows = w.n_rows * world if args.scaling == "weak" else w.n_rows
+    w_local = W.with_rows(w, n)
     dims = {d.name: W.device_dim(w, d, device) for d in w.dims}
-    fact = W.device_fact(w, row0=rank * n, n=n, device=device)  # this rank's shard of the row space
+    fact = W.device_fact(w, row0=row0, n=n, device=device)
     torch.cuda.synchronize()
 
     # every event pair is created (recorded once) up front; the library records them around the fused kernel
@@ -279,17 +518,20 @@ def main():
     builders = sjq.workload_builders(w, dims)  # argument marshalling done once; plan + build run every step
     launches = 0
     info = None
+    merged = None
 
     def step(i=None):
-        nonlocal launches, info
+        nonlocal launches, info, merged
         tables = sjq.build_tables(builders)
         opts = sjq.RunOpts(events=pairs[i] if i is not None else None, specialise=not args.interpret,
                            block_threads=args.block_threads, ctas_per_sm=args.ctas_per_sm)
-        r = sjq.run_workload(w, fact, tables, opts, result=res)
-        if world > 1 and w.mode != "HASHED":
-            shard.merge_dense(res.sums, res.counts)
+        r = sjq.run_workload(w_local, fact, tables, opts, result=res)
+        if world > 1:
+            merged = shard.merge_result(res)
         if i is not None:
             launches += r.info.kernel_launches + sum(sjq.build_launches(t) for t in tables.values())
+            if world > 1 and w.mode == "HASHED":
+                launches += 3  # clear, merge and compaction kernels of sjq_merge_groups
         info = r.info
         return tables
 
@@ -309,7 +551,8 @@ def main():
     torch.cuda.synchronize()
     assert res.status() == 0 and all(t.status() == 0 for t in tables.values())
 
-    sampler = ClockSampler(visible_gpu_index(local_rank))
+    gpu_index = visible_gpu_index(local_rank)
+    sampler = ClockSampler(gpu_index)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if world > 1:
         dist.barrier()
@@ -317,7 +560,7 @@ def main():
     sampler.start()
     ev0.record()
     for i in range(args.steps):
-        step(i)
+        tables = step(i)
     ev1.record()
     if world > 1:
         dist.barrier()
@@ -331,18 +574,26 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     ms_total, fused_ms = float(t[0]), float(t[1])
     ms_per_step = ms_total / args.steps
-    value = world * n / (ms_per_step / 1000.0)
+    value = total_rows / (ms_per_step / 1000.0)
     ref_bytes = w.referenced_bytes_per_row()
-    eff_gbs = world * n * ref_bytes / (ms_per_step / 1000.0) / 1e9
+    eff_gbs = total_rows * ref_bytes / (ms_per_step / 1000.0) / 1e9
+    parity = matches_golden(w, res, golden_for(w)) if world == 1 else None
 
     peak, peak_kind = measured_hbm_peak()
-    alg_bpr = algorithmic_bytes_per_row(w, list(info.order[: info.nstages]))
+    if w.mode == "HASHED":
+        survivors = int(res.counts[: int(res.n_groups.item())].sum().item())
+    else:
+        survivors = int(res.counts.sum().item()) if res.counts is not None else None
+    pass_frac = stage_pass_fractions(w_local, tables, survivors)
+    alg_bpr = algorithmic_bytes_per_row(w, list(info.order[: info.nstages]), pass_frac)
     achieved = n * alg_bpr / (fused_ms / 1000.0) / 1e9
-    traffic_bpr = NCU_DRAM_BYTES_PER_ROW.get(args.workload)
-    roofline = {"bound": "hbm", "kernel": "fused_kernel" if args.interpret else "sjq_jit_kernel", "achieved": achieved, "peak": peak,
+    kernel_name = "fused_kernel" if args.interpret else "sjq_jit_kernel"
+    traffic, traffic_note = profiled_traffic(w, info, kernel_name, n)
+    roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                "traffic": traffic_bpr * n if traffic_bpr else None,
+                "traffic": traffic, "traffic_source": traffic_note,
                 "algorithmic_bytes_per_row": alg_bpr, "kernel_ms": fused_ms,
+                "pass_fractions": {str(k): round(v, 6) for k, v in pass_frac.items()},
                 "effective_gbs_kernel": n * ref_bytes / (fused_ms / 1000.0) / 1e9}
 
     e2e = None
@@ -351,6 +602,9 @@ def main():
             host_fact = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in fact.items()}
             for k, v in fact.items():
                 host_fact[k].copy_(v)
+            host_dims = {dn: {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in cols.items()}
+                         for dn, cols in dims.items()}
+            dim_bytes = sum(v.numel() * v.element_size() for cols in host_dims.values() for v in cols.values())
             torch.cuda.synchronize()
             chunk = min(n, 32 << 20) // 4 * 4 or 4
             staging = torch.empty(sjq.staging_bytes(host_fact, chunk), dtype=torch.uint8, device=device)
@@ -358,8 +612,13 @@ def main():
 
             def e2e_step():
                 nonlocal eres, ehost
+                for dn, cols in host_dims.items():  # the dimension columns come from the host too
+                    for k, v in cols.items():
+                        dims[dn][k].copy_(v, non_blocking=True)
+                for b in builders.values():  # the key-range scans run on side streams: after the copies
+                    b.side.wait_stream(torch.cuda.current_stream(device))
                 tabs = sjq.build_tables(builders)
-                eres, ehost = sjq.run_workload_host(w, host_fact, tabs, staging, chunk,
+                eres, ehost = sjq.run_workload_host(w_local, host_fact, tabs, staging, chunk,
                                                     sjq.RunOpts(specialise=not args.interpret), result=eres, host=ehost)
                 torch.cuda.synchronize()  # the result is on the host when this returns
                 return tabs
@@ -375,7 +634,9 @@ def main():
             if world > 1:
                 dist.all_reduce(tt, op=dist.ReduceOp.MAX)
             dt = float(tt[0])
-            same = bool(torch.equal(ehost.sums, res.sums.cpu())) if world == 1 else None
+            same = None
+            if world == 1 and w.mode != "HASHED":
+                same = bool(torch.equal(ehost.sums, res.sums.cpu()))
             cells = 1 if w.mode == "SCALAR" else w.num_groups if w.mode == "DENSE" else w.capacity
             # bytes over the bus: whole columns for the copied ones; for a column the kernel reads in place, the
             # 32-byte sectors holding a surviving row (estimated from the planner's share of rows reaching it)
@@ -385,16 +646,24 @@ def main():
             copied = sum(n * host_fact[k].element_size() for k, (how, _) in plan.items() if how == "copy")
             in_place = sum(n * host_fact[k].element_size() * (1.0 - (1.0 - sh) ** (32 // host_fact[k].element_size()))
                            for k, (how, sh) in plan.items() if how == "in place")
-            e2e = {"value": world * n / dt, "unit": UNIT, "h2d_bytes_per_step": int(copied + in_place),
-                   "h2d_copied_bytes": int(copied), "h2d_in_place_bytes_estimate": int(in_place),
+            e2e = {"value": total_rows / dt, "unit": UNIT, "h2d_bytes_per_step": int(copied + in_place + dim_bytes),
+                   "h2d_copied_bytes": int(copied), "h2d_dimension_bytes": int(dim_bytes),
+                   "h2d_in_place_bytes_estimate": int(in_place),
+                   "h2d_in_place_note": "sector-model estimate from the planner's shares, not a counter",
                    "columns": {k: how for k, (how, _) in plan.items()},
                    "d2h_bytes_per_step": cells * 8 * (2 if w.agg.want_count else 1) + 4, "ms_per_step": dt * 1000.0,
                    "steps": args.e2e_steps, "chunk_rows": chunk, "matches_device_run": same,
                    "api": "sjq_run_host (pinned host columns: chunked double-buffered copies of the columns most rows need, "
-                          "in-place reads of the sparse ones, result copied back)"}
-            del host_fact, staging
+                          "in-place reads of the sparse ones, result copied back); dimension columns copied from pinned "
+                          "host memory every step before the table builds"}
+            del host_fact, staging, host_dims
         except Exception as ex:  # e.g. not enough page-locked memory on the box
             e2e = {"value": None, "unit": UNIT, "error": repr(ex)[:200]}
+
+    points = None
+    if world == 1 and rank == 0 and not args.no_points:
+        c3_inputs = (w, fact, tables) if (args.workload == "c3" and not args.rows) else None
+        points = run_points(sjq, torch, W, device, not args.interpret, gpu_index, peak, c3_inputs, extras=args.extras)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -404,85 +673,40 @@ def main():
                "sample": f"first {sample} fact rows of the workload; row loop {secs:.2f} s + dimension maps {tb:.2f} s",
                "host_cores_available": os.cpu_count()}
 
-    extras = None
-    if args.extras and world == 1 and rank == 0:
-        del fact
-        torch.cuda.empty_cache()
-        extras = run_extras(sjq, W, device, not args.interpret)
     ablation = None
     if args.ablation and world == 1 and rank == 0:
-        if "fact" in locals():
-            del fact
+        fact.clear()
         torch.cuda.empty_cache()
         ablation = run_ablation(sjq, W, device, not args.interpret)
 
     if rank == 0:
+        exchange = ""
+        if world > 1:
+            exchange = (", then all-gather of the per-rank group lists and a merge kernel" if w.mode == "HASHED"
+                        else ", then one all-reduce of the joined sums, counts and status words")
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": args.scaling,
                 "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-                "config": {"workload": w.name, "rows_per_gpu": n, "referenced_bytes_per_row": ref_bytes,
+                "config": {"workload": w.name, "rows_per_gpu": n, "rows_total": total_rows,
+                           "referenced_bytes_per_row": ref_bytes,
                            "step": "plan+build of every dimension table (on side streams; the key-range scans may overlap the previous step's fused pass), then the fused pass"
-                                   + (", then all-reduce of the dense result" if world > 1 else ""),
+                                   + exchange,
                            "l2": "inputs (%.1f GB) exceed the 126 MB L2; no flush needed" % (n * ref_bytes / 1e9),
                            "parallelism": f"row-sharded x{world}, dimensions replicated", "plan": info.describe(),
                            "fused_kernel": "interpreted descriptor" if args.interpret else
                                            "compiled for the query's shape at run time during warm-up (NVRTC), cached"},
                 "effective_gbs": eff_gbs, "pct_of_8tbs": 100.0 * eff_gbs / world / CONTRACT_HBM_GBS,
-                "pct_of_measured_copy_peak": 100.0 * eff_gbs / world / peak,
+                "pct_of_measured_copy_peak": 100.0 * eff_gbs / world / peak, "parity": parity,
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
                 "clocks": sampler.summary()}
-        if extras is not None:
-            line["other_configs"] = extras
+        if points is not None:
+            line["points"] = points
         if ablation is not None:
             line["ablation"] = ablation
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
     return 0
-
-
-def run_extras(sjq, W, device, specialise=True):
-    """Run-only timings (tables prebuilt) of the other configurations: min and mean of 10 after a warm-up."""
-    import torch
-
-    out = []
-
-    def timed(w):
-        dims = {d.name: W.device_dim(w, d, device) for d in w.dims}
-        tables = sjq.build_workload_tables(w, dims)
-        fact = W.device_fact(w, device=device)
-        opts = sjq.RunOpts(specialise=specialise)
-        res = sjq.run_workload(w, fact, tables, opts)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ts = []
-        for _ in range(10):
-            e0.record()
-            sjq.run_workload(w, fact, tables, opts, result=res)
-            e1.record()
-            torch.cuda.synchronize()
-            ts.append(e0.elapsed_time(e1))
-        eff = w.n_rows * w.referenced_bytes_per_row() / (min(ts) / 1000.0) / 1e9
-        out.append({"workload": w.name, "rows": w.n_rows, "ms_min": min(ts), "ms_mean": sum(ts) / len(ts),
-                    "rows_per_s": w.n_rows / (min(ts) / 1000.0), "effective_gbs": eff,
-                    "pct_of_8tbs": 100.0 * eff / CONTRACT_HBM_GBS, "status": res.status(),
-                    "plan": res.info.describe()})
-        del fact, tables, dims, res
-        torch.cuda.empty_cache()
-
-    timed(W.config1())
-    timed(W.config2())
-    timed(W.config5())
-    timed(W.city_pair())  # beyond the five configurations: many groups, few survivors
-    for s in (0.0001, 0.01, 0.1, 0.5, 1.0):
-        for g in (1, 1000, 100000, 1000000):
-            timed(W.config4(600_000_000, s, g))
-    # the large group counts as DENSE results too (global atomics, no key look-up), for comparison with the
-    # hashed form the configuration asks for
-    for s in (0.1, 1.0):
-        for g in (100000, 1000000):
-            timed(W.config4(600_000_000, s, g, hashed=False))
-    return out
 
 
 def run_ablation(sjq, W, device, specialise=True):

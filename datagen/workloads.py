@@ -283,8 +283,46 @@ def city_pair(n: int = 600_000_000) -> Workload:
                     AggExpr("COL", Term("FACT", "revenue")), "DENSE", num_groups=250 * 250 * 7)
 
 
+def city_brand(n: int = 600_000_000, hashed: bool = True) -> Workload:
+    """Beyond the five benchmark configurations: the paper's city x brand shape (Section 3.3, the Q4.3
+    pattern: group by year, supplier city and part brand; very few rows survive).  Customer is filtered
+    to one region and gathers nothing; supplier is filtered to one nation and gathers its city U[0,249];
+    part is filtered to one category and gathers its brand U[0,999]; the date table keeps 1997-1998 and
+    gathers the year.  Key ((year - 1992) * 250 + city) * 1000 + brand: 1,750,000 possible groups, of which
+    at most 2 * 10 * 1000 can occur; about n / 10,900 rows survive.  sum(revenue - supplycost) and count.
+    Asked for as a hashed list (capacity 32,768) by default, or as the dense array of all possible groups."""
+    base = 700
+    fact = (ColSpec("custkey", UNIFORM_I32, base + 0, 1, 3000000),
+            ColSpec("suppkey", UNIFORM_I32, base + 1, 1, 200000),
+            ColSpec("partkey", UNIFORM_I32, base + 2, 1, 1400000),
+            ColSpec("orderdate", DATE_FK_I32, base + 3),
+            ColSpec("revenue", UNIFORM_I32, base + 4, 100000, 10000000),
+            ColSpec("supplycost", UNIFORM_I32, base + 5, 100000, 10000000))
+    cust = DimSpec("customer", 3000000,
+                   (ColSpec("custkey", SEQ_I32), ColSpec("nation", UNIFORM_I32, base + 50, 0, 24),
+                    ColSpec("region", UNIFORM_DIV_I32, base + 50, 0, 24, div=5)),
+                   key="custkey", preds=(Pred("region", "EQ", 1),))
+    supp = DimSpec("supplier", 200000,
+                   (ColSpec("suppkey", SEQ_I32), ColSpec("city", UNIFORM_I32, base + 60, 0, 249),
+                    ColSpec("nation", UNIFORM_DIV_I32, base + 60, 0, 249, div=10)),
+                   key="suppkey", preds=(Pred("nation", "EQ", 7),), payloads=("city",))
+    part = DimSpec("part", 1400000,
+                   (ColSpec("partkey", SEQ_I32), ColSpec("category", UNIFORM_I32, base + 70, 0, 24),
+                    ColSpec("brand", UNIFORM_I32, base + 71, 0, 999)),
+                   key="partkey", preds=(Pred("category", "EQ", 3),), payloads=("brand",))
+    date = _date_dim(preds=(Pred("year", "BETWEEN", 1997, 1998),), payloads=("year",))
+    key = KeyExpr((Term("PAYLOAD", 3, 0, 250 * 1000), Term("PAYLOAD", 1, 0, 1000), Term("PAYLOAD", 2, 0, 1)),
+                  offset=-1992 * 250 * 1000)
+    return Workload("city_brand_groupby" + ("" if hashed else "_dense"), n, fact, (cust, supp, part, date),
+                    (("custkey", "customer"), ("suppkey", "supplier"), ("partkey", "part"), ("orderdate", "date")),
+                    (), key, AggExpr("SUB", Term("FACT", "revenue"), Term("FACT", "supplycost")),
+                    "HASHED" if hashed else "DENSE", num_groups=7 * 250 * 1000, capacity=32768)
+
+
 def with_rows(w: Workload, n: int) -> Workload:
     return replace(w, n_rows=n)
 
 
 CONFIGS = {"c1": config1, "c2": config2, "c3": config3, "c4": config4, "c5": config5}
+# star-join shapes beyond the five configurations (the paper's high-cardinality group-bys, Section 3.3)
+EXTRA_SHAPES = {"city_pair": city_pair, "city_brand": city_brand}

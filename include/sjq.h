@@ -193,7 +193,12 @@ sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_col, int npa
 
 /*
  * Build the table described by `layout` into caller memory `table_mem`
- * (>= layout->table_bytes, else BUFFER_SMALL) and return a handle.  Enqueues
+ * (>= layout->table_bytes, else BUFFER_SMALL) and return a handle.  The
+ * layout normally comes from sjq_dim_plan; whatever its origin, its sizes are
+ * recomputed and a self-contradictory layout is INVALID_ARG.  A layout that
+ * is consistent but too small for the data is caught on the device
+ * (LAYOUT_MISMATCH: key or payload outside the planned ranges; TABLE_FULL:
+ * the open-addressing table has no free slot left).  Enqueues
  * a fill, the build kernel and a verification kernel; does not synchronise.
  * Direct tables are written by race-free direct stores indexed by key
  * (Section 3.3); hash tables by atomicCAS on the key word with a bounded
@@ -204,6 +209,18 @@ sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_col, int npa
 sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pred *preds, int npreds, int key_col,
                          const int *payload_cols, int npayload, const sjq_dim_layout *layout, void *table_mem,
                          size_t table_bytes, int32_t *status_dev, void *stream, sjq_table **table);
+
+/*
+ * Device bytes a table of the given shape occupies, recomputed from `kind`,
+ * `key_dtype`, `npayload`, `code_bits`, `slots` and `filter_bits` (the
+ * layout's own `table_bytes` is not read).  A caller that edits a planned
+ * layout (Section 4.3.1 lets the engine choose the table form at run time;
+ * here the caller may override that choice, e.g. give an open-addressing
+ * table more slots) must store the answer in `table_bytes` before handing the
+ * layout to sjq_build_dim, which rejects a layout whose fields contradict one
+ * another (INVALID_ARG) instead of writing past `table_mem`.  Host only.
+ */
+sjq_status sjq_dim_layout_bytes(const sjq_dim_layout *layout, size_t *bytes);
 
 /* Copy of the layout the table was built with. */
 sjq_status sjq_table_info(const sjq_table *table, sjq_dim_layout *layout);
@@ -323,6 +340,26 @@ sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *preds, int np
                    const sjq_result *out, const sjq_run_opts *opts, void *stream, sjq_run_info *info);
 
 /*
+ * Merge lists of (key, sum, count) triples into one list with one entry per
+ * distinct key, sums and counts added (int64, wrapping).  This is the exchange
+ * step of a row-sharded run over several GPUs (the paper's second scale point,
+ * Section 5.1, is a table twice the size of the first): every GPU runs sjq_run
+ * on its row range, the per-GPU HASHED lists are gathered, and this call
+ * folds them; integer sums make the result independent of the split.
+ *   keys/sums/counts  device arrays of n entries (8-byte aligned; a key may
+ *                     occur any number of times)
+ *   capacity          maximum number of distinct keys
+ *   out               keys/sums/counts[capacity], n_groups, status, and a
+ *                     workspace of sjq_run_workspace_bytes({SJQ_HASHED, 0,
+ *                     capacity}) bytes; all cleared by this call.  The output
+ *                     arrays must not overlap the inputs.
+ * Enqueues three kernels on `stream`; does not synchronise.  More distinct
+ * keys than `capacity` sets SJQ_ERR_GROUP_OVERFLOW in *out->status.
+ */
+sjq_status sjq_merge_groups(const int64_t *keys, const int64_t *sums, const int64_t *counts, int64_t n,
+                            int64_t capacity, const sjq_result *out, void *stream);
+
+/*
  * The same query over fact columns that live in HOST memory (page-locked for
  * full copy speed): the table is cut into chunks of `chunk_rows` rows; each
  * chunk's columns are copied into one half of the device staging buffer while
@@ -391,15 +428,19 @@ sjq_status sjq_host_transfer_plan(const sjq_col *fact_host, int nfact, const sjq
  *   - `opts->accumulate` is ignored: the table is cleared at the start of
  *     every call, because it is shared by all calls and still holds the
  *     previous call's groups.
- *   - `opts->specialise` is ignored: loading a module compiled at run time
- *     allocates device memory, so this entry point always runs the interpreted
- *     kernel.
+ *   - `opts->specialise` is ignored: a module compiled at run time is loaded
+ *     when its query shape is first met, which places code on the device at an
+ *     arbitrary moment, so this entry point always runs the interpreted kernel.
  *   - Calls whose kernels could overlap on the GPU (different streams, several
  *     host threads) race on the one table; run them one after another.
- *   - The first call on a device looks the array's device address up once; make
- *     that first call outside any stream capture.
- *   - No cudaMalloc, cudaFree or other allocating CUDA call is made, here or in
- *     anything this entry point calls.
+ *   - The first call on a device looks the array's device address up once, and
+ *     the CUDA driver loads each ahead-of-time kernel the first time it is
+ *     launched (that loading is the driver's own and may reserve device memory
+ *     for code).  Make one call per query shape you will use during start-up,
+ *     outside any stream capture; later calls take nothing from the device.
+ *   - What is promised: the library itself calls no cudaMalloc,
+ *     cudaMallocAsync, cudaFree or allocating library routine on this path,
+ *     and needs no workspace from the caller.
  */
 #define SJQ_STATIC_MAX_GROUPS 65536
 #define SJQ_STATIC_WORKSPACE_BYTES ((size_t)3 * 1024 * 1024 + 768 + 3 * 256)

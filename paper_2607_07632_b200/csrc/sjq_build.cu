@@ -282,6 +282,45 @@ int bits_for(uint64_t range)
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Bytes of a direct table's slot array (bitmap words or packed codes), spare entry included.
+size_t direct_array_bytes(const sjq_dim_layout &L)
+{
+    const uint64_t span = (uint64_t)L.slots;
+    const size_t bytes = L.kind == SJQ_TABLE_DIRECT_BITMAP ? (size_t)((span + 32) / 32 * 4)
+                                                           : (size_t)((span + 1) * (uint64_t)(L.code_bits / 8));
+    return align_up(bytes, 16);
+}
+
+// Device bytes a table of this shape occupies, recomputed from kind, slots, code_bits and filter_bits (never
+// taken from the struct); false when the fields contradict one another.  sjq_dim_plan_end sizes tables with
+// it and sjq_build_dim checks a caller-supplied layout against it, so that a stale or hand-edited layout is
+// rejected on the host instead of making the fills and the build kernel write past table_mem.
+bool layout_table_bytes(const sjq_dim_layout &L, size_t *bytes)
+{
+    if (L.slots <= 0 || L.npayload < 0 || L.npayload > SJQ_MAX_PAYLOADS || L.filter_bits < 0) return false;
+    if (L.kind >= SJQ_TABLE_DIRECT_BITMAP && L.kind <= SJQ_TABLE_DIRECT_U64) {
+        if ((uint64_t)L.slots > ((uint64_t)1 << 40)) return false;
+        const int want_bits = L.kind == SJQ_TABLE_DIRECT_BITMAP ? 0 : 8 << (L.kind - SJQ_TABLE_DIRECT_U8);
+        if (L.code_bits != want_bits || (L.kind == SJQ_TABLE_DIRECT_BITMAP) != (L.npayload == 0)) return false;
+        if (L.filter_bits != 0 &&
+            (L.kind == SJQ_TABLE_DIRECT_BITMAP || L.filter_bits <= L.slots || L.filter_bits % 128 != 0))
+            return false;
+        *bytes = kTableHeaderBytes + align_up(direct_array_bytes(L), 256) + align_up((size_t)(L.filter_bits / 8), 256);
+        return true;
+    }
+    if (L.kind == SJQ_TABLE_HASH_I32 || L.kind == SJQ_TABLE_HASH_I64) {
+        if ((L.kind == SJQ_TABLE_HASH_I64) != (L.key_dtype == SJQ_I64)) return false;
+        if (L.slots < 16 || (L.slots & (L.slots - 1)) || L.slots > ((int64_t)1 << 31)) return false;
+        if (L.npayload == 0 ? L.code_bits != 0 : (L.code_bits != 32 && L.code_bits != 64)) return false;
+        if ((L.filter_bits & (L.filter_bits - 1)) || L.filter_bits > ((int64_t)1 << 32)) return false;
+        const size_t kb = (size_t)L.slots * (L.key_dtype == SJQ_I64 ? 8 : 4);
+        const size_t cb = (size_t)L.slots * (size_t)(L.code_bits / 8);
+        *bytes = kTableHeaderBytes + align_up(kb, 256) + align_up(cb, 256) + align_up((size_t)(L.filter_bits / 8), 256);
+        return true;
+    }
+    return false;
+}
+
 sjq_status fill_dim_params(const sjq_col *cols, int ncols, const sjq_pred *preds, int npreds, int key_col,
                            const int *payload_cols, int npayload, DimParams *P)
 {
@@ -505,13 +544,9 @@ extern "C" sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_c
                  : code_bits == 16 ? SJQ_TABLE_DIRECT_U16
                  : code_bits == 32 ? SJQ_TABLE_DIRECT_U32
                                    : SJQ_TABLE_DIRECT_U64;
-        L.table_bytes = kTableHeaderBytes + align_up(direct_bytes, 256);
-        if (npayload > 0) {
-            // a code array is 8 to 64 times the size of a bitmap over the same slots: keep both, so that a
-            // filter stage probes the bitmap and only the survivors gather their payload from the codes
-            L.filter_bits = (int64_t)((span_m1 + 129) / 128 * 128); // at least one spare bit after the last slot
-            L.table_bytes += align_up((size_t)(L.filter_bits / 8), 256);
-        }
+        // a code array is 8 to 64 times the size of a bitmap over the same slots: keep both, so that a
+        // filter stage probes the bitmap and only the survivors gather their payload from the codes
+        if (npayload > 0) L.filter_bits = (int64_t)((span_m1 + 129) / 128 * 128); // at least one spare bit after the last slot
     } else {
         uint64_t want = ((uint64_t)L.entries * 100u + (uint64_t)load_pct - 1) / (uint64_t)load_pct;
         uint64_t slots = 16;
@@ -519,14 +554,12 @@ extern "C" sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_c
         L.slots = (int64_t)slots;
         L.kind = L.key_dtype == SJQ_I64 ? SJQ_TABLE_HASH_I64 : SJQ_TABLE_HASH_I32;
         L.code_bits = npayload == 0 ? 0 : (code_bits <= 32 ? 32 : 64);
-        const size_t kb = (size_t)slots * (L.key_dtype == SJQ_I64 ? 8 : 4);
-        const size_t cb = (size_t)slots * (size_t)(L.code_bits / 8);
         // presence bitmap: 16 bits per entry (about 6 % false positives), at least 1024 bits, at most 2^32
         uint64_t fbits = 1024;
         while (fbits < (uint64_t)L.entries * 16 && fbits < ((uint64_t)1 << 32)) fbits <<= 1;
         L.filter_bits = (int64_t)fbits;
-        L.table_bytes = kTableHeaderBytes + align_up(kb, 256) + align_up(cb, 256) + align_up((size_t)(fbits / 8), 256);
     }
+    if (!layout_table_bytes(L, &L.table_bytes)) return SJQ_ERR_UNSUPPORTED;
     *layout = L;
     return SJQ_OK;
 }
@@ -542,17 +575,15 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
     sjq_status st = fill_dim_params(cols, ncols, preds, npreds, key_col, payload_cols, npayload, &B.dim);
     if (st != SJQ_OK) return st;
     const sjq_dim_layout &L = *layout;
-    if (L.kind < SJQ_TABLE_DIRECT_BITMAP || L.kind > SJQ_TABLE_HASH_I64) return SJQ_ERR_INVALID_ARG;
-    if (L.kind >= SJQ_TABLE_HASH_I32 &&
-        (L.filter_bits < 0 || (L.filter_bits & (L.filter_bits - 1)) || L.filter_bits > ((int64_t)1 << 32)))
+    // The layout is the caller's: every size used below is recomputed from its shape fields, never taken
+    // from its table_bytes, and a layout whose fields contradict one another is rejected here.
+    size_t need_bytes = 0;
+    if (L.npayload != npayload || L.key_dtype != cols[key_col].dtype || L.dim_rows != B.dim.n ||
+        !layout_table_bytes(L, &need_bytes) || need_bytes != L.table_bytes)
         return SJQ_ERR_INVALID_ARG;
-    if (L.kind <= SJQ_TABLE_DIRECT_U64 && L.filter_bits != 0 &&
-        (L.kind == SJQ_TABLE_DIRECT_BITMAP || L.filter_bits <= L.slots || L.filter_bits % 128 != 0))
-        return SJQ_ERR_INVALID_ARG;
-    if (L.kind < SJQ_TABLE_DIRECT_BITMAP || L.kind > SJQ_TABLE_HASH_I64 || L.npayload != npayload ||
-        L.key_dtype != cols[key_col].dtype || L.slots <= 0 || L.dim_rows != B.dim.n)
-        return SJQ_ERR_INVALID_ARG;
-    if (table_bytes < L.table_bytes) return SJQ_ERR_BUFFER_SMALL;
+    for (int i = 0; i < npayload; ++i)
+        if (L.pay_bits[i] < 0 || L.pay_bits[i] > 63) return SJQ_ERR_INVALID_ARG;
+    if (table_bytes < need_bytes) return SJQ_ERR_BUFFER_SMALL;
     DeviceInfo dev;
     if ((st = device_info(&dev)) != SJQ_OK) return st;
     cudaStream_t stream = (cudaStream_t)stream_;
@@ -583,10 +614,7 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
     bool ok = cudaMemsetAsync(T->base, 0, kTableHeaderBytes, stream) == cudaSuccess;
     const bool direct = L.kind <= SJQ_TABLE_DIRECT_U64;
     if (direct) {
-        const uint64_t span = (uint64_t)L.slots;
-        size_t bytes = L.kind == SJQ_TABLE_DIRECT_BITMAP ? (size_t)((span + 32) / 32 * 4)
-                                                         : (size_t)((span + 1) * (uint64_t)(L.code_bits / 8));
-        bytes = align_up(bytes, 16);
+        const size_t bytes = direct_array_bytes(L);
         T->slots_bytes = bytes;
         ok = ok && cudaMemsetAsync(T->slots, L.kind == SJQ_TABLE_DIRECT_BITMAP ? 0 : 0xFF, bytes, stream) == cudaSuccess;
         if (L.filter_bits) {
@@ -626,6 +654,12 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
     }
     *table = T;
     return SJQ_OK;
+}
+
+extern "C" sjq_status sjq_dim_layout_bytes(const sjq_dim_layout *layout, size_t *bytes)
+{
+    if (!layout || !bytes) return SJQ_ERR_INVALID_ARG;
+    return layout_table_bytes(*layout, bytes) ? SJQ_OK : SJQ_ERR_INVALID_ARG;
 }
 
 extern "C" sjq_status sjq_table_info(const sjq_table *table, sjq_dim_layout *layout)

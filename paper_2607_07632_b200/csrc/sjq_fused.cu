@@ -64,6 +64,22 @@ __global__ void __launch_bounds__(256) compact_kernel(const CompactParams C)
     }
 }
 
+struct MergeParams {
+    const int64_t *keys, *sums, *counts; // the lists to merge, n entries
+    int64_t n;
+    int64_t *gkeys, *gsums, *gcounts; // group table
+    uint64_t gmask;
+    int32_t *status;
+};
+
+// Lists of (key, sum, count) -> group table: one insert-or-find and two adds per entry.
+__global__ void __launch_bounds__(256) merge_kernel(const MergeParams M)
+{
+    const int64_t stride = (int64_t)blockDim.x * gridDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < M.n; i += stride)
+        group_table_add(M.gkeys, M.gsums, M.gcounts, M.gmask, M.status, M.keys[i], M.sums[i], M.counts[i]);
+}
+
 typedef void (*fused_fn)(const RunParams);
 
 fused_fn pick_kernel(int agg, bool mul, bool hash)
@@ -145,6 +161,18 @@ sjq_status clear_launch(int64_t *sums, int64_t *counts, int64_t cells, int64_t *
     if (blocks > (int64_t)sm_count * 8) blocks = (int64_t)sm_count * 8;
     if (blocks < 1) blocks = 1;
     clear_kernel<<<(int)blocks, 256, 0, stream>>>(C);
+    return cudaGetLastError() == cudaSuccess ? SJQ_OK : SJQ_ERR_CUDA;
+}
+
+sjq_status merge_launch(const int64_t *keys, const int64_t *sums, const int64_t *counts, int64_t n, int64_t *gkeys,
+                        int64_t *gsums, int64_t *gcounts, uint64_t gmask, int32_t *status, int sm_count,
+                        cudaStream_t stream)
+{
+    if (n <= 0) return SJQ_OK;
+    MergeParams M{keys, sums, counts, n, gkeys, gsums, gcounts, gmask, status};
+    int64_t blocks = (n + 255) / 256;
+    if (blocks > (int64_t)sm_count * 8) blocks = (int64_t)sm_count * 8;
+    merge_kernel<<<(int)blocks, 256, 0, stream>>>(M);
     return cudaGetLastError() == cudaSuccess ? SJQ_OK : SJQ_ERR_CUDA;
 }
 

@@ -36,6 +36,10 @@ sjq_status compact_launch(const int64_t *gkeys, const int64_t *gsums, const int6
                           int64_t dense_base, int64_t *keys, int64_t *sums, int64_t *counts, int64_t capacity,
                           int64_t *n_groups, int32_t *status, int sm_count, cudaStream_t stream);
 
+sjq_status merge_launch(const int64_t *keys, const int64_t *sums, const int64_t *counts, int64_t n, int64_t *gkeys,
+                        int64_t *gsums, int64_t *gcounts, uint64_t gmask, int32_t *status, int sm_count,
+                        cudaStream_t stream);
+
 namespace {
 
 struct StageSpec {
@@ -660,6 +664,42 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     return SJQ_OK;
 }
 
+
+// ---------------------------------------------------------------------------
+// Merge of hashed results (the exchange step of a row-sharded run).
+extern "C" sjq_status sjq_merge_groups(const int64_t *keys, const int64_t *sums, const int64_t *counts, int64_t n,
+                                       int64_t capacity, const sjq_result *out, void *stream_)
+{
+    if (n < 0 || capacity <= 0 || !out || !out->keys || !out->sums || !out->counts || !out->n_groups ||
+        !out->status || !out->workspace || (n > 0 && (!keys || !sums || !counts)))
+        return SJQ_ERR_INVALID_ARG;
+    if (!aligned16(out->sums) || !aligned16(out->counts) || !aligned16(out->keys) || !aligned16(out->workspace) ||
+        (reinterpret_cast<uintptr_t>(keys) & 7u) || (reinterpret_cast<uintptr_t>(sums) & 7u) ||
+        (reinterpret_cast<uintptr_t>(counts) & 7u) || (reinterpret_cast<uintptr_t>(out->status) & 3u) ||
+        (reinterpret_cast<uintptr_t>(out->n_groups) & 7u))
+        return SJQ_ERR_ALIGN;
+    sjq_result_spec spec{SJQ_HASHED, 0, capacity};
+    size_t need = 0;
+    sjq_run_workspace_bytes(&spec, &need);
+    if (out->workspace_bytes < need) return SJQ_ERR_BUFFER_SMALL;
+    DeviceInfo dev;
+    sjq_status st = device_info(&dev);
+    if (st != SJQ_OK) return st;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const uint64_t gslots = hashed_slots(capacity);
+    const size_t arr = align_up((size_t)(gslots + 1) * 8, 256);
+    int64_t *gkeys = reinterpret_cast<int64_t *>(static_cast<char *>(out->workspace));
+    int64_t *gsums = reinterpret_cast<int64_t *>(static_cast<char *>(out->workspace) + arr);
+    int64_t *gcounts = reinterpret_cast<int64_t *>(static_cast<char *>(out->workspace) + 2 * arr);
+    if ((st = clear_launch(gsums, gcounts, (int64_t)gslots + 1, gkeys, (int64_t)gslots + 1, out->n_groups, out->status,
+                           dev.sm_count, stream)) != SJQ_OK)
+        return st;
+    if ((st = merge_launch(keys, sums, counts, n, gkeys, gsums, gcounts, gslots - 1, out->status, dev.sm_count,
+                           stream)) != SJQ_OK)
+        return st;
+    return compact_launch(gkeys, gsums, gcounts, (int64_t)gslots, -1, out->keys, out->sums, out->counts, capacity,
+                          out->n_groups, out->status, dev.sm_count, stream);
+}
 
 // ---------------------------------------------------------------------------
 // Host-buffer entry point: chunked, double-buffered copy + run.

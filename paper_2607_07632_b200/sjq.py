@@ -174,6 +174,8 @@ def lib():
         L.sjq_build_dim.restype = ctypes.c_int32
         L.sjq_build_dim.argtypes = [ctypes.POINTER(_Col), ip, ctypes.POINTER(_Pred), ip, ip, ctypes.POINTER(ip), ip,
                                     ctypes.POINTER(DimLayout), vp, ctypes.c_size_t, vp, vp, ctypes.POINTER(vp)]
+        L.sjq_dim_layout_bytes.restype = ctypes.c_int32
+        L.sjq_dim_layout_bytes.argtypes = [ctypes.POINTER(DimLayout), ctypes.POINTER(ctypes.c_size_t)]
         L.sjq_table_info.restype = ctypes.c_int32
         L.sjq_table_info.argtypes = [vp, ctypes.POINTER(DimLayout)]
         L.sjq_table_destroy.restype = None
@@ -189,6 +191,8 @@ def lib():
                                    ctypes.POINTER(_KeyExpr), ctypes.POINTER(_AggExpr), ctypes.POINTER(_ResultSpec),
                                    ctypes.POINTER(_Result), ctypes.POINTER(_RunOpts), vp, ctypes.c_size_t,
                                    ctypes.c_int64, vp, vp, vp, vp, vp, vp]
+        L.sjq_merge_groups.restype = ctypes.c_int32
+        L.sjq_merge_groups.argtypes = [vp, vp, vp, ctypes.c_int64, ctypes.c_int64, ctypes.POINTER(_Result), vp]
         L.sjq_run_hashed_static.restype = ctypes.c_int32
         L.sjq_run_hashed_static.argtypes = [ctypes.POINTER(_Col), ip, ctypes.POINTER(_Pred), ip,
                                             ctypes.POINTER(_Join), ip, ctypes.POINTER(_KeyExpr),
@@ -232,6 +236,15 @@ def _preds(preds, names: Sequence[str]):
     return arr, keep
 
 
+def layout_bytes(layout: DimLayout) -> int:
+    """sjq_dim_layout_bytes: device bytes a table of this shape needs (raises if the shape is inconsistent)."""
+    n = ctypes.c_size_t(0)
+    rc = lib().sjq_dim_layout_bytes(ctypes.byref(layout), ctypes.byref(n))
+    if rc != 0:
+        raise SjqError(rc, "sjq_dim_layout_bytes")
+    return int(n.value)
+
+
 class Table:
     """A built dimension table: host handle + the device memory it lives in."""
 
@@ -254,8 +267,10 @@ class Table:
 
 
 def build_dim(cols: dict, key: str, preds=(), payloads=(), force_kind: int = 0, hash_load_pct: int = 0,
-              max_direct_bytes: int = 0) -> Table:
-    """sjq_dim_plan + sjq_build_dim over a dict of CUDA tensors (dimension columns)."""
+              max_direct_bytes: int = 0, edit_layout=None) -> Table:
+    """sjq_dim_plan + sjq_build_dim over a dict of CUDA tensors (dimension columns).  `edit_layout`, if
+    given, is called with the planned DimLayout and may change it before the build (sjq_build_dim takes
+    the layout from its caller: tests use this to hand it an undersized or inconsistent one)."""
     names = list(cols.keys())
     tensors = [cols[n] for n in names]
     device = tensors[0].device
@@ -271,7 +286,10 @@ def build_dim(cols: dict, key: str, preds=(), payloads=(), force_kind: int = 0, 
                                 ctypes.byref(opts), scratch.data_ptr(), stream, ctypes.byref(layout))
         if rc != 0:
             raise SjqError(rc, "sjq_dim_plan")
-        mem = torch.empty(layout.table_bytes, dtype=torch.uint8, device=device)
+        planned_bytes = layout.table_bytes
+        if edit_layout is not None:
+            edit_layout(layout)
+        mem = torch.empty(max(planned_bytes, layout.table_bytes), dtype=torch.uint8, device=device)
         status = torch.zeros(1, dtype=torch.int32, device=device)
         handle = ctypes.c_void_p()
         rc = lib().sjq_build_dim(carr, len(names), parr, len(preds), names.index(key), pay, len(payloads),
@@ -379,6 +397,8 @@ class Result:
     status_dev: torch.Tensor
     workspace: Optional[torch.Tensor]
     info: RunInfo = field(default_factory=RunInfo)
+    joined: Optional[torch.Tensor] = None  # SCALAR / DENSE: sums, counts and one spare cell as views of one int64
+    #                                        buffer, so that a multi-GPU merge is a single all-reduce
 
     def status(self) -> int:
         return int(self.status_dev.item())
@@ -407,9 +427,16 @@ def _term(t, names) -> _Term:
 def alloc_result(mode: str, num_groups: int, capacity: int, want_count: bool, device) -> Result:
     spec = _ResultSpec(MODES[mode], num_groups, capacity)
     n = 1 if mode == "SCALAR" else num_groups if mode == "DENSE" else capacity
-    sums = torch.empty(n, dtype=torch.int64, device=device)
-    counts = torch.empty(n, dtype=torch.int64, device=device) if (want_count or mode == "HASHED") else None
-    keys = n_groups = ws = None
+    keys = n_groups = ws = joined = None
+    if mode != "HASHED":
+        # one allocation: [sums | counts | one cell for the merged status]; each part starts 16-byte aligned
+        pad = (n + 1) // 2 * 2
+        joined = torch.empty(2 * pad + 2 if want_count else pad + 2, dtype=torch.int64, device=device)
+        sums = joined[:n]
+        counts = joined[pad:pad + n] if want_count else None
+    else:
+        sums = torch.empty(n, dtype=torch.int64, device=device)
+        counts = torch.empty(n, dtype=torch.int64, device=device)
     if mode == "HASHED":
         keys = torch.empty(n, dtype=torch.int64, device=device)
         n_groups = torch.zeros(1, dtype=torch.int64, device=device)
@@ -419,7 +446,26 @@ def alloc_result(mode: str, num_groups: int, capacity: int, want_count: bool, de
             raise SjqError(rc, "sjq_run_workspace_bytes")
         ws = torch.empty(nbytes.value, dtype=torch.uint8, device=device)
     status = torch.zeros(1, dtype=torch.int32, device=device)
-    return Result(mode, sums, counts, keys, n_groups, status, ws)
+    return Result(mode, sums, counts, keys, n_groups, status, ws, joined=joined)
+
+
+def merge_groups(keys: torch.Tensor, sums: torch.Tensor, counts: torch.Tensor, capacity: int,
+                 result: Optional[Result] = None) -> Result:
+    """sjq_merge_groups: fold lists of (key, sum, count) triples (CUDA int64 tensors of equal length) into
+    a HASHED result with one entry per distinct key."""
+    device = keys.device
+    n = keys.numel()
+    for t in (keys, sums, counts):
+        if t.dtype != torch.int64 or not t.is_cuda or not t.is_contiguous() or t.numel() != n:
+            raise ValueError("merge_groups takes contiguous int64 CUDA tensors of equal length")
+    with torch.cuda.device(device):
+        res = result if result is not None else alloc_result("HASHED", 0, capacity, True, device)
+        cres = _result_struct(res)
+        rc = lib().sjq_merge_groups(keys.data_ptr(), sums.data_ptr(), counts.data_ptr(), n, capacity,
+                                    ctypes.byref(cres), _stream_ptr(device))
+        if rc != 0:
+            raise SjqError(rc, "sjq_merge_groups")
+    return res
 
 
 def _query(names: Sequence[str], preds, joins, key, agg):

@@ -3,9 +3,10 @@
 full sizes (tests/golden/full_*.json).  Calls only the CPU oracle and the
 seeded input generator; nothing here touches the CUDA path.
 
-    python tests/golden/make_full_size.py [c1 c2 c3 c5 c4:<sel>:<groups> ...]   (default: everything)
+    python tests/golden/make_full_size.py [c1 c2 c3 c5 c4:<sel>:<groups> city_pair ...]   (default: everything)
 
-A dense result is stored whole; a hashed result is stored as its group count,
+A dense result is stored whole (beyond 20 000 groups: its totals and a SHA-256
+over the sums array followed by the counts array); a hashed result is stored as its group count,
 the totals, and a SHA-256 over the (key, sum, count) triples in ascending key
 order (int64 little-endian), which is what the GPU test recomputes.
 """
@@ -68,6 +69,13 @@ def compute(w, tag):
     if w.mode == "SCALAR":
         s, c = acc.get(0, (0, 0))
         out.update(sum=int(s), count=int(c))
+    elif w.mode == "DENSE" and w.num_groups > 20_000:
+        # a large dense result is stored like a hashed one: totals and a digest of the two whole arrays
+        h = hashlib.sha256()
+        h.update(np.ascontiguousarray(acc[0], dtype="<i8").tobytes())
+        h.update(np.ascontiguousarray(acc[1], dtype="<i8").tobytes())
+        out.update(groups=int(np.count_nonzero(acc[1])), total_sum=int(acc[0].sum()), total_count=int(acc[1].sum()),
+                   dense_sha256=h.hexdigest())
     elif w.mode == "DENSE":
         out.update(sums=[int(x) for x in acc[0]], counts=[int(x) for x in acc[1]])
     else:
@@ -85,10 +93,13 @@ def compute(w, tag):
 
 
 def main():
-    todo = sys.argv[1:] or (["c1", "c2", "c3", "c5"] +
+    todo = sys.argv[1:] or (["c1", "c2", "c3", "c5"] + list(W.EXTRA_SHAPES) +
                             [f"c4:{s:g}:{g}" for s in W.C4_THRESHOLDS for g in W.C4_GROUPS])
     for item in todo:
-        if item.startswith("c4"):
+        if item in W.EXTRA_SHAPES:
+            w = W.EXTRA_SHAPES[item]()
+            tag = item
+        elif item.startswith("c4"):
             _, s, g = item.split(":")
             w = W.config4(600_000_000, float(s), int(g))
             tag = f"c4_s{float(s):g}_g{int(g)}"

@@ -114,3 +114,55 @@ def test_more_than_2_pow_32_rows_equals_split_runs():
             assert int(whole.counts.sum().item()) == int((p < 2500).sum().item())
     del p, fact, parts
     torch.cuda.empty_cache()
+
+
+def test_more_than_2_pow_32_rows_through_three_queue_levels():
+    """The same edge with a longer pipeline: a predicate at level 0, then a second predicate and a
+    filtering join with a gathered payload as queue-fed levels, then the final level, so that the
+    tile-relative offsets and the per-tile drain run through every queue of a warp.  Checked by
+    split-and-add against two halves below 2^32 rows and by the survivor count recomputed from the
+    columns with plain tensor operations (a property that holds at any size)."""
+    import paper_2607_07632_b200 as sjq
+    from datagen import UNIFORM_I32, fill_device
+    from datagen.workloads import AggExpr, KeyExpr, Pred, Term
+
+    n = (1 << 32) + 8203
+    free, _ = torch.cuda.mem_get_info()
+    if free < 4 * n * 4 + (12 << 30):
+        pytest.skip("not enough device memory for four 17 GB columns")
+    seed = 20260707
+    p = fill_device(UNIFORM_I32, seed, 911, 0, n, 0, 9)
+    q = fill_device(UNIFORM_I32, seed, 912, 0, n, 0, 99)
+    fk = fill_device(UNIFORM_I32, seed, 913, 0, n, 1, 50_000)
+    m = fill_device(UNIFORM_I32, seed, 914, 0, n, 0, 1_000_000)
+    dim = {"k": torch.arange(1, 40_001, dtype=torch.int32, device="cuda"),
+           "f": torch.arange(0, 40_000, dtype=torch.int32, device="cuda") % 2,
+           "w": torch.arange(0, 40_000, dtype=torch.int32, device="cuda") % 11}
+    table = sjq.build_dim(dim, "k", (Pred("f", "EQ", 1),), ("w",)).check()
+    fact = {"p": p, "q": q, "fk": fk, "m": m}
+    half = 1 << 31
+    parts = [{k: v[:half] for k, v in fact.items()}, {k: v[half:] for k, v in fact.items()}]
+    preds = (Pred("p", "EQ", 3), Pred("q", "BETWEEN", 10, 59))
+    joins = (("fk", table),)
+    agg = AggExpr("ADD", Term("FACT", "m"), Term("PAYLOAD", 0, 0, 3))
+    kw = dict(mode="DENSE", key=KeyExpr((Term("PAYLOAD", 0, 0),)), num_groups=11)
+    order = (0, 1, 2)  # p, q, the join: one level each
+    acc = sjq.run(parts[0], preds, joins, agg=agg, opts=sjq.RunOpts(order=order), **kw)
+    acc = sjq.run(parts[1], preds, joins, agg=agg, opts=sjq.RunOpts(order=order, accumulate=True), result=acc, **kw)
+    # survivors: p == 3, 10 <= q <= 59, fk even (row r of the dimension has key r + 1 and passes iff r is odd)
+    alive = (p == 3)
+    alive &= (q >= 10)
+    alive &= (q <= 59)
+    alive &= (fk <= 40_000)
+    alive &= (fk % 2 == 0)
+    expected_count = int(alive.sum().item())
+    del alive
+    for specialise in (False, True):
+        whole = sjq.run(fact, preds, joins, agg=agg, opts=sjq.RunOpts(specialise=specialise, order=order), **kw)
+        torch.cuda.synchronize()
+        assert whole.status() == 0 and acc.status() == 0
+        assert whole.info.reserved_levels == 3, whole.info.describe()
+        assert torch.equal(whole.sums, acc.sums) and torch.equal(whole.counts, acc.counts)
+        assert int(whole.counts.sum().item()) == expected_count > 0
+    del p, q, fk, m, fact, parts
+    torch.cuda.empty_cache()

@@ -147,6 +147,31 @@ def test_duplicate_key_is_reported():
             assert t.status() == 0
 
 
+@pytest.mark.parametrize("wide", [False, True])
+def test_undersized_hash_table_reports_table_full(wide):
+    """A consistent layout with too few slots for the rows that pass (a stale plan, a caller's own
+    sizing): the bounded insert loop gives up and the status word says TABLE_FULL; nothing is written
+    outside the (smaller) table and the context stays usable."""
+    dt = torch.int64 if wide else torch.int32
+    cols = {"k": torch.arange(1, 1001, dtype=dt, device="cuda") * 7919,
+            "p": torch.arange(0, 1000, dtype=torch.int32, device="cuda")}
+
+    def shrink(L):
+        assert L.kind_name == ("HASH_I64" if wide else "HASH_I32") and L.slots >= 2000
+        L.slots = 64
+        L.table_bytes = sjq.layout_bytes(L)
+
+    for pay in ((), ("p",)):
+        t = sjq.build_dim(cols, "k", (), pay, force_kind=sjq.sjq.FORCE_HASH, edit_layout=shrink)
+        assert t.status() == 17 and "full" in sjq.strerror(17)
+        # exactly as many rows as slots still fit
+        t = sjq.build_dim(cols, "k", (Pred("p", "LT", 64),), pay, force_kind=sjq.sjq.FORCE_HASH, edit_layout=shrink)
+        assert t.status() == 0
+        t = sjq.build_dim(cols, "k", (Pred("p", "LT", 65),), pay, force_kind=sjq.sjq.FORCE_HASH, edit_layout=shrink)
+        assert t.status() == 17
+    assert sjq.build_dim(cols, "k", (), ("p",), force_kind=sjq.sjq.FORCE_HASH).status() == 0
+
+
 def test_reserved_key_and_empty_dimension():
     cols = {"k": torch.tensor([-(2 ** 63), 4], dtype=torch.int64, device="cuda")}
     assert sjq.build_dim(cols, "k", force_kind=sjq.sjq.FORCE_HASH).status() == 20

@@ -96,3 +96,67 @@ def test_compiled_modules_can_be_cached_on_disk(libsjq, tmp_path, monkeypatch):
     assert b"loaded from" in log.value
     assert libsjq.sjq_jit_selftest(1, log, len(log)) == 0  # another shape: another file
     assert len([f for f in os.listdir(tmp_path) if f.endswith(".cubin")]) == 2
+
+
+def test_build_rejects_inconsistent_layouts_on_the_host(libsjq):
+    """sjq_build_dim takes the table shape from its caller.  Every size it uses is recomputed from the shape
+    fields, so a layout whose fields contradict one another (or whose table_bytes was not recomputed after
+    an edit) is rejected before anything is enqueued: no device is needed to see that, and the pointers
+    below are never dereferenced."""
+    import paper_2607_07632_b200.sjq as b
+
+    n = 1000
+    cols = (b._Col * 2)(b._Col(0x10000, 0, n), b._Col(0x20000, 0, n))
+    pay = (ctypes.c_int * 1)(1)
+    handle = ctypes.c_void_p()
+
+    def build(layout, table_bytes=1 << 30):
+        return b.lib().sjq_build_dim(cols, 2, None, 0, 0, pay, 1, ctypes.byref(layout), 0x100000, table_bytes,
+                                     0x30000, None, ctypes.byref(handle))
+
+    def direct():
+        L = b.DimLayout()
+        L.kind, L.key_dtype, L.npayload, L.code_bits = 2, 0, 1, 8  # DIRECT_U8
+        L.dim_rows, L.entries, L.kmin, L.kmax, L.slots = n, n, 1, n, n
+        L.pay_bits[0] = 3
+        L.filter_bits = 1152
+        L.table_bytes = b.layout_bytes(L)
+        return L
+
+    def hashed():
+        L = direct()
+        L.kind, L.code_bits, L.slots, L.filter_bits = 6, 32, 2048, 16384  # HASH_I32
+        L.table_bytes = b.layout_bytes(L)
+        return L
+
+    for mk in (direct, hashed):
+        good = mk()
+        assert good.table_bytes > good.slots
+        assert build(good, good.table_bytes - 1) == 5  # consistent, but the caller's buffer is too small
+        L = mk()
+        L.table_bytes -= 256  # stale size
+        assert build(L) == 1
+        L = mk()
+        L.code_bits = 16  # does not match the kind
+        assert build(L) == 1
+        L = mk()
+        L.slots = 0
+        assert build(L) == 1
+        L = mk()
+        L.dim_rows = n + 1  # planned for another dimension
+        assert build(L) == 1
+    L = hashed()
+    L.slots = 2040  # an open-addressing table is made of whole buckets
+    with pytest.raises(b.SjqError):
+        b.layout_bytes(L)
+    L.table_bytes = hashed().table_bytes
+    assert build(L) == 1
+    L = hashed()
+    L.filter_bits = 1000  # the presence bitmap of an open-addressing table is a power of two
+    assert build(L) == 1
+    L = direct()
+    L.filter_bits = 640  # fewer bits than slots
+    assert build(L) == 1
+    L = direct()
+    L.kind, L.code_bits = 1, 0  # a bitmap table cannot carry the payload the call names
+    assert build(L) == 1
