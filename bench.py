@@ -339,6 +339,8 @@ def measure_point(sjq, torch, w, fact, tables, specialise, gpu_index, peak, extr
     point under load), each timed with its own CUDA events: the whole call (clear + fused kernel + compaction)
     and the fused kernel alone."""
     kw = dict(extra_opts or {})
+    # planning: the fact predicates' pass fractions are measured once (outside the timed runs, like the table builds)
+    kw["pass_ppm"] = sjq.sample_preds({c.name: fact[c.name] for c in w.fact_cols}, w.preds)
     res = sjq.run_workload(w, fact, tables, sjq.RunOpts(specialise=specialise, **kw))
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -389,6 +391,7 @@ def measure_point(sjq, torch, w, fact, tables, specialise, gpu_index, peak, extr
            "referenced_bytes_per_row": ref_bytes, "effective_gbs_kernel": eff,
            "pct_of_8tbs": 100.0 * eff / CONTRACT_HBM_GBS, "survivors": survivors,
            "pass_fractions": {str(k): round(v, 6) for k, v in frac.items()},
+           "sampled_pass_ppm": list(kw["pass_ppm"]),
            "l2": "256 MB written between runs" if small else "inputs exceed the L2",
            "status": status, "parity": matches_golden(w, res, golden_for(w)) if status == 0 else False,
            "plan": plan, "table_kinds": {k: t.layout.kind_name for k, t in tables.items()},
@@ -516,15 +519,20 @@ def main():
         b.record()
     res = sjq.alloc_result(w.mode, w.num_groups, w.capacity, w.agg.want_count, device)
     builders = sjq.workload_builders(w, dims)  # argument marshalling done once; plan + build run every step
+    pred_sampler = sjq.PredSampler({c.name: fact[c.name] for c in w.fact_cols}, w.preds)
     launches = 0
     info = None
     merged = None
 
     def step(i=None):
         nonlocal launches, info, merged
+        pred_sampler.begin()  # planning: measured pass fractions of the fact predicates, beside the key-range scans
         tables = sjq.build_tables(builders)
         opts = sjq.RunOpts(events=pairs[i] if i is not None else None, specialise=not args.interpret,
-                           block_threads=args.block_threads, ctas_per_sm=args.ctas_per_sm)
+                           block_threads=args.block_threads, ctas_per_sm=args.ctas_per_sm,
+                           pass_ppm=pred_sampler.end())
+        if i is not None and w.preds:
+            launches += 1
         r = sjq.run_workload(w_local, fact, tables, opts, result=res)
         if world > 1:
             merged = shard.merge_result(res)

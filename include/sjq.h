@@ -124,7 +124,7 @@ enum {
     SJQ_TABLE_DIRECT_U16 = 3,
     SJQ_TABLE_DIRECT_U32 = 4,
     SJQ_TABLE_DIRECT_U64 = 5,
-    SJQ_TABLE_HASH_I32 = 6, /* open addressing, linear probing, int32 keys */
+    SJQ_TABLE_HASH_I32 = 6, /* open addressing over 64-byte buckets of keys and codes, linear probing, int32 keys */
     SJQ_TABLE_HASH_I64 = 7,
     SJQ_TABLE_FORCE_DIRECT = 100, /* build option only */
     SJQ_TABLE_FORCE_HASH = 101    /* build option only */
@@ -135,7 +135,7 @@ enum {
 
 typedef struct sjq_build_opts {
     int32_t force_kind;       /* SJQ_TABLE_AUTO, SJQ_TABLE_FORCE_DIRECT or SJQ_TABLE_FORCE_HASH */
-    int32_t hash_load_pct;    /* 0 = default 50: slots >= entries * 100 / pct, power of two */
+    int32_t hash_load_pct;    /* 0 = default 50: slots >= entries * 100 / pct, in whole 64-byte buckets; <= 90 */
     int64_t max_direct_bytes; /* 0 = default 64 MiB: larger direct tables fall back to hashing */
 } sjq_build_opts;
 
@@ -151,7 +151,9 @@ typedef struct sjq_dim_layout {
     int64_t pay_min[SJQ_MAX_PAYLOADS]; /* payload i is stored as (value - pay_min[i]) in pay_bits[i] bits */
     int64_t pay_max[SJQ_MAX_PAYLOADS];
     int32_t pay_bits[SJQ_MAX_PAYLOADS];
-    int64_t slots;      /* direct: kmax-kmin+1; hash: power-of-two slot count */
+    int64_t slots;      /* direct: kmax-kmin+1; hash: key slots = 64-byte buckets x keys per bucket (a bucket holds
+                           K keys then their K codes: K = 16, 8 or 5 for 32-bit keys and 8, 5 or 4 for 64-bit keys
+                           with no, 32-bit or 64-bit codes) */
     int64_t filter_bits; /* direct with payloads: bits of the presence bitmap over the slots (a multiple of 128);
                             hash: size (power of two, 0 = none) of the presence bitmap indexed by the key's hash,
                             probed before the table so that most absent keys never touch it */
@@ -281,8 +283,6 @@ typedef struct sjq_run_opts {
     int32_t order[SJQ_MAX_PREDS + SJQ_MAX_JOINS]; /* entry < npreds: predicate index; else npreds + join index */
     void *event_before; /* optional cudaEvent_t recorded on `stream` right before the fused kernel */
     void *event_after;  /* optional cudaEvent_t recorded right after it (both or neither) */
-    int32_t dense_reach_permille; /* experiment knob: level 0 keeps the filter stages that more than this share of
-                                     the rows still reach (0 = default, 300) */
     int32_t specialise; /* 1 = compile the fused kernel for this query's shape at run time (NVRTC) and cache the
                            module for later runs of the same shape; 0 = interpret the descriptor (default).  Key
                            ranges, thresholds, table sizes and pointers stay run-time values, so a compiled module
@@ -299,7 +299,14 @@ typedef struct sjq_run_opts {
     int32_t group_hash_always; /* HASHED results: 1 = always use the group hash table; 0 = a key taken modulo M whose
                                   2M - 1 possible values fit the workspace is aggregated in a table indexed by the
                                   key itself */
-    int32_t reserved[1];
+    int32_t pass_ppm[SJQ_MAX_PREDS + SJQ_MAX_JOINS]; /* measured pass fractions in parts per million, predicates
+                                  first, then joins (index npreds + join): 0 = not known, the library estimates
+                                  (a fact predicate from its operator alone, a join from the share of dimension
+                                  rows its table holds); k > 0 = k / 1e6 of the rows pass that filter taken on its
+                                  own (use 1 for "none seen").  sjq_pred_sample measures the predicates.  The
+                                  estimates order the stages, split them into levels, pick the aggregation path
+                                  and decide copy versus in-place reads in sjq_run_host: they change the run time,
+                                  never the result. */
 } sjq_run_opts;
 
 /* What the planner decided for a run (for reports and tests). */
@@ -315,6 +322,30 @@ typedef struct sjq_run_info {
     int32_t smem_bytes;
     int32_t kernel_launches; /* kernels enqueued by the call */
 } sjq_run_info;
+
+/*
+ * Measure the pass fraction of every fact predicate on an evenly spaced
+ * sample of the table (65 536 groups of four rows), each predicate on its own.
+ * Section 3.2 of the paper ties run time to the bytes the lazily loaded columns
+ * move, which the selectivities decide, and Section 4.3.1 has the engine check
+ * properties of the data at run time instead of assuming them; here the
+ * planner's selectivity guesses are replaced by measured ones.
+ *   scratch_dev  device scratch of SJQ_PLAN_SCRATCH_BYTES bytes
+ *   pass_ppm     receives npreds entries, laid out like sjq_run_opts.pass_ppm
+ *                (a predicate that passed no sampled row gets 1, not 0)
+ * sjq_pred_sample enqueues one small kernel on `stream`, copies the counters
+ * back and SYNCHRONISES the stream.  The two halves let the wait be shared
+ * with other planning work: `_begin` enqueues the kernel and an asynchronous
+ * copy of SJQ_MAX_PREDS + 1 counters into `host_counts` (page-locked host
+ * memory) and returns; after the caller has synchronised that stream, `_end`
+ * turns the counters into pass_ppm on the host.
+ * Errors: INVALID_ARG, ALIGN, CUDA.
+ */
+sjq_status sjq_pred_sample(const sjq_col *fact, int nfact, const sjq_pred *preds, int npreds, void *scratch_dev,
+                           void *stream, int32_t *pass_ppm);
+sjq_status sjq_pred_sample_begin(const sjq_col *fact, int nfact, const sjq_pred *preds, int npreds,
+                                 void *scratch_dev, int64_t *host_counts, void *stream);
+sjq_status sjq_pred_sample_end(const int64_t *host_counts, int npreds, int32_t *pass_ppm);
 
 /* Device bytes needed at sjq_result.workspace for `spec` (0 unless HASHED). */
 sjq_status sjq_run_workspace_bytes(const sjq_result_spec *spec, size_t *bytes);

@@ -6,6 +6,7 @@
 // with a reserved all-ones sentinel for "filtered out".  Sparse keys fall back
 // to an open-addressing table populated with atomicCAS.  Section 4.3.1: the
 // key range is verified at run time and the packed or unpacked form chosen.
+#include <algorithm>
 #include <new>
 
 #include "sjq_internal.h"
@@ -112,11 +113,12 @@ struct BuildParams {
     int32_t code_bits;
     int64_t kmin;
     uint64_t span;  // direct
-    uint64_t hmask; // hash: slots - 1
+    uint32_t buckets; // hash: number of 64-byte buckets
+    int32_t bucket_k; // hash: keys per bucket
+    int32_t code_off; // hash: byte offset of the codes inside a bucket
     int64_t pay_min[SJQ_MAX_PAYLOADS], pay_max[SJQ_MAX_PAYLOADS];
     int32_t pay_bits[SJQ_MAX_PAYLOADS];
     void *slots;
-    void *codes;
     unsigned int *filter; // presence bitmap words (hash: indexed by a hash of the key; direct with payloads: by slot)
     uint32_t fmask;       // hash: filter bits - 1
     unsigned long long *header; // [0] rows inserted, [1] slots occupied
@@ -155,6 +157,35 @@ __device__ inline void store_code(void *codes, int bits, uint64_t idx, uint64_t 
     }
 }
 
+// Claim the first free slot on the key's probe path (bucket after bucket from its home bucket, the slots of
+// a bucket in order) with atomicCAS on the key word, then store the code beside it.  Bounded by the number
+// of buckets; a key met on the way is a duplicate.
+template <typename W>
+__device__ inline void hash_insert(const BuildParams &B, W key, W empty, uint64_t hashed, uint64_t code)
+{
+    char *base = static_cast<char *>(B.slots);
+    uint32_t b = home_bucket(hashed, B.buckets);
+    for (uint32_t it = 0; it < B.buckets; ++it) {
+        char *bucket = base + (size_t)b * kBucketBytes;
+        W *keys = reinterpret_cast<W *>(bucket);
+        for (int j = 0; j < B.bucket_k; ++j) {
+            W old = *reinterpret_cast<volatile W *>(&keys[j]);
+            if (old == empty) old = atomicCAS(&keys[j], empty, key);
+            if (old == empty) {
+                if (B.code_bits == 32) reinterpret_cast<uint32_t *>(bucket + B.code_off)[j] = (uint32_t)code;
+                else if (B.code_bits == 64) reinterpret_cast<uint64_t *>(bucket + B.code_off)[j] = code;
+                return;
+            }
+            if (old == key) {
+                set_status(B.status, SJQ_ERR_DUP_KEY);
+                return;
+            }
+        }
+        b = b + 1 == B.buckets ? 0 : b + 1;
+    }
+    set_status(B.status, SJQ_ERR_TABLE_FULL);
+}
+
 __global__ void __launch_bounds__(256) build_kernel(const __grid_constant__ BuildParams B)
 {
     const DimParams &P = B.dim;
@@ -186,56 +217,22 @@ __global__ void __launch_bounds__(256) build_kernel(const __grid_constant__ Buil
                 set_status(B.status, SJQ_ERR_RESERVED_KEY);
                 continue;
             }
-            unsigned long long *keys = static_cast<unsigned long long *>(B.slots);
             if (B.filter) {
                 const uint32_t fb = filter_hash((uint64_t)k) & B.fmask;
                 atomicOr(B.filter + (fb >> 5), 1u << (fb & 31));
             }
-            uint64_t slot = (hash64((uint64_t)k) * kBucketKeys64) & B.hmask; // first slot of the home bucket
-            bool done = false;
-            for (uint64_t it = 0; it <= B.hmask; ++it) {
-                unsigned long long old = atomicCAS(&keys[slot], (unsigned long long)kEmptyKey64, (unsigned long long)k);
-                if (old == (unsigned long long)kEmptyKey64) {
-                    store_code(B.codes, B.code_bits, slot, code);
-                    done = true;
-                    break;
-                }
-                if (old == (unsigned long long)k) {
-                    set_status(B.status, SJQ_ERR_DUP_KEY);
-                    done = true;
-                    break;
-                }
-                slot = (slot + 1) & B.hmask;
-            }
-            if (!done) set_status(B.status, SJQ_ERR_TABLE_FULL);
+            hash_insert<unsigned long long>(B, (unsigned long long)k, (unsigned long long)kEmptyKey64, (uint64_t)k, code);
         } else { // HASH_I32
             const int32_t k32 = (int32_t)k;
             if (k32 == kEmptyKey32) {
                 set_status(B.status, SJQ_ERR_RESERVED_KEY);
                 continue;
             }
-            int *keys = static_cast<int *>(B.slots);
             if (B.filter) {
                 const uint32_t fb = filter_hash((uint64_t)(int64_t)k32) & B.fmask;
                 atomicOr(B.filter + (fb >> 5), 1u << (fb & 31));
             }
-            uint64_t slot = (hash64((uint64_t)(int64_t)k32) * kBucketKeys32) & B.hmask; // first slot of the home bucket
-            bool done = false;
-            for (uint64_t it = 0; it <= B.hmask; ++it) {
-                int old = atomicCAS(&keys[slot], kEmptyKey32, k32);
-                if (old == kEmptyKey32) {
-                    store_code(B.codes, B.code_bits, slot, code);
-                    done = true;
-                    break;
-                }
-                if (old == k32) {
-                    set_status(B.status, SJQ_ERR_DUP_KEY);
-                    done = true;
-                    break;
-                }
-                slot = (slot + 1) & B.hmask;
-            }
-            if (!done) set_status(B.status, SJQ_ERR_TABLE_FULL);
+            hash_insert<unsigned int>(B, (unsigned int)k32, (unsigned int)kEmptyKey32, (uint64_t)(int64_t)k32, code);
         }
     }
     inserted = (unsigned long long)warp_sum((int64_t)inserted);
@@ -310,12 +307,12 @@ bool layout_table_bytes(const sjq_dim_layout &L, size_t *bytes)
     }
     if (L.kind == SJQ_TABLE_HASH_I32 || L.kind == SJQ_TABLE_HASH_I64) {
         if ((L.kind == SJQ_TABLE_HASH_I64) != (L.key_dtype == SJQ_I64)) return false;
-        if (L.slots < 16 || (L.slots & (L.slots - 1)) || L.slots > ((int64_t)1 << 31)) return false;
         if (L.npayload == 0 ? L.code_bits != 0 : (L.code_bits != 32 && L.code_bits != 64)) return false;
+        const int k = bucket_keys(L.key_dtype == SJQ_I64 ? 8 : 4, L.code_bits / 8);
+        if (L.slots % k != 0 || L.slots > ((int64_t)1 << 31)) return false; // whole buckets
         if ((L.filter_bits & (L.filter_bits - 1)) || L.filter_bits > ((int64_t)1 << 32)) return false;
-        const size_t kb = (size_t)L.slots * (L.key_dtype == SJQ_I64 ? 8 : 4);
-        const size_t cb = (size_t)L.slots * (size_t)(L.code_bits / 8);
-        *bytes = kTableHeaderBytes + align_up(kb, 256) + align_up(cb, 256) + align_up((size_t)(L.filter_bits / 8), 256);
+        *bytes = kTableHeaderBytes + align_up((size_t)(L.slots / k) * kBucketBytes, 256) +
+                 align_up((size_t)(L.filter_bits / 8), 256);
         return true;
     }
     return false;
@@ -548,12 +545,12 @@ extern "C" sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_c
         // filter stage probes the bitmap and only the survivors gather their payload from the codes
         if (npayload > 0) L.filter_bits = (int64_t)((span_m1 + 129) / 128 * 128); // at least one spare bit after the last slot
     } else {
-        uint64_t want = ((uint64_t)L.entries * 100u + (uint64_t)load_pct - 1) / (uint64_t)load_pct;
-        uint64_t slots = 16;
-        while (slots < want) slots <<= 1;
-        L.slots = (int64_t)slots;
         L.kind = L.key_dtype == SJQ_I64 ? SJQ_TABLE_HASH_I64 : SJQ_TABLE_HASH_I32;
         L.code_bits = npayload == 0 ? 0 : (code_bits <= 32 ? 32 : 64);
+        const uint64_t k = (uint64_t)bucket_keys(L.key_dtype == SJQ_I64 ? 8 : 4, L.code_bits / 8);
+        const uint64_t want = ((uint64_t)L.entries * 100u + (uint64_t)load_pct - 1) / (uint64_t)load_pct;
+        const uint64_t buckets = std::max<uint64_t>((want + k - 1) / k, 2);
+        L.slots = (int64_t)(buckets * k);
         // presence bitmap: 16 bits per entry (about 6 % false positives), at least 1024 bits, at most 2^32
         uint64_t fbits = 1024;
         while (fbits < (uint64_t)L.entries * 16 && fbits < ((uint64_t)1 << 32)) fbits <<= 1;
@@ -593,7 +590,6 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
     T->layout = L;
     T->base = static_cast<char *>(table_mem);
     T->slots = T->base + kTableHeaderBytes;
-    T->codes = nullptr;
     T->filter = nullptr;
     T->magic = kTableMagic;
 
@@ -601,7 +597,6 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
     B.code_bits = L.code_bits;
     B.kmin = L.kmin;
     B.span = (uint64_t)L.slots;
-    B.hmask = (uint64_t)L.slots - 1;
     for (int i = 0; i < SJQ_MAX_PAYLOADS; ++i) {
         B.pay_min[i] = L.pay_min[i];
         B.pay_max[i] = L.pay_max[i];
@@ -623,24 +618,26 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
             ok = ok && cudaMemsetAsync(T->filter, 0, (size_t)(L.filter_bits / 8), stream) == cudaSuccess;
         }
     } else {
-        const size_t kb = (size_t)L.slots * (L.key_dtype == SJQ_I64 ? 8 : 4);
-        T->slots_bytes = kb;
-        const size_t cb = (size_t)L.slots * (size_t)(L.code_bits / 8);
-        if (L.code_bits) T->codes = T->slots + align_up(kb, 256);
-        B.codes = T->codes;
+        const int kb = L.key_dtype == SJQ_I64 ? 8 : 4, cb = L.code_bits / 8;
+        B.bucket_k = bucket_keys(kb, cb);
+        B.code_off = bucket_code_offset(kb, cb, B.bucket_k);
+        B.buckets = (uint32_t)(L.slots / B.bucket_k);
+        const size_t bytes = (size_t)B.buckets * kBucketBytes;
+        T->slots_bytes = bytes;
         if (L.filter_bits) {
-            T->filter = T->slots + align_up(kb, 256) + align_up(cb, 256);
+            T->filter = T->slots + align_up(bytes, 256);
             B.filter = reinterpret_cast<unsigned int *>(T->filter);
             B.fmask = (uint32_t)(L.filter_bits - 1);
             ok = ok && cudaMemsetAsync(T->filter, 0, (size_t)(L.filter_bits / 8), stream) == cudaSuccess;
         }
-        const int g = grid_for(L.slots, dev.sm_count);
+        // Every word of a bucket starts as the empty marker's pattern: both markers (the minimum of the key
+        // type) are a repeated 0x80 00 .. 00 word, so the codes start as that pattern too and are overwritten
+        // when their slot is claimed.
+        const int g = grid_for((int64_t)(bytes / 8), dev.sm_count);
         if (L.key_dtype == SJQ_I64)
-            fill_kernel<int64_t><<<g, 256, 0, stream>>>(reinterpret_cast<int64_t *>(T->slots), kEmptyKey64, (size_t)L.slots);
+            fill_kernel<int64_t><<<g, 256, 0, stream>>>(reinterpret_cast<int64_t *>(T->slots), kEmptyKey64, bytes / 8);
         else
-            fill_kernel<int32_t><<<g, 256, 0, stream>>>(reinterpret_cast<int32_t *>(T->slots), kEmptyKey32, (size_t)L.slots);
-        if (L.code_bits)
-            ok = ok && cudaMemsetAsync(T->codes, 0, (size_t)L.slots * (size_t)(L.code_bits / 8), stream) == cudaSuccess;
+            fill_kernel<int32_t><<<g, 256, 0, stream>>>(reinterpret_cast<int32_t *>(T->slots), kEmptyKey32, bytes / 4);
     }
     if (ok && B.dim.n > 0) build_kernel<<<grid_for(B.dim.n, dev.sm_count), 256, 0, stream>>>(B);
     if (ok && direct) {

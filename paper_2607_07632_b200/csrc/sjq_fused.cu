@@ -80,6 +80,42 @@ __global__ void __launch_bounds__(256) merge_kernel(const MergeParams M)
         group_table_add(M.gkeys, M.gsums, M.gcounts, M.gmask, M.status, M.keys[i], M.sums[i], M.counts[i]);
 }
 
+struct SampleParams {
+    const void *col[SJQ_MAX_PREDS];
+    DPred preds[SJQ_MAX_PREDS];
+    int32_t npreds;
+    int64_t n;       // rows of the table
+    int64_t groups;  // sampled groups of four consecutive rows
+    int64_t stride;  // rows between the starts of two sampled groups (a multiple of 4)
+    unsigned long long *counts; // [0] rows sampled, [1 + p] rows among them passing predicate p
+};
+
+// Every predicate evaluated on its own over an evenly spaced sample of the table: the marginal pass
+// fractions the planner orders the stages by.  One 16- or 32-byte load per predicate and group.
+__global__ void __launch_bounds__(256) sample_kernel(const __grid_constant__ SampleParams S)
+{
+    __shared__ unsigned int block_counts[SJQ_MAX_PREDS + 1];
+    if (threadIdx.x <= SJQ_MAX_PREDS) block_counts[threadIdx.x] = 0;
+    __syncthreads();
+    const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g < S.groups) {
+        const int64_t r0 = g * S.stride;
+        const int rows = (int)(S.n - r0 < 4 ? S.n - r0 : 4);
+        atomicAdd(&block_counts[0], (unsigned int)rows);
+        for (int p = 0; p < S.npreds; ++p) {
+            const DPred &d = S.preds[p];
+            unsigned int pass = 0;
+            for (int r = 0; r < rows; ++r)
+                pass += d.is64 ? pred_eval<int64_t>(d, static_cast<const int64_t *>(S.col[p])[r0 + r])
+                               : pred_eval<int32_t>(d, static_cast<const int32_t *>(S.col[p])[r0 + r]);
+            if (pass) atomicAdd(&block_counts[1 + p], pass);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x <= S.npreds && block_counts[threadIdx.x])
+        atomicAdd(&S.counts[threadIdx.x], (unsigned long long)block_counts[threadIdx.x]);
+}
+
 typedef void (*fused_fn)(const RunParams);
 
 fused_fn pick_kernel(int agg, bool mul, bool hash)
@@ -161,6 +197,28 @@ sjq_status clear_launch(int64_t *sums, int64_t *counts, int64_t cells, int64_t *
     if (blocks > (int64_t)sm_count * 8) blocks = (int64_t)sm_count * 8;
     if (blocks < 1) blocks = 1;
     clear_kernel<<<(int)blocks, 256, 0, stream>>>(C);
+    return cudaGetLastError() == cudaSuccess ? SJQ_OK : SJQ_ERR_CUDA;
+}
+
+// Enqueue the sampling kernel: `counts` (device, SJQ_MAX_PREDS + 1 words) is cleared first.
+sjq_status sample_launch(const sjq_col *fact, const DPred *preds, int npreds, int64_t n, unsigned long long *counts,
+                         cudaStream_t stream)
+{
+    if (cudaMemsetAsync(counts, 0, (SJQ_MAX_PREDS + 1) * sizeof(unsigned long long), stream) != cudaSuccess)
+        return SJQ_ERR_CUDA;
+    if (n <= 0 || npreds <= 0) return SJQ_OK;
+    SampleParams S{};
+    for (int p = 0; p < npreds; ++p) {
+        S.col[p] = fact[preds[p].col].data;
+        S.preds[p] = preds[p];
+    }
+    S.npreds = npreds;
+    S.n = n;
+    const int64_t quads = (n + 3) / 4;
+    const int64_t want = (int64_t)1 << 16; // 65 536 groups of four rows
+    S.groups = quads < want ? quads : want;
+    S.stride = 4 * (quads / S.groups);
+    sample_kernel<<<(int)((S.groups + 255) / 256), 256, 0, stream>>>(S);
     return cudaGetLastError() == cudaSuccess ? SJQ_OK : SJQ_ERR_CUDA;
 }
 

@@ -28,11 +28,26 @@ bool canon_pred(const sjq_pred &p, int dtype, DPred *out);
 // ---------------------------------------------------------------- tables
 constexpr int64_t kEmptyKey64 = INT64_MIN;
 constexpr int32_t kEmptyKey32 = INT32_MIN;
-// An open-addressing table is read one 32-byte bucket at a time: a key's linear probe starts at the
-// first slot of its home bucket, so a lookup loads whole buckets and stops at the first one with a
-// free slot.
-constexpr int kBucketKeys64 = 4;
-constexpr int kBucketKeys32 = 8;
+// An open-addressing table is an array of 64-byte buckets, each holding K keys followed by their K payload
+// codes, so that a hit costs one DRAM burst (Section 3.3's point about the unpacked table: what a probe
+// touches decides its cost).  A key's linear probe starts at its home bucket (multiply-high range reduction
+// of its hash, so the bucket count need not be a power of two), a lookup loads whole buckets and stops at
+// the first one with a free slot; inserts fill a bucket's slots in order.
+constexpr int kBucketBytes = 64;
+// keys per bucket for a key of kb bytes with a code of cb bytes (0, 4 or 8): the largest K with
+// K * kb rounded up to the code's alignment + K * cb <= 64
+__host__ __device__ constexpr int bucket_code_offset(int kb, int cb, int k)
+{
+    return cb == 0 ? k * kb : (k * kb + cb - 1) / cb * cb;
+}
+__host__ __device__ constexpr int bucket_keys(int kb, int cb)
+{
+    int k = kBucketBytes / (kb + cb);
+    while (k > 1 && bucket_code_offset(kb, cb, k) + k * cb > kBucketBytes) --k;
+    return k;
+}
+static_assert(bucket_keys(8, 4) == 5 && bucket_keys(8, 8) == 4 && bucket_keys(8, 0) == 8, "64-bit keys");
+static_assert(bucket_keys(4, 4) == 8 && bucket_keys(4, 8) == 5 && bucket_keys(4, 0) == 16, "32-bit keys");
 constexpr size_t kTableHeaderBytes = 256; // device-side counters at the start of table_mem
 
 } // namespace sjq
@@ -40,10 +55,9 @@ constexpr size_t kTableHeaderBytes = 256; // device-side counters at the start o
 struct sjq_table {
     sjq_dim_layout layout;
     char *base;          // table_mem
-    char *slots;         // direct: code array / bitmap words; hash: key array
-    char *codes;         // hash: code array (NULL when no payload)
-    char *filter;        // hash: presence bitmap (NULL when none)
-    size_t slots_bytes;  // bytes of the direct array (for shared-memory staging)
+    char *slots;         // direct: code array / bitmap words; hash: bucket array
+    char *filter;        // presence bitmap (NULL when none)
+    size_t slots_bytes;  // bytes of the direct array (for shared-memory staging) or of the bucket array
     uint32_t magic;
 };
 
@@ -61,6 +75,12 @@ __host__ __device__ inline uint64_t hash64(uint64_t k)
     k ^= k >> 32;
     k *= 0x9E3779B97F4A7C15ULL;
     return k >> 32;
+}
+
+// Home bucket of a key in a table of `buckets` buckets (any count below 2^32).
+__host__ __device__ inline uint32_t home_bucket(uint64_t k, uint32_t buckets)
+{
+    return (uint32_t)((hash64(k) * (uint64_t)buckets) >> 32);
 }
 
 // A second, independent hash for the presence bitmap in front of an open-addressing table.

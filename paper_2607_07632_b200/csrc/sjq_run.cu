@@ -36,6 +36,8 @@ sjq_status compact_launch(const int64_t *gkeys, const int64_t *gsums, const int6
                           int64_t dense_base, int64_t *keys, int64_t *sums, int64_t *counts, int64_t capacity,
                           int64_t *n_groups, int32_t *status, int sm_count, cudaStream_t stream);
 
+sjq_status sample_launch(const sjq_col *fact, const DPred *preds, int npreds, int64_t n, unsigned long long *counts,
+                         cudaStream_t stream);
 sjq_status merge_launch(const int64_t *keys, const int64_t *sums, const int64_t *counts, int64_t n, int64_t *gkeys,
                         int64_t *gsums, int64_t *gcounts, uint64_t gmask, int32_t *status, int sm_count,
                         cudaStream_t stream);
@@ -88,15 +90,20 @@ sjq_status order_stages(const sjq_col *fact, const sjq_pred *preds, int npreds, 
 {
     std::vector<StageSpec> &specs = *specs_out;
     std::vector<int> &order = *order_out;
+    // a measured pass fraction (parts per million) replaces the estimate where the caller supplies one
+    auto hinted = [&](int i, double estimate) {
+        const int32_t ppm = opts.pass_ppm[i];
+        return ppm > 0 ? std::min(1.0, ppm / 1e6) : estimate;
+    };
     for (int p = 0; p < npreds; ++p) {
         const double bytes = fact[preds[p].col].dtype == SJQ_I64 ? 2.0 : 1.0;
-        specs.push_back({ST_PRED, p, preds[p].col, pred_selectivity(preds[p]), bytes, 0});
+        specs.push_back({ST_PRED, p, preds[p].col, hinted(p, pred_selectivity(preds[p])), bytes, 0});
     }
     for (int j = 0; j < njoins; ++j) {
         const sjq_table *T = joins[j].table;
         const sjq_dim_layout &L = T->layout;
         const double bytes = L.key_dtype == SJQ_I64 ? 2.0 : 1.0;
-        double sel = L.dim_rows > 0 ? (double)L.entries / (double)L.dim_rows : 0.0;
+        const double sel = hinted(npreds + j, L.dim_rows > 0 ? (double)L.entries / (double)L.dim_rows : 0.0);
         // bytes a filter stage on this table touches: the presence bitmap when a direct table has one
         const size_t tb = (L.kind <= SJQ_TABLE_DIRECT_U64 && L.filter_bits > 0 && T->filter && !opts.no_filter_bitmap)
                               ? (size_t)(L.filter_bits / 8)
@@ -159,6 +166,70 @@ extern "C" sjq_status sjq_run_workspace_bytes(const sjq_result_spec *spec, size_
         return SJQ_ERR_INVALID_ARG;
     }
     return SJQ_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Measured predicate selectivities.
+namespace {
+
+int32_t ppm_of(int64_t passed, int64_t sampled)
+{
+    if (sampled <= 0) return 0; // nothing sampled: no hint
+    const int64_t ppm = (passed * 1000000 + sampled / 2) / sampled;
+    return (int32_t)std::min<int64_t>(std::max<int64_t>(ppm, 1), 1000000);
+}
+
+} // namespace
+
+extern "C" sjq_status sjq_pred_sample_begin(const sjq_col *fact, int nfact, const sjq_pred *preds, int npreds,
+                                            void *scratch_dev, int64_t *host_counts, void *stream_)
+{
+    if (!fact || nfact <= 0 || nfact > 64 || npreds < 0 || npreds > SJQ_MAX_PREDS || (npreds && !preds) ||
+        !scratch_dev || !host_counts)
+        return SJQ_ERR_INVALID_ARG;
+    if (!aligned16(scratch_dev)) return SJQ_ERR_ALIGN;
+    const int64_t n = fact[0].n;
+    DPred d[SJQ_MAX_PREDS];
+    for (int c = 0; c < nfact; ++c) {
+        if (fact[c].n != n || n < 0 || (fact[c].dtype != SJQ_I32 && fact[c].dtype != SJQ_I64) ||
+            (n > 0 && !fact[c].data))
+            return SJQ_ERR_INVALID_ARG;
+        if (!aligned16(fact[c].data)) return SJQ_ERR_ALIGN;
+    }
+    for (int p = 0; p < npreds; ++p) {
+        if (preds[p].col < 0 || preds[p].col >= nfact) return SJQ_ERR_INVALID_ARG;
+        if (!canon_pred(preds[p], fact[preds[p].col].dtype, &d[p])) return SJQ_ERR_INVALID_ARG;
+    }
+    cudaStream_t stream = (cudaStream_t)stream_;
+    unsigned long long *counts = static_cast<unsigned long long *>(scratch_dev);
+    sjq_status st = sample_launch(fact, d, npreds, n, counts, stream);
+    if (st != SJQ_OK) return st;
+    if (cudaMemcpyAsync(host_counts, counts, (SJQ_MAX_PREDS + 1) * sizeof(int64_t), cudaMemcpyDeviceToHost, stream) !=
+        cudaSuccess) {
+        (void)cudaGetLastError();
+        return SJQ_ERR_CUDA;
+    }
+    return SJQ_OK;
+}
+
+extern "C" sjq_status sjq_pred_sample_end(const int64_t *host_counts, int npreds, int32_t *pass_ppm)
+{
+    if (!host_counts || npreds < 0 || npreds > SJQ_MAX_PREDS || (npreds && !pass_ppm)) return SJQ_ERR_INVALID_ARG;
+    for (int p = 0; p < npreds; ++p) pass_ppm[p] = ppm_of(host_counts[1 + p], host_counts[0]);
+    return SJQ_OK;
+}
+
+extern "C" sjq_status sjq_pred_sample(const sjq_col *fact, int nfact, const sjq_pred *preds, int npreds,
+                                      void *scratch_dev, void *stream_, int32_t *pass_ppm)
+{
+    int64_t h[SJQ_MAX_PREDS + 1];
+    sjq_status st = sjq_pred_sample_begin(fact, nfact, preds, npreds, scratch_dev, h, stream_);
+    if (st != SJQ_OK) return st;
+    if (cudaStreamSynchronize((cudaStream_t)stream_) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SJQ_ERR_CUDA;
+    }
+    return sjq_pred_sample_end(h, npreds, pass_ppm);
 }
 
 extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *preds, int npreds,
@@ -287,19 +358,24 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
                              : L.kind == SJQ_TABLE_HASH_I32    ? OP_HASH32
                                                                : OP_HASH64);
             S.tab = T->slots;
-            S.codes = T->codes;
-            if (sp.prefilter == 1) {
-                S.op = OP_HASHBITS;
-                S.tab = T->filter;
-                S.codes = nullptr;
-            }
+            S.codes = nullptr;
             S.kmin = L.kmin;
             S.last = (uint64_t)L.slots - 1;
+            if (L.kind >= SJQ_TABLE_HASH_I32) {
+                S.last = (uint64_t)(T->slots_bytes / kBucketBytes); // bucket count
+                if (sp.prefilter == 1) {
+                    S.op = OP_HASHBITS;
+                    S.tab = T->filter;
+                    // a table that cannot stay in L2 beside the streamed columns: rows that pass the bitmap
+                    // prefetch their home bucket for the exact probe that follows
+                    if (T->slots_bytes > ((size_t)8 << 20)) S.codes = T->slots;
+                }
+            }
             S.kmin32 = (int32_t)L.kmin;
             S.last32 = (uint32_t)std::min<uint64_t>((uint64_t)L.slots - 1, 0xFFFFFFFFull);
             // with 2^32 slots or more every 32-bit index is in range and nothing is clamped
             S.clamp32 = (uint32_t)std::min<uint64_t>((uint64_t)L.slots, 0xFFFFFFFFull);
-            S.hmask = sp.prefilter == 1 ? (uint64_t)L.filter_bits - 1 : (uint64_t)L.slots - 1;
+            S.hmask = sp.prefilter == 1 ? (uint64_t)L.filter_bits - 1 : 0;
             S.pmin0 = L.pay_min[0];
             S.pmin1 = L.pay_min[1];
             S.pbits0 = (uint8_t)L.pay_bits[0];
@@ -342,7 +418,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     if (!direct) {
         nd0 = 1;
         if (opts.compaction != 2) {
-            const double dense_reach = opts.dense_reach_permille > 0 ? opts.dense_reach_permille / 1000.0 : 0.3;
+            const double dense_reach = 0.3;
             while (nd0 < nfilter && specs[order[nd0]].sel < 0.9 && reach[nd0] > dense_reach &&
                    specs[order[nd0]].prefilter != 2)
                 ++nd0;
@@ -746,9 +822,10 @@ enum { HOST_COPY = 0, HOST_IN_PLACE = 1, HOST_SKIP = 2 };
 // for (< 0: never).  Invalid queries get "copy everything" and are rejected later by sjq_run.
 void host_transfer_plan(const sjq_col *fact_host, int nfact, const sjq_pred *preds, int npreds,
                         const sjq_join *joins, int njoins, const sjq_key_expr *key, const sjq_agg_expr *agg,
-                        const sjq_run_opts &opts, std::vector<int> *how_out, std::vector<const char *> *base_out,
+                        sjq_run_opts *opts_io, std::vector<int> *how_out, std::vector<const char *> *base_out,
                         std::vector<double> *need_out)
 {
+    sjq_run_opts &opts = *opts_io; // predicates measured here are written back as hints for the runs
     std::vector<int> &how = *how_out;
     std::vector<const char *> &direct_base = *base_out;
     how.assign(nfact, HOST_COPY);
@@ -768,7 +845,33 @@ void host_transfer_plan(const sjq_col *fact_host, int nfact, const sjq_pred *pre
     ok = ok && term_ok(agg->x) && (agg->op == SJQ_AGG_COL || term_ok(agg->y));
     std::vector<StageSpec> specs;
     std::vector<int> order;
-    if (!ok || order_stages(fact_host, preds, npreds, joins, njoins, opts, &specs, &order) != SJQ_OK) return;
+    // The columns are in host memory here, so predicates without a measured pass fraction are measured on
+    // the spot: a few thousand evenly spaced rows read by the host.  (A guess that is far too low would send
+    // a column most rows need over the bus sector by sector.)
+    sjq_run_opts &measured = opts;
+    for (int p = 0; ok && p < npreds; ++p) {
+        if (measured.pass_ppm[p] > 0) continue;
+        const sjq_col &c = fact_host[preds[p].col];
+        DPred d;
+        if (!c.data || !canon_pred(preds[p], c.dtype, &d)) continue;
+        const int64_t samples = std::min<int64_t>(n, 8192), stride = n / samples;
+        int64_t pass = 0;
+        for (int64_t i = 0; i < samples; ++i) {
+            const int64_t r = i * stride;
+            const int64_t v = c.dtype == SJQ_I64 ? static_cast<const int64_t *>(c.data)[r]
+                                                 : (int64_t) static_cast<const int32_t *>(c.data)[r];
+            bool in;
+            if (d.nset) {
+                in = false;
+                for (int k = 0; k < d.nset; ++k) in |= v == d.set[k];
+            } else {
+                in = (v >= d.lo && v <= d.hi) != (bool)d.neg;
+            }
+            pass += in;
+        }
+        measured.pass_ppm[p] = ppm_of(pass, samples);
+    }
+    if (!ok || order_stages(fact_host, preds, npreds, joins, njoins, measured, &specs, &order) != SJQ_OK) return;
     std::vector<double> &need = *need_out;
     need.assign(nfact, -1.0);
     double reach = 1.0;
@@ -812,7 +915,7 @@ extern "C" sjq_status sjq_host_transfer_plan(const sjq_col *fact_host, int nfact
     std::vector<int> h;
     std::vector<const char *> base;
     std::vector<double> need;
-    host_transfer_plan(fact_host, nfact, preds, npreds, joins, njoins, key, agg, opts, &h, &base, &need);
+    host_transfer_plan(fact_host, nfact, preds, npreds, joins, njoins, key, agg, &opts, &h, &base, &need);
     for (int c = 0; c < nfact; ++c) {
         how[c] = h[c];
         if (share) share[c] = need[c] < 0 ? 0.0 : need[c];
@@ -853,7 +956,7 @@ extern "C" sjq_status sjq_run_host(const sjq_col *fact_host, int nfact, const sj
     std::vector<int> how;
     std::vector<const char *> direct_base;
     std::vector<double> need_share;
-    host_transfer_plan(fact_host, nfact, preds, npreds, joins, njoins, key, agg, opts, &how, &direct_base, &need_share);
+    host_transfer_plan(fact_host, nfact, preds, npreds, joins, njoins, key, agg, &opts, &how, &direct_base, &need_share);
 
     // internal streams start after whatever is already queued on the caller's stream
     if (cudaEventRecord(hp->start, stream) != cudaSuccess) return SJQ_ERR_CUDA;

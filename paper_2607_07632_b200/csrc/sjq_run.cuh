@@ -54,12 +54,12 @@ constexpr int kMaxQueues = 3;            // queue-fed levels per warp (the last 
 
 struct DStage {
     const void *col;   // fact column read by this stage
-    const void *tab;   // direct: code array / bitmap words; hash: key array
-    const void *codes; // hash: payload codes
+    const void *tab;   // direct: code array / bitmap words; hash: bucket array; presence bitmap: its words
+    const void *codes; // presence bitmap of a hash table: the bucket array to prefetch from (NULL = no prefetch)
     int64_t kmin;      // direct: slot index = key - kmin
-    uint64_t last;     // direct: last valid slot index (slots - 1)
+    uint64_t last;     // direct: last valid slot index (slots - 1); hash (and its bitmap stage): bucket count
     int64_t lo, hi;    // 64-bit predicate range
-    uint64_t hmask;    // hash: slots - 1
+    uint64_t hmask;    // presence bitmap of a hash table: bits - 1
     int64_t pmin0, pmin1;
     uint64_t pmask0;
     int64_t mult[9];

@@ -8,7 +8,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from dataclasses import dataclass, field
+from dataclasses import dataclass, field, replace
 from typing import Optional, Sequence
 
 import torch
@@ -91,10 +91,10 @@ class _RunOpts(ctypes.Structure):
                 ("agg_path", ctypes.c_int32), ("smem_tables", ctypes.c_int32), ("compaction", ctypes.c_int32),
                 ("accumulate", ctypes.c_int32), ("norder", ctypes.c_int32),
                 ("order", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS)), ("event_before", ctypes.c_void_p),
-                ("event_after", ctypes.c_void_p), ("dense_reach_permille", ctypes.c_int32), ("specialise", ctypes.c_int32),
+                ("event_after", ctypes.c_void_p), ("specialise", ctypes.c_int32),
                 ("rows_per_lane", ctypes.c_int32), ("no_filter_bitmap", ctypes.c_int32),
                 ("host_copy_all", ctypes.c_int32), ("dense_slots", ctypes.c_int32),
-                ("group_hash_always", ctypes.c_int32), ("reserved", ctypes.c_int32 * 1)]
+                ("group_hash_always", ctypes.c_int32), ("pass_ppm", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS))]
 
 
 class RunInfo(ctypes.Structure):
@@ -122,13 +122,13 @@ class RunOpts:
     accumulate: bool = False
     order: Sequence[int] = ()
     events: Optional[tuple] = None  # (torch.cuda.Event, torch.cuda.Event), both already recorded once
-    dense_reach_permille: int = 0  # experiment knob: level 0 keeps stages reached by more than this share of rows
     specialise: bool = False  # compile the fused kernel for this query's shape at run time (cached per shape)
     rows_per_lane: int = 0  # queue-fed levels: 0 auto, 4, or 8 (8 needs specialise)
     no_filter_bitmap: bool = False  # filter stages probe the code array of a direct table, not its bitmap
     host_copy_all: bool = False  # run_host: copy every referenced column instead of reading sparse ones in place
     dense_slots: int = 0  # level 0: 0 auto, 2, or 4 groups of four rows per thread (4 needs specialise)
     group_hash_always: bool = False  # HASHED: keep the group hash table even when the key domain is small
+    pass_ppm: Sequence[int] = ()  # measured pass fractions (parts per million): predicates, then joins; 0 = unknown
 
     def to_c(self) -> _RunOpts:
         o = _RunOpts()
@@ -138,7 +138,8 @@ class RunOpts:
         o.norder = len(self.order)
         for i, v in enumerate(self.order):
             o.order[i] = v
-        o.dense_reach_permille = self.dense_reach_permille
+        for i, v in enumerate(self.pass_ppm):
+            o.pass_ppm[i] = int(v)
         o.specialise = int(self.specialise)
         o.rows_per_lane = self.rows_per_lane
         o.no_filter_bitmap = int(self.no_filter_bitmap)
@@ -180,6 +181,13 @@ def lib():
         L.sjq_table_info.argtypes = [vp, ctypes.POINTER(DimLayout)]
         L.sjq_table_destroy.restype = None
         L.sjq_table_destroy.argtypes = [vp]
+        L.sjq_pred_sample.restype = ctypes.c_int32
+        L.sjq_pred_sample.argtypes = [ctypes.POINTER(_Col), ip, ctypes.POINTER(_Pred), ip, vp, vp,
+                                      ctypes.POINTER(ctypes.c_int32)]
+        L.sjq_pred_sample_begin.restype = ctypes.c_int32
+        L.sjq_pred_sample_begin.argtypes = [ctypes.POINTER(_Col), ip, ctypes.POINTER(_Pred), ip, vp, vp, vp]
+        L.sjq_pred_sample_end.restype = ctypes.c_int32
+        L.sjq_pred_sample_end.argtypes = [vp, ip, ctypes.POINTER(ctypes.c_int32)]
         L.sjq_run_workspace_bytes.restype = ctypes.c_int32
         L.sjq_run_workspace_bytes.argtypes = [ctypes.POINTER(_ResultSpec), ctypes.POINTER(ctypes.c_size_t)]
         L.sjq_run.restype = ctypes.c_int32
@@ -385,6 +393,59 @@ def build_tables(builders: dict) -> dict:
     for b in builders.values():
         torch.cuda.current_stream(b.device).wait_stream(b.side)
     return tables
+
+
+def sample_preds(fact: dict, preds=()) -> tuple:
+    """sjq_pred_sample: measured pass fraction (parts per million) of every fact predicate, in the form
+    RunOpts.pass_ppm takes.  Synchronises the current stream."""
+    if not preds:
+        return ()
+    names = list(fact.keys())
+    tensors = [fact[n] for n in names]
+    device = tensors[0].device
+    with torch.cuda.device(device):
+        carr = _cols(tensors)
+        parr, keep = _preds(preds, names)
+        scratch = torch.empty(PLAN_SCRATCH_BYTES, dtype=torch.uint8, device=device)
+        out = (ctypes.c_int32 * len(preds))()
+        rc = lib().sjq_pred_sample(carr, len(names), parr, len(preds), scratch.data_ptr(), _stream_ptr(device), out)
+        if rc != 0:
+            raise SjqError(rc, "sjq_pred_sample")
+    return tuple(out)
+
+
+class PredSampler:
+    """The fact predicates of a query prepared for repeated sampling on a side stream (sjq_pred_sample_begin /
+    _end), so that a planning step shares one wait between the dimension scans and the sample."""
+
+    def __init__(self, fact: dict, preds=()):
+        self.names = list(fact.keys())
+        self.tensors = [fact[n] for n in self.names]
+        self.device = self.tensors[0].device
+        self.npreds = len(preds)
+        with torch.cuda.device(self.device):
+            self.carr = _cols(self.tensors)
+            self.parr, self._keep = _preds(preds, self.names)
+            self.scratch = torch.empty(PLAN_SCRATCH_BYTES, dtype=torch.uint8, device=self.device)
+            self.counts = torch.zeros(MAX_PREDS + 1, dtype=torch.int64, pin_memory=True)
+            self.side = torch.cuda.Stream(self.device)
+        self.out = (ctypes.c_int32 * max(1, self.npreds))()
+
+    def begin(self):
+        if self.npreds:
+            rc = lib().sjq_pred_sample_begin(self.carr, len(self.names), self.parr, self.npreds,
+                                             self.scratch.data_ptr(), self.counts.data_ptr(), self.side.cuda_stream)
+            if rc != 0:
+                raise SjqError(rc, "sjq_pred_sample_begin")
+
+    def end(self) -> tuple:
+        if not self.npreds:
+            return ()
+        self.side.synchronize()
+        rc = lib().sjq_pred_sample_end(self.counts.data_ptr(), self.npreds, self.out)
+        if rc != 0:
+            raise SjqError(rc, "sjq_pred_sample_end")
+        return tuple(self.out[: self.npreds])
 
 
 @dataclass
@@ -665,7 +726,12 @@ def build_workload_tables(w, dims: dict) -> dict:
 
 
 def run_workload(w, fact: dict, tables: dict, opts: Optional[RunOpts] = None,
-                 result: Optional[Result] = None) -> Result:
+                 result: Optional[Result] = None, sample: bool = False) -> Result:
+    """Run a workload description.  sample: measure the fact predicates' pass fractions first (one small
+    kernel and a stream synchronisation) unless the options already carry measured ones."""
     fact = {c.name: fact[c.name] for c in w.fact_cols}
+    if sample and w.preds and not (opts is not None and any(opts.pass_ppm)):
+        opts = replace(opts) if opts is not None else RunOpts()
+        opts.pass_ppm = sample_preds(fact, w.preds)
     return run(fact, w.preds, [(fk, tables[dn]) for fk, dn in w.joins], w.key, w.agg, w.mode, w.num_groups,
                w.capacity, opts, result)

@@ -146,7 +146,7 @@ def test_build_rejects_inconsistent_layouts_on_the_host(libsjq):
         L.dim_rows = n + 1  # planned for another dimension
         assert build(L) == 1
     L = hashed()
-    L.slots = 2040  # an open-addressing table is made of whole buckets
+    L.slots = 2044  # an open-addressing table is made of whole buckets
     with pytest.raises(b.SjqError):
         b.layout_bytes(L)
     L.table_bytes = hashed().table_bytes
@@ -160,3 +160,41 @@ def test_build_rejects_inconsistent_layouts_on_the_host(libsjq):
     L = direct()
     L.kind, L.code_bits = 1, 0  # a bitmap table cannot carry the payload the call names
     assert build(L) == 1
+
+
+def test_mis_guessed_predicates_do_not_send_dense_columns_over_the_bus_piecemeal(libsjq):
+    """sjq_run_host reads a column in place over the bus when the planner expects only a few per cent of the
+    rows to reach it.  By their operators alone two equality predicates look as if they kept 1 % of the rows;
+    here they keep all of them.  The planning call measures predicates on host-resident columns, so every
+    column must be planned as a whole copy (and with predicates that keep nothing, later columns are expected
+    to be reached by almost no row)."""
+    import torch
+
+    import paper_2607_07632_b200.sjq as b
+    from datagen.workloads import AggExpr, Pred, Term
+
+    n = 100_000
+    fact = {"a": torch.full((n,), 7, dtype=torch.int32), "b": torch.full((n,), 9, dtype=torch.int64),
+            "m": torch.arange(n, dtype=torch.int32), "unused": torch.zeros(n, dtype=torch.int32)}
+    agg = AggExpr("COL", Term("FACT", "m"))
+    plan = b.host_transfer_plan(fact, (Pred("a", "EQ", 7), Pred("b", "EQ", 9)), (), None, agg)
+    assert plan["unused"][0] == "not transferred"
+    for c in ("a", "b", "m"):
+        assert plan[c] == ("copy", 1.0), (c, plan[c])
+    # the same predicates keeping nothing: the measured share of rows reaching the later columns is tiny
+    plan = b.host_transfer_plan(fact, (Pred("a", "EQ", 8), Pred("b", "EQ", 9)), (), None, agg)
+    assert plan["a"][1] == 1.0 and plan["m"][1] < 1e-4
+    # a caller's own measured fractions are taken as they are
+    plan = b.host_transfer_plan(fact, (Pred("a", "EQ", 8), Pred("b", "EQ", 9)), (), None, agg,
+                                b.RunOpts(pass_ppm=(500_000, 500_000)))
+    assert abs(plan["m"][1] - 0.25) < 1e-9
+
+
+def test_sampled_counters_become_parts_per_million(libsjq):
+    import paper_2607_07632_b200.sjq as b
+
+    counts = (ctypes.c_int64 * 17)(*([262144, 0, 26, 262144, 131072] + [0] * 12))
+    out = (ctypes.c_int32 * 4)()
+    assert b.lib().sjq_pred_sample_end(counts, 4, out) == 0
+    assert list(out) == [1, 99, 1_000_000, 500_000]  # none seen -> 1 ppm, never "unknown"
+    assert b.lib().sjq_pred_sample_end(None, 4, out) == 1
