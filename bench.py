@@ -717,6 +717,39 @@ def main():
     return 0
 
 
+def unfused_bytes_model(w, res, tables):
+    """DRAM bytes each pass of the operator-at-a-time arm moves, by construction: every filter pass reads its
+    whole fact column, reads (except the first) and writes one flag byte per row, and a gathering join writes
+    its payload code for the 32-byte sectors holding a survivor; the aggregation pass reads the flags and, for
+    sectors holding a survivor, the measure columns and the materialised payloads."""
+    survivors = int(res.counts.sum().item()) if w.mode != "HASHED" else int(res.counts[: int(res.n_groups.item())].sum().item())
+    frac = stage_pass_fractions(w, tables, survivors)
+    plan = res.info.describe()
+    cols = [p.col for p in w.preds] + [fk for fk, _ in w.joins]
+    n, reach, passes, seen = w.n_rows, 1.0, [], set()
+    nfilter = len(w.preds) + len(w.joins)
+    gathered = {j for t in ((w.key.terms if w.key else ()) + (w.agg.x,) + ((w.agg.y,) if w.agg.y else ()))
+                if t.src == "PAYLOAD" for j in [int(t.a)]}
+    first = True
+    for idx in plan["order"]:
+        if idx < 0 or idx in seen:
+            continue
+        seen.add(idx)
+        width = 8 if w.fact_col(cols[idx]).is64 else 4
+        b = n * width + (0 if first else n) + n
+        reach *= frac.get(idx, 1.0)
+        if idx >= len(w.preds) and (idx - len(w.preds)) in gathered:
+            b += n * 4 * (1.0 - (1.0 - reach) ** 8)
+        passes.append({"stage": idx, "bytes": int(b)})
+        first = False
+    sector = 1.0 - (1.0 - reach) ** 8
+    measure = {t.a for t in ((w.key.terms if w.key else ()) + (w.agg.x,) + ((w.agg.y,) if w.agg.y else ())) if t.src == "FACT"}
+    agg = (n if nfilter else 0) + sum(n * (8 if w.fact_col(c).is64 else 4) * sector for c in measure) + \
+        len(gathered) * n * 4 * sector
+    passes.append({"stage": "aggregate", "bytes": int(agg)})
+    return {"passes": passes, "total": int(sum(p["bytes"] for p in passes))}
+
+
 def run_ablation(sjq, W, device, specialise=True):
     """The paper's A/B experiments restated on this kernel (run-only, min of 5 after a warm-up):
     lazy vs unconditional column loads (its tile-vs-direct table), survivor queues on/off, packed
@@ -748,7 +781,10 @@ def run_ablation(sjq, W, device, specialise=True):
             e1.record()
             torch.cuda.synchronize()
             ts.append(e0.elapsed_time(e1))
-        out.append({"workload": w.name, "variant": label, "ms_min": min(ts),
+        row_extra = {}
+        if label == UNFUSED:
+            row_extra["bytes_moved_model"] = unfused_bytes_model(w, res, tables)
+        out.append({"workload": w.name, "variant": label, "ms_min": min(ts), **row_extra,
                     "rows_per_s": w.n_rows / (min(ts) / 1000.0), "status": res.status(),
                     "table_kinds": {k: t.layout.kind_name for k, t in tables.items()},
                     "table_bytes": {k: int(t.layout.table_bytes) for k, t in tables.items()},
@@ -756,6 +792,7 @@ def run_ablation(sjq, W, device, specialise=True):
         return fact, dims
 
     INTERPRETED = "query descriptor interpreted (no run-time specialisation)"
+    UNFUSED = "operator at a time: one kernel per predicate / join over a flag array, payload columns materialised"
     for mk in (W.config3, W.config2):
         w = mk()
         fact, dims = timed(w, "default")
@@ -768,7 +805,8 @@ def run_ablation(sjq, W, device, specialise=True):
                             ("every direct table in shared memory that fits", sjq.RunOpts(smem_tables=2)),
                             ("no table in shared memory", sjq.RunOpts(smem_tables=1)),
                             ("filter stages probe the packed code arrays, not their presence bitmaps",
-                             sjq.RunOpts(no_filter_bitmap=True))):
+                             sjq.RunOpts(no_filter_bitmap=True)),
+                            (UNFUSED, sjq.RunOpts(unfused_scratch=sjq.unfused_scratch(w.n_rows, len(w.joins), device)))):
             try:
                 timed(w, label, opts, fact=fact, dims=dims)
             except sjq.SjqError as e:

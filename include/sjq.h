@@ -126,6 +126,9 @@ enum {
     SJQ_TABLE_DIRECT_U64 = 5,
     SJQ_TABLE_HASH_I32 = 6, /* open addressing over 64-byte buckets of keys and codes, linear probing, int32 keys */
     SJQ_TABLE_HASH_I64 = 7,
+    SJQ_TABLE_DIRECT_U4 = 8, /* 4 bits per key, eight codes to a 32-bit word: 0xF = miss unless every key of the
+                                range is present (entries == slots), in which case the range test alone decides */
+    SJQ_TABLE_DIRECT_U2 = 9, /* 2 bits per key, sixteen to a word; same rule */
     SJQ_TABLE_FORCE_DIRECT = 100, /* build option only */
     SJQ_TABLE_FORCE_HASH = 101    /* build option only */
 };
@@ -137,6 +140,10 @@ typedef struct sjq_build_opts {
     int32_t force_kind;       /* SJQ_TABLE_AUTO, SJQ_TABLE_FORCE_DIRECT or SJQ_TABLE_FORCE_HASH */
     int32_t hash_load_pct;    /* 0 = default 50: slots >= entries * 100 / pct, in whole 64-byte buckets; <= 90 */
     int64_t max_direct_bytes; /* 0 = default 64 MiB: larger direct tables fall back to hashing */
+    int32_t min_code_bits;    /* narrowest packed code of a direct table: 0 = default 2 (sub-byte codes where the
+                                 payload range allows: a probed structure a quarter the size of Section 3.3's byte
+                                 map stays closer to the SMs), 8 = one byte or wider, as in the paper */
+    int32_t reserved;
 } sjq_build_opts;
 
 /* Shape of a table, decided from the data by sjq_dim_plan. Plain host data. */
@@ -144,7 +151,7 @@ typedef struct sjq_dim_layout {
     int32_t kind;      /* one of SJQ_TABLE_DIRECT_* / SJQ_TABLE_HASH_* */
     int32_t key_dtype; /* SJQ_I32 / SJQ_I64 */
     int32_t npayload;
-    int32_t code_bits;                 /* width of the packed payload code stored per key (0, 8, 16, 32, 64) */
+    int32_t code_bits;                 /* width of the packed payload code stored per key (0, 2, 4, 8, 16, 32, 64) */
     int64_t dim_rows;                  /* rows of the dimension */
     int64_t entries;                   /* rows passing the filter */
     int64_t kmin, kmax;                /* key range among the passing rows (0,0 if none) */
@@ -299,6 +306,13 @@ typedef struct sjq_run_opts {
     int32_t group_hash_always; /* HASHED results: 1 = always use the group hash table; 0 = a key taken modulo M whose
                                   2M - 1 possible values fit the workspace is aggregated in a table indexed by the
                                   key itself */
+    int32_t unfused; /* 1 = ablation: run the query operator at a time instead of fused (Section 4.1's engine before
+                        fusion, Section 5.4's first step): one kernel per predicate and per join over the whole
+                        table, a flag byte per row that every operator reads and rewrites, gathered payloads
+                        written out as columns, then an aggregation kernel with global atomics.  Same result;
+                        needs `unfused_scratch`.  Ignores specialise and the queue / shared-memory options. */
+    void *unfused_scratch;       /* device scratch of at least sjq_unfused_scratch_bytes() bytes (16-byte aligned) */
+    size_t unfused_scratch_bytes;
     int32_t pass_ppm[SJQ_MAX_PREDS + SJQ_MAX_JOINS]; /* measured pass fractions in parts per million, predicates
                                   first, then joins (index npreds + join): 0 = not known, the library estimates
                                   (a fact predicate from its operator alone, a join from the share of dimension
@@ -346,6 +360,10 @@ sjq_status sjq_pred_sample(const sjq_col *fact, int nfact, const sjq_pred *preds
 sjq_status sjq_pred_sample_begin(const sjq_col *fact, int nfact, const sjq_pred *preds, int npreds,
                                  void *scratch_dev, int64_t *host_counts, void *stream);
 sjq_status sjq_pred_sample_end(const int64_t *host_counts, int npreds, int32_t *pass_ppm);
+
+/* Device bytes the operator-at-a-time ablation (sjq_run_opts.unfused) needs as scratch for a fact table of
+ * `rows` rows and `njoins` joins: one flag byte per row and one 8-byte cell per row and join. */
+sjq_status sjq_unfused_scratch_bytes(int64_t rows, int njoins, size_t *bytes);
 
 /* Device bytes needed at sjq_result.workspace for `spec` (0 unless HASHED). */
 sjq_status sjq_run_workspace_bytes(const sjq_result_spec *spec, size_t *bytes);

@@ -148,6 +148,15 @@ __device__ inline bool pack_code(const BuildParams &B, int64_t r, uint64_t *code
 
 __device__ inline void store_code(void *codes, int bits, uint64_t idx, uint64_t c)
 {
+    if (bits < 8) {
+        // several codes share a word that starts as all ones: clear this code's zero bits (the keys are
+        // unique, so no two rows touch the same bits)
+        const int per = 32 / bits;
+        const unsigned int sh = (unsigned int)(idx % (uint64_t)per) * (unsigned int)bits;
+        const unsigned int mask = ((1u << bits) - 1u) << sh;
+        atomicAnd(static_cast<unsigned int *>(codes) + idx / (uint64_t)per, ~mask | ((unsigned int)c << sh));
+        return;
+    }
     switch (bits) {
     case 8: static_cast<uint8_t *>(codes)[idx] = (uint8_t)c; break;
     case 16: static_cast<uint16_t *>(codes)[idx] = (uint16_t)c; break;
@@ -200,7 +209,7 @@ __global__ void __launch_bounds__(256) build_kernel(const __grid_constant__ Buil
             continue;
         }
         ++inserted;
-        if (B.kind <= SJQ_TABLE_DIRECT_U64) {
+        if (B.kind != SJQ_TABLE_HASH_I32 && B.kind != SJQ_TABLE_HASH_I64) {
             const uint64_t idx = (uint64_t)k - (uint64_t)B.kmin;
             if (idx >= B.span) {
                 set_status(B.status, SJQ_ERR_LAYOUT_MISMATCH);
@@ -245,9 +254,10 @@ __global__ void __launch_bounds__(256) direct_count_kernel(const __grid_constant
 {
     const uint64_t stride = (uint64_t)blockDim.x * gridDim.x;
     unsigned long long occ = 0;
-    if (B.kind == SJQ_TABLE_DIRECT_BITMAP) {
+    if (B.kind == SJQ_TABLE_DIRECT_BITMAP || B.filter) {
+        // one bit per occupied slot: the table itself, or the presence bitmap beside the codes
         const uint64_t words = (B.span + 31) >> 5;
-        const unsigned int *w = static_cast<const unsigned int *>(B.slots);
+        const unsigned int *w = B.kind == SJQ_TABLE_DIRECT_BITMAP ? static_cast<const unsigned int *>(B.slots) : B.filter;
         for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < words; i += stride) occ += __popc(w[i]);
     } else {
         for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < B.span; i += stride) {
@@ -265,9 +275,15 @@ __global__ void __launch_bounds__(256) direct_count_kernel(const __grid_constant
     if ((threadIdx.x & 31) == 0 && occ) atomicAdd(&B.header[1], occ);
 }
 
-__global__ void direct_verify_kernel(const unsigned long long *header, int32_t *status)
+// `expect_full` >= 0: the layout promises that every key of the range is present (a probe then trusts the
+// range test alone), so exactly that many rows must have been stored.
+__global__ void direct_verify_kernel(const unsigned long long *header, int32_t *status, long long expect_full)
 {
-    if (threadIdx.x == 0 && blockIdx.x == 0 && header[0] != header[1]) set_status(status, SJQ_ERR_DUP_KEY);
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        if (header[0] != header[1]) set_status(status, SJQ_ERR_DUP_KEY);
+        else if (expect_full >= 0 && header[1] != (unsigned long long)expect_full)
+            set_status(status, SJQ_ERR_LAYOUT_MISMATCH);
+    }
 }
 
 int bits_for(uint64_t range)
@@ -283,9 +299,8 @@ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 size_t direct_array_bytes(const sjq_dim_layout &L)
 {
     const uint64_t span = (uint64_t)L.slots;
-    const size_t bytes = L.kind == SJQ_TABLE_DIRECT_BITMAP ? (size_t)((span + 32) / 32 * 4)
-                                                           : (size_t)((span + 1) * (uint64_t)(L.code_bits / 8));
-    return align_up(bytes, 16);
+    const uint64_t bits = L.kind == SJQ_TABLE_DIRECT_BITMAP ? 1 : (uint64_t)L.code_bits;
+    return align_up((size_t)(((span + 1) * bits + 31) / 32 * 4), 16); // whole 32-bit words
 }
 
 // Device bytes a table of this shape occupies, recomputed from kind, slots, code_bits and filter_bits (never
@@ -295,10 +310,12 @@ size_t direct_array_bytes(const sjq_dim_layout &L)
 bool layout_table_bytes(const sjq_dim_layout &L, size_t *bytes)
 {
     if (L.slots <= 0 || L.npayload < 0 || L.npayload > SJQ_MAX_PAYLOADS || L.filter_bits < 0) return false;
-    if (L.kind >= SJQ_TABLE_DIRECT_BITMAP && L.kind <= SJQ_TABLE_DIRECT_U64) {
+    if (is_direct_kind(L.kind)) {
         if ((uint64_t)L.slots > ((uint64_t)1 << 40)) return false;
-        const int want_bits = L.kind == SJQ_TABLE_DIRECT_BITMAP ? 0 : 8 << (L.kind - SJQ_TABLE_DIRECT_U8);
-        if (L.code_bits != want_bits || (L.kind == SJQ_TABLE_DIRECT_BITMAP) != (L.npayload == 0)) return false;
+        if (L.code_bits != direct_kind_bits(L.kind) || (L.kind == SJQ_TABLE_DIRECT_BITMAP) != (L.npayload == 0))
+            return false;
+        // a sub-byte table without its presence bitmap could not tell a repeated key from a missing one
+        if (L.code_bits > 0 && L.code_bits < 8 && L.filter_bits == 0) return false;
         if (L.filter_bits != 0 &&
             (L.kind == SJQ_TABLE_DIRECT_BITMAP || L.filter_bits <= L.slots || L.filter_bits % 128 != 0))
             return false;
@@ -501,9 +518,17 @@ extern "C" sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_c
         maxcode |= range << total_bits;
         total_bits += L.pay_bits[i];
     }
+    // Narrowest code that leaves all-ones free as the miss marker; a table that holds every key of its range
+    // (entries == slots) needs no marker below one byte, because there the range test alone decides a hit.
+    const uint64_t span_if_any = (uint64_t)L.kmax - (uint64_t)L.kmin; // span - 1
+    const bool every_key = L.entries > 0 && span_if_any + 1 == (uint64_t)L.entries;
+    const int min_bits = (opts && opts->min_code_bits > 0) ? opts->min_code_bits : 2;
+    if (min_bits != 2 && min_bits != 4 && min_bits != 8) return SJQ_ERR_INVALID_ARG;
     int code_bits = 0;
     if (npayload > 0) {
-        if (maxcode < 0xFFu) code_bits = 8;
+        if (min_bits <= 2 && (every_key ? maxcode <= 0x3u : maxcode < 0x3u)) code_bits = 2;
+        else if (min_bits <= 4 && (every_key ? maxcode <= 0xFu : maxcode < 0xFu)) code_bits = 4;
+        else if (maxcode < 0xFFu) code_bits = 8;
         else if (maxcode < 0xFFFFu) code_bits = 16;
         else if (maxcode < 0xFFFFFFFFu) code_bits = 32;
         else code_bits = 64;
@@ -521,8 +546,7 @@ extern "C" sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_c
     if (direct_ok) {
         const uint64_t span = span_m1 + 1;
         // one spare entry after the last slot, never set: a probe clamps its index there instead of testing the range
-        direct_bytes = npayload == 0 ? (size_t)((span + 32) / 32 * 4) : (size_t)((span + 1) * (uint64_t)(code_bits / 8));
-        direct_bytes = align_up(direct_bytes, 16);
+        direct_bytes = align_up((size_t)(((span + 1) * (uint64_t)(npayload == 0 ? 1 : code_bits) + 31) / 32 * 4), 16);
     }
     bool use_direct;
     if (force == SJQ_TABLE_FORCE_DIRECT) {
@@ -537,6 +561,8 @@ extern "C" sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_c
         L.slots = (int64_t)(span_m1 + 1);
         L.code_bits = code_bits;
         L.kind = npayload == 0 ? SJQ_TABLE_DIRECT_BITMAP
+                 : code_bits == 2 ? SJQ_TABLE_DIRECT_U2
+                 : code_bits == 4 ? SJQ_TABLE_DIRECT_U4
                  : code_bits == 8 ? SJQ_TABLE_DIRECT_U8
                  : code_bits == 16 ? SJQ_TABLE_DIRECT_U16
                  : code_bits == 32 ? SJQ_TABLE_DIRECT_U32
@@ -607,7 +633,7 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
     B.slots = T->slots;
 
     bool ok = cudaMemsetAsync(T->base, 0, kTableHeaderBytes, stream) == cudaSuccess;
-    const bool direct = L.kind <= SJQ_TABLE_DIRECT_U64;
+    const bool direct = is_direct_kind(L.kind);
     if (direct) {
         const size_t bytes = direct_array_bytes(L);
         T->slots_bytes = bytes;
@@ -642,7 +668,8 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
     if (ok && B.dim.n > 0) build_kernel<<<grid_for(B.dim.n, dev.sm_count), 256, 0, stream>>>(B);
     if (ok && direct) {
         direct_count_kernel<<<grid_for(L.slots, dev.sm_count), 256, 0, stream>>>(B);
-        direct_verify_kernel<<<1, 32, 0, stream>>>(B.header, status_dev);
+        const bool promises_every_key = L.code_bits > 0 && L.code_bits < 8 && L.entries == L.slots;
+        direct_verify_kernel<<<1, 32, 0, stream>>>(B.header, status_dev, promises_every_key ? (long long)L.entries : -1);
     }
     if (!ok || cudaGetLastError() != cudaSuccess) {
         (void)cudaGetLastError();

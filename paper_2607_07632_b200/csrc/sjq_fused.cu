@@ -214,6 +214,7 @@ sjq_status sample_launch(const sjq_col *fact, const DPred *preds, int npreds, in
     }
     S.npreds = npreds;
     S.n = n;
+    S.counts = counts;
     const int64_t quads = (n + 3) / 4;
     const int64_t want = (int64_t)1 << 16; // 65 536 groups of four rows
     S.groups = quads < want ? quads : want;

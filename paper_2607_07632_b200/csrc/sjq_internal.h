@@ -65,6 +65,26 @@ namespace sjq {
 
 constexpr uint32_t kTableMagic = 0x534a5154u; // "SJQT"
 
+inline bool is_hash_kind(int kind) { return kind == SJQ_TABLE_HASH_I32 || kind == SJQ_TABLE_HASH_I64; }
+inline bool is_direct_kind(int kind)
+{
+    return (kind >= SJQ_TABLE_DIRECT_BITMAP && kind <= SJQ_TABLE_DIRECT_U64) || kind == SJQ_TABLE_DIRECT_U4 ||
+           kind == SJQ_TABLE_DIRECT_U2;
+}
+// width of the code a direct kind stores per key (0: bitmap)
+inline int direct_kind_bits(int kind)
+{
+    switch (kind) {
+    case SJQ_TABLE_DIRECT_U2: return 2;
+    case SJQ_TABLE_DIRECT_U4: return 4;
+    case SJQ_TABLE_DIRECT_U8: return 8;
+    case SJQ_TABLE_DIRECT_U16: return 16;
+    case SJQ_TABLE_DIRECT_U32: return 32;
+    case SJQ_TABLE_DIRECT_U64: return 64;
+    default: return 0;
+    }
+}
+
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Hash of a 64-bit key for the dimension hash tables and the group hash table: fold the high half

@@ -36,6 +36,9 @@ sjq_status compact_launch(const int64_t *gkeys, const int64_t *gsums, const int6
                           int64_t dense_base, int64_t *keys, int64_t *sums, int64_t *counts, int64_t capacity,
                           int64_t *n_groups, int32_t *status, int sm_count, cudaStream_t stream);
 
+size_t unfused_scratch_bytes(int64_t n, int gathering_joins);
+sjq_status unfused_launch(const RunParams &P, int nfilter, int agg, bool mul, bool has_hash, void *scratch,
+                          size_t scratch_bytes, int sm_count, cudaStream_t stream, int *launches);
 sjq_status sample_launch(const sjq_col *fact, const DPred *preds, int npreds, int64_t n, unsigned long long *counts,
                          cudaStream_t stream);
 sjq_status merge_launch(const int64_t *keys, const int64_t *sums, const int64_t *counts, int64_t n, int64_t *gkeys,
@@ -52,6 +55,9 @@ struct StageSpec {
     double cost;  // relative cost per row evaluated
     int prefilter; // 1: only the presence bitmap of a hashed join; 2: the exact probe that follows one
 };
+
+// share of the rows surviving all filters from which a compiled kernel drops the survivor queues
+constexpr double kDirectSurvival = 0.35;
 
 double pred_selectivity(const sjq_pred &p)
 {
@@ -105,13 +111,13 @@ sjq_status order_stages(const sjq_col *fact, const sjq_pred *preds, int npreds, 
         const double bytes = L.key_dtype == SJQ_I64 ? 2.0 : 1.0;
         const double sel = hinted(npreds + j, L.dim_rows > 0 ? (double)L.entries / (double)L.dim_rows : 0.0);
         // bytes a filter stage on this table touches: the presence bitmap when a direct table has one
-        const size_t tb = (L.kind <= SJQ_TABLE_DIRECT_U64 && L.filter_bits > 0 && T->filter && !opts.no_filter_bitmap)
+        const size_t tb = (is_direct_kind(L.kind) && L.filter_bits > 0 && T->filter && !opts.no_filter_bitmap)
                               ? (size_t)(L.filter_bits / 8)
                               : L.table_bytes;
         // relative cost of one probe: a table the L1 mostly holds, one the L2 holds (measured on the four-join
         // workload: the 3 MB map before the 175 KB bitmap when it drops twice as many rows), one in HBM
         double probe = tb <= (size_t)200 << 10 ? 0.3 : tb <= (size_t)32 << 20 ? 0.6 : 4.0;
-        if (L.kind >= SJQ_TABLE_HASH_I32 && T->filter && L.filter_bits > 0) {
+        if (is_hash_kind(L.kind) && T->filter && L.filter_bits > 0) {
             // a hashed join is two stages: its presence bitmap (cheap, passes the hits and ~1/16 of the
             // misses) early, the exact probe (expensive) on what is left
             const double fp = std::min(1.0, (double)L.entries / (double)L.filter_bits);
@@ -154,6 +160,13 @@ sjq_status order_stages(const sjq_col *fact, const sjq_pred *preds, int npreds, 
 } // namespace sjq
 
 using namespace sjq;
+
+extern "C" sjq_status sjq_unfused_scratch_bytes(int64_t rows, int njoins, size_t *bytes)
+{
+    if (rows < 0 || njoins < 0 || njoins > SJQ_MAX_JOINS || !bytes) return SJQ_ERR_INVALID_ARG;
+    *bytes = unfused_scratch_bytes(rows, njoins);
+    return SJQ_OK;
+}
 
 extern "C" sjq_status sjq_run_workspace_bytes(const sjq_result_spec *spec, size_t *bytes)
 {
@@ -349,19 +362,22 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         } else if (sp.kind == ST_PROBE) {
             const sjq_table *T = joins[sp.index].table;
             const sjq_dim_layout &L = T->layout;
-            if (L.slots > ((int64_t)1 << 31) && L.kind >= SJQ_TABLE_HASH_I32) return SJQ_ERR_UNSUPPORTED;
+            if (L.slots > ((int64_t)1 << 31) && is_hash_kind(L.kind)) return SJQ_ERR_UNSUPPORTED;
             S.op = (uint8_t)(L.kind == SJQ_TABLE_DIRECT_BITMAP ? OP_DIRECT_BITMAP
                              : L.kind == SJQ_TABLE_DIRECT_U8   ? OP_DIRECT_U8
                              : L.kind == SJQ_TABLE_DIRECT_U16  ? OP_DIRECT_U16
                              : L.kind == SJQ_TABLE_DIRECT_U32  ? OP_DIRECT_U32
                              : L.kind == SJQ_TABLE_DIRECT_U64  ? OP_DIRECT_U64
+                             : L.kind == SJQ_TABLE_DIRECT_U4   ? OP_DIRECT_U4
+                             : L.kind == SJQ_TABLE_DIRECT_U2   ? OP_DIRECT_U2
                              : L.kind == SJQ_TABLE_HASH_I32    ? OP_HASH32
                                                                : OP_HASH64);
             S.tab = T->slots;
             S.codes = nullptr;
             S.kmin = L.kmin;
             S.last = (uint64_t)L.slots - 1;
-            if (L.kind >= SJQ_TABLE_HASH_I32) {
+            S.full = (uint8_t)(L.code_bits > 0 && L.code_bits < 8 && L.entries == L.slots);
+            if (is_hash_kind(L.kind)) {
                 S.last = (uint64_t)(T->slots_bytes / kBucketBytes); // bucket count
                 if (sp.prefilter == 1) {
                     S.op = OP_HASHBITS;
@@ -414,7 +430,12 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     // Up to kMaxQueues - 1 later filter stages run as queue-fed levels; the rest at the final level.
     // Eager loading and compaction = never use no queue at all.
     int nd0 = 0, nfq = 0;
-    const bool direct = opts.eager_loads || opts.compaction == 1 || nfilter == 0;
+    // Most rows surviving every filter (by the measured fractions): each column is read for nearly every
+    // 32-byte sector anyway, so queues would only add shared-memory traffic and turn 128-bit loads into 4-byte
+    // ones.  A kernel compiled for the query then keeps thread-owned rows throughout and requests its columns
+    // up front.
+    const bool mostly_survive = opts.specialise && opts.compaction == 0 && reach[nfilter] >= kDirectSurvival;
+    const bool direct = opts.eager_loads || opts.compaction == 1 || nfilter == 0 || opts.unfused || mostly_survive;
     if (!direct) {
         nd0 = 1;
         if (opts.compaction != 2) {
@@ -490,7 +511,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     if (!opts.no_filter_bitmap) {
         for (int s = 0; s < ndense; ++s) {
             DStage &S = P.st[s];
-            if (S.kind != ST_PROBE || S.op < OP_DIRECT_U8 || S.op > OP_DIRECT_U64) continue;
+            if (S.kind != ST_PROBE || !is_code_op(S.op)) continue;
             const sjq_table *T = joins[specs[order[s]].index].table;
             if (!T->filter || T->layout.filter_bits <= 0) continue;
             S.op = OP_DIRECT_BITMAP;
@@ -525,12 +546,16 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     // Load schedule of the final level (used by kernels compiled for the query): a column is requested
     // once the last stage before it that is expected to drop rows has produced its mask, and at most
     // three columns ahead of the stage being processed.
-    if (P.nq) {
-        const int first = ndense;
+    // Without queues a thread keeps its four consecutive rows and loads them with one 128-bit load, which is
+    // skipped only when all four are dead: waiting for a mask pays only behind a stage that keeps less than
+    // about one row in six; everything else is requested up front, four columns deep.
+    {
+        const int first = ndense, depth = P.nq ? 3 : 4;
+        const double drop_below = P.nq ? 0.9 : 0.16;
         int last_barrier = first - 1;
         for (int t = first; t < ns; ++t) {
-            P.st[t].issue_after = (int8_t)std::max(std::max(last_barrier, t - 3), first - 1);
-            const bool drops = t < nfilter && specs[order[t]].sel < 0.9;
+            P.st[t].issue_after = (int8_t)std::max(std::max(last_barrier, t - depth), first - 1);
+            const bool drops = t < nfilter && specs[order[t]].sel < drop_below;
             if (drops) last_barrier = t;
         }
     }
@@ -562,7 +587,9 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         const size_t gb = (size_t)table_groups * 8 * (P.want_count ? 2 : 1);
         const bool fits = gb <= (size_t)64 << 10;
         bool contended = survivors / approx_grid >= 8.0 * (double)table_groups;
-        if (opts.agg_path == 1) {
+        if (opts.unfused) {
+            aggp = AGG_GLOBAL;
+        } else if (opts.agg_path == 1) {
             if (!fits) return SJQ_ERR_UNSUPPORTED;
             aggp = AGG_SMEM;
         } else if (opts.agg_path == 2) {
@@ -608,10 +635,10 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         if (fixed > smem_cap) return false;
         const size_t table_budget = smem_cap - fixed;
         size_t tables = 0;
-        if (opts.smem_tables != 1) {
+        if (opts.smem_tables != 1 && !opts.unfused) {
             std::vector<int> cand;
             for (int s = 0; s < nfilter; ++s)
-                if (P.st[s].op >= OP_DIRECT_BITMAP && P.st[s].op <= OP_DIRECT_U64) cand.push_back(s);
+                if (is_direct_op(P.st[s].op)) cand.push_back(s);
             std::stable_sort(cand.begin(), cand.end(), [&](int a, int b) {
                 return reach[a] / (double)P.st[a].tab_bytes > reach[b] / (double)P.st[b].tab_bytes;
             });
@@ -668,7 +695,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
 
     // ------------------------------------------------------------ launch shape
     int per_sm = 0;
-    const bool jit = opts.specialise != 0;
+    const bool jit = opts.specialise != 0 && !opts.unfused;
     // register budget a specialised kernel is compiled for
     // (three blocks of 384 threads when their shared memory leaves the L1 alone: 56 registers are enough for the
     // short pipelines that have so little state, and 36 warps hide more latency than 24)
@@ -705,7 +732,12 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     if ((opts.event_before != nullptr) != (opts.event_after != nullptr)) return SJQ_ERR_INVALID_ARG;
     if (opts.event_before && cudaEventRecord((cudaEvent_t)opts.event_before, stream) != cudaSuccess)
         return SJQ_ERR_CUDA;
-    if (n > 0) {
+    if (n > 0 && opts.unfused) {
+        if (!aligned16(opts.unfused_scratch)) return SJQ_ERR_ALIGN;
+        st = unfused_launch(P, nfilter, aggp, mul, has_hash, opts.unfused_scratch, opts.unfused_scratch_bytes,
+                            dev.sm_count, stream, &launches);
+        if (st != SJQ_OK) return st;
+    } else if (n > 0) {
         st = jit ? jit_launch(P, aggp, mul, has_hash, grid, block, lb_blocks, smem, stream)
                  : fused_launch(aggp, mul, has_hash, grid, block, smem, P, stream);
         if (st != SJQ_OK) return st;

@@ -24,8 +24,15 @@ enum : uint8_t {
     OP_DIRECT_U64 = 7,
     OP_HASH32 = 8,
     OP_HASH64 = 9,
-    OP_HASHBITS = 10 // presence bitmap in front of an open-addressing table, indexed by a hash of the key
+    OP_HASHBITS = 10, // presence bitmap in front of an open-addressing table, indexed by a hash of the key
+    OP_DIRECT_U4 = 11, // sub-byte codes, eight / sixteen to a 32-bit word
+    OP_DIRECT_U2 = 12
 };
+__host__ __device__ constexpr bool is_code_op(int op)
+{
+    return (op >= OP_DIRECT_U8 && op <= OP_DIRECT_U64) || op == OP_DIRECT_U4 || op == OP_DIRECT_U2;
+}
+__host__ __device__ constexpr bool is_direct_op(int op) { return op == OP_DIRECT_BITMAP || is_code_op(op); }
 
 // which accumulators a stage's values feed: bit = 3 * source + destination,
 // source 0 = the fact value itself, 1 = payload 0, 2 = payload 1;
@@ -77,7 +84,8 @@ struct DStage {
     uint8_t simple; // 1 + destination (0 key, 1 X, 2 Y): plain int32 load feeding one accumulator through mult32
     int8_t issue_after; // final level of a compiled kernel: the column is requested once this stage's mask is known
                         // (a stage before the level's first one = on entry)
-    uint8_t pad[2];
+    uint8_t full;   // sub-byte direct table holding every key of its range: a probe hits iff its key is in range
+    uint8_t pad[1];
 };
 static_assert(sizeof(DStage) % 8 == 0, "stage descriptors are copied as 64-bit words");
 

@@ -22,7 +22,8 @@ OPS = {"EQ": 0, "NE": 1, "LT": 2, "LE": 3, "GT": 4, "GE": 5, "BETWEEN": 6, "IN":
 AGGS = {"COL": 0, "MUL": 1, "SUB": 2, "ADD": 3}
 MODES = {"SCALAR": 0, "DENSE": 1, "HASHED": 2}
 TABLE_KINDS = {1: "DIRECT_BITMAP", 2: "DIRECT_U8", 3: "DIRECT_U16", 4: "DIRECT_U32", 5: "DIRECT_U64", 6: "HASH_I32",
-               7: "HASH_I64"}
+               7: "HASH_I64", 8: "DIRECT_U4", 9: "DIRECT_U2"}
+HASH_KINDS = (6, 7)
 FORCE_DIRECT, FORCE_HASH = 100, 101
 AGG_PATHS = {0: "registers", 1: "shared", 2: "global", 3: "hash"}
 
@@ -57,7 +58,7 @@ class _AggExpr(ctypes.Structure):
 
 class _BuildOpts(ctypes.Structure):
     _fields_ = [("force_kind", ctypes.c_int32), ("hash_load_pct", ctypes.c_int32),
-                ("max_direct_bytes", ctypes.c_int64)]
+                ("max_direct_bytes", ctypes.c_int64), ("min_code_bits", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 class DimLayout(ctypes.Structure):
@@ -94,7 +95,9 @@ class _RunOpts(ctypes.Structure):
                 ("event_after", ctypes.c_void_p), ("specialise", ctypes.c_int32),
                 ("rows_per_lane", ctypes.c_int32), ("no_filter_bitmap", ctypes.c_int32),
                 ("host_copy_all", ctypes.c_int32), ("dense_slots", ctypes.c_int32),
-                ("group_hash_always", ctypes.c_int32), ("pass_ppm", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS))]
+                ("group_hash_always", ctypes.c_int32), ("unfused", ctypes.c_int32),
+                ("unfused_scratch", ctypes.c_void_p), ("unfused_scratch_bytes", ctypes.c_size_t),
+                ("pass_ppm", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS))]
 
 
 class RunInfo(ctypes.Structure):
@@ -128,6 +131,7 @@ class RunOpts:
     host_copy_all: bool = False  # run_host: copy every referenced column instead of reading sparse ones in place
     dense_slots: int = 0  # level 0: 0 auto, 2, or 4 groups of four rows per thread (4 needs specialise)
     group_hash_always: bool = False  # HASHED: keep the group hash table even when the key domain is small
+    unfused_scratch: Optional[torch.Tensor] = None  # ablation: run operator at a time with this CUDA uint8 scratch
     pass_ppm: Sequence[int] = ()  # measured pass fractions (parts per million): predicates, then joins; 0 = unknown
 
     def to_c(self) -> _RunOpts:
@@ -140,6 +144,10 @@ class RunOpts:
             o.order[i] = v
         for i, v in enumerate(self.pass_ppm):
             o.pass_ppm[i] = int(v)
+        if self.unfused_scratch is not None:
+            o.unfused = 1
+            o.unfused_scratch = self.unfused_scratch.data_ptr()
+            o.unfused_scratch_bytes = self.unfused_scratch.numel()
         o.specialise = int(self.specialise)
         o.rows_per_lane = self.rows_per_lane
         o.no_filter_bitmap = int(self.no_filter_bitmap)
@@ -275,7 +283,7 @@ class Table:
 
 
 def build_dim(cols: dict, key: str, preds=(), payloads=(), force_kind: int = 0, hash_load_pct: int = 0,
-              max_direct_bytes: int = 0, edit_layout=None) -> Table:
+              max_direct_bytes: int = 0, edit_layout=None, min_code_bits: int = 0) -> Table:
     """sjq_dim_plan + sjq_build_dim over a dict of CUDA tensors (dimension columns).  `edit_layout`, if
     given, is called with the planned DimLayout and may change it before the build (sjq_build_dim takes
     the layout from its caller: tests use this to hand it an undersized or inconsistent one)."""
@@ -286,7 +294,7 @@ def build_dim(cols: dict, key: str, preds=(), payloads=(), force_kind: int = 0, 
         carr = _cols(tensors)
         parr, keep = _preds(preds, names)
         pay = (ctypes.c_int * max(1, len(payloads)))(*[names.index(p) for p in payloads])
-        opts = _BuildOpts(force_kind, hash_load_pct, max_direct_bytes)
+        opts = _BuildOpts(force_kind, hash_load_pct, max_direct_bytes, min_code_bits, 0)
         scratch = torch.empty(PLAN_SCRATCH_BYTES, dtype=torch.uint8, device=device)
         layout = DimLayout()
         stream = _stream_ptr(device)
@@ -314,7 +322,7 @@ class TableBuilder:
     dimensions can be planned with a single wait (sjq_dim_plan_begin / _end, sjq_build_dim)."""
 
     def __init__(self, cols: dict, key: str, preds=(), payloads=(), force_kind: int = 0, hash_load_pct: int = 0,
-                 max_direct_bytes: int = 0):
+                 max_direct_bytes: int = 0, min_code_bits: int = 0):
         self.names = list(cols.keys())
         self.tensors = [cols[n] for n in self.names]
         self.device = self.tensors[0].device
@@ -324,7 +332,7 @@ class TableBuilder:
             self.npreds, self.npay = len(preds), len(payloads)
             self.key_col = self.names.index(key)
             self.pay = (ctypes.c_int * max(1, len(payloads)))(*[self.names.index(p) for p in payloads])
-            self.opts = _BuildOpts(force_kind, hash_load_pct, max_direct_bytes)
+            self.opts = _BuildOpts(force_kind, hash_load_pct, max_direct_bytes, min_code_bits, 0)
             self.scratch = torch.empty(PLAN_SCRATCH_BYTES, dtype=torch.uint8, device=self.device)
             self.stats = torch.zeros(8, dtype=torch.int64, pin_memory=True)
             self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
@@ -393,6 +401,18 @@ def build_tables(builders: dict) -> dict:
     for b in builders.values():
         torch.cuda.current_stream(b.device).wait_stream(b.side)
     return tables
+
+
+def unfused_scratch(rows: int, njoins: int, device="cuda:0") -> torch.Tensor:
+    """Scratch for RunOpts.unfused_scratch (the operator-at-a-time ablation): sjq_unfused_scratch_bytes."""
+    n = ctypes.c_size_t(0)
+    L = lib()
+    L.sjq_unfused_scratch_bytes.restype = ctypes.c_int32
+    L.sjq_unfused_scratch_bytes.argtypes = [ctypes.c_int64, ctypes.c_int, ctypes.POINTER(ctypes.c_size_t)]
+    rc = L.sjq_unfused_scratch_bytes(rows, njoins, ctypes.byref(n))
+    if rc != 0:
+        raise SjqError(rc, "sjq_unfused_scratch_bytes")
+    return torch.empty(n.value, dtype=torch.uint8, device=device)
 
 
 def sample_preds(fact: dict, preds=()) -> tuple:
@@ -711,7 +731,7 @@ def jit_log() -> str:
 
 def build_launches(table: "Table") -> int:
     """Kernels enqueued by sjq_dim_plan + sjq_build_dim for this table (cudaMemset calls not counted)."""
-    direct = table.layout.kind <= 5
+    direct = table.layout.kind not in HASH_KINDS
     rows = table.layout.dim_rows > 0
     return 1 + (1 if rows else 0) + (1 if rows else 0) + (2 if direct else 1)
 

@@ -51,6 +51,7 @@ def test_random_queries_option_matrix(seed):
                  sjq.RunOpts(block_threads=128, ctas_per_sm=1), sjq.RunOpts(block_threads=256, compaction=2, smem_tables=1), sjq.RunOpts(agg_path=2),
                  sjq.RunOpts(compaction=2), sjq.RunOpts(compaction=1), sjq.RunOpts(no_filter_bitmap=True),
                  sjq.RunOpts(group_hash_always=True),
+                 sjq.RunOpts(unfused_scratch=sjq.unfused_scratch(w.n_rows, len(w.joins))),
                  sjq.RunOpts(order=tuple(reversed(range(len(w.preds) + len(w.joins)))))):
         res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)
         assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)
@@ -492,3 +493,24 @@ def test_any_pass_fraction_hint_gives_the_same_result(seed):
                                         check=False, dev_fact=dev_fact, tables=tables)
             assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)
             compare(w, res, exp)
+
+
+@pytest.mark.parametrize("mk", [lambda: W.config1(1_000_003), lambda: W.config2(2_000_003), lambda: W.config3(2_500_001),
+                                lambda: W.config4(1_000_003, 0.5, 1000), lambda: W.config4(1_000_003, 0.1, 100000),
+                                lambda: W.config5(1_200_005, 300000), lambda: W.city_brand(3_000_001)])
+def test_operator_at_a_time_ablation_matches_the_oracle(mk):
+    """The unfused arm of the ablation (one kernel per operator, flag array, materialised payload columns)
+    computes the same query: bit-exact against the oracle, and one launch per operator is reported."""
+    w = mk()
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    scratch = sjq.unfused_scratch(w.n_rows, len(w.joins))
+    res, exp, tables = run_both(w, fact, hd, opts=sjq.RunOpts(unfused_scratch=scratch))
+    assert res.status() == 0
+    compare(w, res, exp)
+    passes = len(w.preds) + sum(2 if (t.layout.kind >= 6 and t.layout.filter_bits) else 1 for t in tables.values())
+    assert res.info.kernel_launches == 1 + passes + 1 + (1 if w.mode == "HASHED" else 0)
+    # too little scratch is refused on the host
+    with pytest.raises(sjq.SjqError) as e:
+        sjq.run_workload(w, to_dev(fact), tables, sjq.RunOpts(unfused_scratch=scratch[: w.n_rows // 2]))
+    assert e.value.status == 5
