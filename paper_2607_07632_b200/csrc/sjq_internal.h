@@ -33,7 +33,10 @@ constexpr int32_t kEmptyKey32 = INT32_MIN;
 // touches decides its cost).  A key's linear probe starts at its home bucket (multiply-high range reduction
 // of its hash, so the bucket count need not be a power of two), a lookup loads whole buckets and stops at
 // the first one with a free slot; inserts fill a bucket's slots in order.
-constexpr int kBucketBytes = 64;
+#ifndef SJQ_BUCKET_BYTES
+#define SJQ_BUCKET_BYTES 64
+#endif
+constexpr int kBucketBytes = SJQ_BUCKET_BYTES;
 // keys per bucket for a key of kb bytes with a code of cb bytes (0, 4 or 8): the largest K with
 // K * kb rounded up to the code's alignment + K * cb <= 64
 __host__ __device__ constexpr int bucket_code_offset(int kb, int cb, int k)
@@ -46,8 +49,10 @@ __host__ __device__ constexpr int bucket_keys(int kb, int cb)
     while (k > 1 && bucket_code_offset(kb, cb, k) + k * cb > kBucketBytes) --k;
     return k;
 }
+#if SJQ_BUCKET_BYTES == 64
 static_assert(bucket_keys(8, 4) == 5 && bucket_keys(8, 8) == 4 && bucket_keys(8, 0) == 8, "64-bit keys");
 static_assert(bucket_keys(4, 4) == 8 && bucket_keys(4, 8) == 5 && bucket_keys(4, 0) == 16, "32-bit keys");
+#endif
 constexpr size_t kTableHeaderBytes = 256; // device-side counters at the start of table_mem
 
 } // namespace sjq

@@ -62,7 +62,6 @@ constexpr int kMaxQueues = 3;            // queue-fed levels per warp (the last 
 struct DStage {
     const void *col;   // fact column read by this stage
     const void *tab;   // direct: code array / bitmap words; hash: bucket array; presence bitmap: its words
-    const void *codes; // presence bitmap of a hash table: the bucket array to prefetch from (NULL = no prefetch)
     int64_t kmin;      // direct: slot index = key - kmin
     uint64_t last;     // direct: last valid slot index (slots - 1); hash (and its bitmap stage): bucket count
     int64_t lo, hi;    // 64-bit predicate range
@@ -115,6 +114,7 @@ struct RunParams {
     int32_t eager;   // load every column for every row
     int32_t has_key; // scalar path of a one-group dense result: key is computed and range-checked
     int32_t mod32;   // modulo fits in 32 bits
+    int32_t warp_agg; // group-by terminal: equal keys of a warp are added inside the warp before the atomics
     uint32_t smem_stages; // byte offset of the stage descriptors copied to shared memory
     uint32_t smem_groups; // byte offset of the shared group table
     uint32_t smem_queue;  // byte offset of the per-warp survivor queues

@@ -95,7 +95,7 @@ class _RunOpts(ctypes.Structure):
                 ("event_after", ctypes.c_void_p), ("specialise", ctypes.c_int32),
                 ("rows_per_lane", ctypes.c_int32), ("no_filter_bitmap", ctypes.c_int32),
                 ("host_copy_all", ctypes.c_int32), ("dense_slots", ctypes.c_int32),
-                ("group_hash_always", ctypes.c_int32), ("unfused", ctypes.c_int32),
+                ("group_hash_always", ctypes.c_int32), ("warp_agg", ctypes.c_int32), ("unfused", ctypes.c_int32),
                 ("unfused_scratch", ctypes.c_void_p), ("unfused_scratch_bytes", ctypes.c_size_t),
                 ("pass_ppm", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS))]
 
@@ -131,6 +131,7 @@ class RunOpts:
     host_copy_all: bool = False  # run_host: copy every referenced column instead of reading sparse ones in place
     dense_slots: int = 0  # level 0: 0 auto, 2, or 4 groups of four rows per thread (4 needs specialise)
     group_hash_always: bool = False  # HASHED: keep the group hash table even when the key domain is small
+    warp_agg: int = 0  # group-by terminal: 0 auto, 1 add equal keys inside the warp before the atomics, 2 never
     unfused_scratch: Optional[torch.Tensor] = None  # ablation: run operator at a time with this CUDA uint8 scratch
     pass_ppm: Sequence[int] = ()  # measured pass fractions (parts per million): predicates, then joins; 0 = unknown
 
@@ -144,6 +145,7 @@ class RunOpts:
             o.order[i] = v
         for i, v in enumerate(self.pass_ppm):
             o.pass_ppm[i] = int(v)
+        o.warp_agg = self.warp_agg
         if self.unfused_scratch is not None:
             o.unfused = 1
             o.unfused_scratch = self.unfused_scratch.data_ptr()

@@ -48,6 +48,8 @@ def test_random_queries_option_matrix_specialised(seed):
                  spec(block_threads=1024, ctas_per_sm=1), spec(block_threads=512, compaction=2, smem_tables=2),
                  spec(agg_path=2), spec(compaction=1), spec(rows_per_lane=8), spec(rows_per_lane=8, compaction=2),
                  spec(no_filter_bitmap=True), spec(group_hash_always=True), spec(dense_slots=4), spec(dense_slots=4, block_threads=768, ctas_per_sm=1),
+                 spec(warp_agg=1), spec(warp_agg=1, agg_path=2), spec(warp_agg=2, compaction=1),
+                 spec(pass_ppm=(900_000,) * (len(w.preds) + len(w.joins))),  # "most rows survive": the queue-free plan
                  spec(order=tuple(reversed(range(len(w.preds) + len(w.joins)))))):
         res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)
         assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)
@@ -81,9 +83,12 @@ def test_configs_multi_tile_specialised(mk):
     assert res.status() == 0
     compare(w, res, exp)
     dev_fact = to_dev(fact)
+    nf = len(w.preds) + len(w.joins)
     for opts in (spec(eager_loads=True, smem_tables=1, compaction=1),
                  spec(agg_path=2 if w.mode == "DENSE" else 0, block_threads=768, ctas_per_sm=1, compaction=2),
-                 spec(rows_per_lane=8, no_filter_bitmap=True, smem_tables=2), spec(dense_slots=4)):
+                 spec(rows_per_lane=8, no_filter_bitmap=True, smem_tables=2), spec(dense_slots=4),
+                 spec(warp_agg=1), spec(warp_agg=1, agg_path=1 if (w.mode == "DENSE" and 1 < w.num_groups <= 4096) else 0),
+                 spec(pass_ppm=(950_000,) * nf), spec(pass_ppm=(950_000,) * nf, warp_agg=1, block_threads=256)):
         res2, _, _ = run_both(w, fact, hd, opts=opts, dev_fact=dev_fact, tables=tables)
         compare(w, res2, exp)
 

@@ -50,7 +50,7 @@ def test_random_queries_option_matrix(seed):
     for opts in (sjq.RunOpts(), sjq.RunOpts(eager_loads=True), sjq.RunOpts(smem_tables=1),
                  sjq.RunOpts(block_threads=128, ctas_per_sm=1), sjq.RunOpts(block_threads=256, compaction=2, smem_tables=1), sjq.RunOpts(agg_path=2),
                  sjq.RunOpts(compaction=2), sjq.RunOpts(compaction=1), sjq.RunOpts(no_filter_bitmap=True),
-                 sjq.RunOpts(group_hash_always=True),
+                 sjq.RunOpts(group_hash_always=True), sjq.RunOpts(warp_agg=1), sjq.RunOpts(warp_agg=1, agg_path=2),
                  sjq.RunOpts(unfused_scratch=sjq.unfused_scratch(w.n_rows, len(w.joins))),
                  sjq.RunOpts(order=tuple(reversed(range(len(w.preds) + len(w.joins)))))):
         res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)
@@ -112,16 +112,26 @@ def test_table_kinds_and_sizes():
     w = W.config3(10)
     dims = {d.name: W.device_dim(w, d) for d in w.dims}
     tabs = sjq.build_workload_tables(w, dims)
-    L = tabs["customer"].layout
+    # with byte-or-wider codes, as in the paper: the 3 MB customer map
+    L = sjq.build_dim(dims["customer"], "custkey", w.dim("customer").preds, ("nation",), min_code_bits=8).layout
     # the key range is taken among the rows passing the filter
     assert L.kind_name == "DIRECT_U8" and 2_999_000 <= L.slots <= 3_000_000 and L.code_bits == 8
     # byte-packed codes plus the presence bitmap over the same slots (an eighth of a byte per slot)
     assert L.filter_bits >= L.slots and L.filter_bits % 128 == 0
     assert L.slots + L.slots // 8 <= L.table_bytes <= 3_000_000 + 375_000 + 1024
+    # by default the five nations of the region (codes 0..4, 0xF = filtered out) take four bits: half of that
+    L = tabs["customer"].layout
+    assert L.kind_name == "DIRECT_U4" and L.code_bits == 4 and L.pay_bits[0] == 3
+    assert L.slots // 2 + L.slots // 8 <= L.table_bytes <= 1_500_000 + 375_000 + 1024
     assert tabs["supplier"].layout.kind_name == "DIRECT_BITMAP" and 199_900 <= tabs["supplier"].layout.slots <= 200_000
     assert tabs["part"].layout.kind_name == "DIRECT_BITMAP"
-    d = tabs["date"].layout
-    assert d.kind_name == "DIRECT_U8" and d.entries == 729 and d.kmin == 19970101 and d.kmax == 19981230
+    d = tabs["date"].layout  # two years: one payload bit, the marker needs a second
+    assert d.kind_name == "DIRECT_U2" and d.entries == 729 and d.kmin == 19970101 and d.kmax == 19981230
+    # an unfiltered dimension with contiguous keys holds every key of its range: no marker, the range test decides
+    w4 = W.config4(10)
+    t4 = sjq.build_workload_tables(w4, {x.name: W.device_dim(w4, x) for x in w4.dims})["dim"]
+    assert t4.layout.kind_name == "DIRECT_U2" and t4.layout.entries == t4.layout.slots == 3_000_000
+    assert t4.layout.pay_max[0] - t4.layout.pay_min[0] == 3 and t4.check().status() == 0
     # forcing the unpacked form: open addressing at load <= 0.5
     t = sjq.build_dim(dims["customer"], "custkey", w.dim("customer").preds, ("nation",), force_kind=sjq.sjq.FORCE_HASH)
     assert t.layout.kind_name == "HASH_I32" and t.layout.slots >= 2 * t.layout.entries
@@ -171,6 +181,49 @@ def test_undersized_hash_table_reports_table_full(wide):
         t = sjq.build_dim(cols, "k", (Pred("p", "LT", 81),), pay, force_kind=sjq.sjq.FORCE_HASH, edit_layout=shrink)
         assert t.status() == 17
     assert sjq.build_dim(cols, "k", (), ("p",), force_kind=sjq.sjq.FORCE_HASH).status() == 0
+
+
+def test_sub_byte_tables_with_and_without_the_miss_marker():
+    """2- and 4-bit codes.  A dimension that holds every key of its range uses all code values and lets the
+    range test decide a hit; any other keeps all-ones as the miss marker.  Keys outside the range, keys
+    filtered out and duplicate keys behave as for the byte-wide maps, and a layout that promises "every key"
+    for data that lacks one is reported, not followed."""
+    import ctypes
+
+    rng = np.random.default_rng(7)
+    n = 4099
+    for width, hi in ((2, 3), (4, 15)):
+        keys = np.arange(100, 100 + 577, dtype=np.int32)
+        dim = {"k": keys, "w": rng.integers(0, hi + 1, keys.size).astype(np.int32), "f": (keys % 3).astype(np.int32)}
+        dim["w"][:hi + 1] = np.arange(hi + 1)  # every code value occurs, all-ones included
+        fact = {"fk": rng.integers(60, 720, n).astype(np.int32), "m": rng.integers(0, 1000, n).astype(np.int32)}
+        for preds, full in (([], True), ([Pred("f", "NE", 0)], False)):
+            w = adhoc("sub", fact, [("d", dim, "k", preds, ["w"])], [("fk", "d")], [],
+                      KeyExpr((Term("PAYLOAD", 0, 0),)), AggExpr("ADD", Term("FACT", "m"), Term("PAYLOAD", 0, 0, 7)),
+                      "DENSE", num_groups=hi + 1)
+            for opts in (None, sjq.RunOpts(specialise=True), sjq.RunOpts(compaction=1),
+                         sjq.RunOpts(specialise=True, pass_ppm=(990_000,)), sjq.RunOpts(smem_tables=1),
+                         sjq.RunOpts(no_filter_bitmap=True)):
+                res, exp, tabs = run_both(w, fact, {"d": dim}, opts=opts)
+                L = tabs["d"].layout
+                # without the marker the narrow width holds all values; with it the next width is needed
+                assert L.kind_name == (f"DIRECT_U{width}" if full else {2: "DIRECT_U4", 4: "DIRECT_U8"}[width])
+                assert (L.entries == L.slots) == full and res.status() == 0
+                compare(w, res, exp)
+    # duplicate key in a sub-byte table
+    cols = {"k": torch.tensor([5, 6, 7, 6], dtype=torch.int32, device="cuda"),
+            "p": torch.tensor([1, 2, 0, 1], dtype=torch.int32, device="cuda")}
+    assert sjq.build_dim(cols, "k", (), ("p",)).status() == 16
+    # a layout planned for the full dimension, used to build from data that lacks a key
+    full_cols = {"k": torch.arange(1, 101, dtype=torch.int32, device="cuda"),
+                 "p": torch.arange(0, 100, dtype=torch.int32, device="cuda") % 4}
+    planned = sjq.build_dim(full_cols, "k", (), ("p",))
+    assert planned.layout.kind_name == "DIRECT_U2" and planned.status() == 0
+
+    def stale(L):
+        ctypes.memmove(ctypes.byref(L), ctypes.byref(planned.layout), ctypes.sizeof(L))
+
+    assert sjq.build_dim(full_cols, "k", (Pred("k", "NE", 50),), ("p",), edit_layout=stale).status() == 21
 
 
 def test_reserved_key_and_empty_dimension():
