@@ -124,7 +124,7 @@ enum {
     SJQ_TABLE_DIRECT_U16 = 3,
     SJQ_TABLE_DIRECT_U32 = 4,
     SJQ_TABLE_DIRECT_U64 = 5,
-    SJQ_TABLE_HASH_I32 = 6, /* open addressing over 64-byte buckets of keys and codes, linear probing, int32 keys */
+    SJQ_TABLE_HASH_I32 = 6, /* open addressing over 32-byte buckets of keys and codes, linear probing, int32 keys */
     SJQ_TABLE_HASH_I64 = 7,
     SJQ_TABLE_DIRECT_U4 = 8, /* 4 bits per key, eight codes to a 32-bit word: 0xF = miss unless every key of the
                                 range is present (entries == slots), in which case the range test alone decides */
@@ -138,7 +138,7 @@ enum {
 
 typedef struct sjq_build_opts {
     int32_t force_kind;       /* SJQ_TABLE_AUTO, SJQ_TABLE_FORCE_DIRECT or SJQ_TABLE_FORCE_HASH */
-    int32_t hash_load_pct;    /* 0 = default 50: slots >= entries * 100 / pct, in whole 64-byte buckets; <= 90 */
+    int32_t hash_load_pct;    /* 0 = default 50: slots >= entries * 100 / pct, in whole 32-byte buckets; <= 90 */
     int64_t max_direct_bytes; /* 0 = default 64 MiB: larger direct tables fall back to hashing */
     int32_t min_code_bits;    /* narrowest packed code of a direct table: 0 = default 2 (sub-byte codes where the
                                  payload range allows: a probed structure a quarter the size of Section 3.3's byte
@@ -158,8 +158,8 @@ typedef struct sjq_dim_layout {
     int64_t pay_min[SJQ_MAX_PAYLOADS]; /* payload i is stored as (value - pay_min[i]) in pay_bits[i] bits */
     int64_t pay_max[SJQ_MAX_PAYLOADS];
     int32_t pay_bits[SJQ_MAX_PAYLOADS];
-    int64_t slots;      /* direct: kmax-kmin+1; hash: key slots = 64-byte buckets x keys per bucket (a bucket holds
-                           K keys then their K codes: K = 16, 8 or 5 for 32-bit keys and 8, 5 or 4 for 64-bit keys
+    int64_t slots;      /* direct: kmax-kmin+1; hash: key slots = 32-byte buckets x keys per bucket (a bucket holds
+                           K keys then their K codes: K = 8, 4 or 2 for 32-bit keys and 4, 2 or 2 for 64-bit keys
                            with no, 32-bit or 64-bit codes) */
     int64_t filter_bits; /* direct with payloads: bits of the presence bitmap over the slots (a multiple of 128);
                             hash: size (power of two, 0 = none) of the presence bitmap indexed by the key's hash,
@@ -171,7 +171,12 @@ typedef struct sjq_table sjq_table; /* opaque host handle */
 
 /*
  * Scan the filtered dimension once (key range, passing-row count, payload
- * ranges) and choose the table shape.  Enqueues one kernel on `stream`, copies
+ * ranges) and choose the table shape: Section 4.3.1 of the paper has the
+ * engine verify the key range at run time and pick the packed direct map or
+ * the unpacked table; Section 3.3 gives the forms.  The layout also carries
+ * the device bytes the table needs, so this call stands where a separate
+ * "how much memory" query would: the caller allocates `table_bytes` and hands
+ * them to sjq_build_dim.  Enqueues one kernel on `stream`, copies
  * 64 bytes back and SYNCHRONISES the stream before returning.
  *   cols/ncols      dimension columns (device), all of equal length
  *   preds/npreds    conjunction over those columns (npreds <= 16)
@@ -231,8 +236,12 @@ sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pred *preds, 
  */
 sjq_status sjq_dim_layout_bytes(const sjq_dim_layout *layout, size_t *bytes);
 
-/* Copy of the layout the table was built with. */
+/* Copy of the layout the table was built with: kind, key range, entries, slots and bytes, i.e. what decides
+ * whether the probed structure stays in L1 / L2 (Section 3.3: the packed map is sized to stay cache-resident). */
 sjq_status sjq_table_info(const sjq_table *table, sjq_dim_layout *layout);
+
+/* Kernels sjq_build_dim enqueued for this table (fills done with memsets are not kernels). */
+int32_t sjq_table_kernel_launches(const sjq_table *table);
 
 /* Frees the host handle only (the device memory belongs to the caller). */
 void sjq_table_destroy(sjq_table *table);
@@ -277,7 +286,8 @@ typedef struct sjq_result {
 
 /* Tuning and ablation switches; a zeroed struct (or NULL) means defaults. */
 typedef struct sjq_run_opts {
-    int32_t block_threads; /* 0 = default (512); else 128..512, multiple of 32 */
+    int32_t block_threads; /* 0 = library chooses (384; a kernel compiled for the query may run 1024); else a
+                              multiple of 32 in 128..384, or up to 1024 together with `specialise` */
     int32_t ctas_per_sm;   /* 0 = as many as fit */
     int32_t eager_loads;   /* 1 = load every column for every row (ablation of lazy loading) */
     int32_t agg_path;      /* 0 auto, 1 shared-memory privatised table, 2 global atomics (DENSE) */
@@ -369,11 +379,19 @@ sjq_status sjq_pred_sample_end(const int64_t *host_counts, int npreds, int32_t *
  * `rows` rows and `njoins` joins: one flag byte per row and one 8-byte cell per row and join. */
 sjq_status sjq_unfused_scratch_bytes(int64_t rows, int njoins, size_t *bytes);
 
-/* Device bytes needed at sjq_result.workspace for `spec` (0 unless HASHED). */
+/* Device bytes needed at sjq_result.workspace for `spec` (0 unless HASHED): room for the global group table
+ * of Section 3.3 ("the global table" kept for queries with very many groups), three int64 arrays of twice the
+ * capacity, rounded up to a power of two, plus one side slot. */
 sjq_status sjq_run_workspace_bytes(const sjq_result_spec *spec, size_t *bytes);
 
 /*
- * One fused pass over the fact table.
+ * One fused pass over the fact table: Section 4.2.2's operator vocabulary
+ * (a selection narrows the set of passing rows, a join probe drops the rows
+ * without a match, a gather pulls one dimension attribute into the row, the
+ * terminal consumes the survivors) run per row in one kernel, with Section
+ * 3.2's lazy loading (a later column is read only for rows that are still
+ * alive) and Section 3.3's terminals (register sum with one atomic per block,
+ * shared-memory privatised group table, global table).
  *   fact/nfact   fact columns (device), equal length N >= 0 (N need not be a
  *                multiple of anything)
  *   preds        conjunction over fact columns (npreds <= SJQ_MAX_PREDS)
@@ -506,10 +524,21 @@ const char *sjq_strerror(sjq_status status);
 const char *sjq_version(void);
 
 /*
+ * Give back what the library holds on behalf of the calling thread and the
+ * process: the two internal streams and three events sjq_run_host creates per
+ * device and thread on first use, the modules compiled at run time, and the
+ * remembered occupancy answers.  Nothing the library enqueued may still be
+ * running.  Later calls create what they need again.  Returns the number of
+ * objects released.  (Host-side bookkeeping only; the paper has no counterpart.)
+ */
+int32_t sjq_release(void);
+
+/*
  * Run-time specialisation (Section 4.2 of the paper fuses a query's operators before it runs; here the fused
  * kernel is compiled for the query's shape with NVRTC when sjq_run_opts.specialise is set).
- * Compiled modules are cached per process; when the environment variable SJQ_JIT_CACHE_DIR names a writable
- * directory they are also kept there as files, so that a later process loads instead of compiling.
+ * Compiled modules are cached per process, keyed by the query's shape.  The compiler needs the device sources:
+ * they are looked for in csrc/ beside the library and ../include (the environment variables SJQ_SOURCE_DIR and
+ * SJQ_INCLUDE_DIR name other places); SJQ_JIT_VERBOSE=1 prints the compiler's output to stderr.
  * sjq_jit_log copies the compiler output of the most recent compilation into `buf` (NUL-terminated, truncated
  * to `bytes`) and returns its full length.  sjq_jit_selftest compiles one of a few built-in query shapes
  * (shape_id 0 .. sjq_jit_selftest(-1, ...) - 1) without touching a device: SJQ_OK if the device code

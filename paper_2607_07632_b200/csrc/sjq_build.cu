@@ -113,7 +113,7 @@ struct BuildParams {
     int32_t code_bits;
     int64_t kmin;
     uint64_t span;  // direct
-    uint32_t buckets; // hash: number of 64-byte buckets
+    uint32_t buckets; // hash: number of buckets
     int32_t bucket_k; // hash: keys per bucket
     int32_t code_off; // hash: byte offset of the codes inside a bucket
     int64_t pay_min[SJQ_MAX_PAYLOADS], pay_max[SJQ_MAX_PAYLOADS];
@@ -664,9 +664,14 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
             fill_kernel<int64_t><<<g, 256, 0, stream>>>(reinterpret_cast<int64_t *>(T->slots), kEmptyKey64, bytes / 8);
         else
             fill_kernel<int32_t><<<g, 256, 0, stream>>>(reinterpret_cast<int32_t *>(T->slots), kEmptyKey32, bytes / 4);
+        ++T->launches;
     }
-    if (ok && B.dim.n > 0) build_kernel<<<grid_for(B.dim.n, dev.sm_count), 256, 0, stream>>>(B);
+    if (ok && B.dim.n > 0) {
+        build_kernel<<<grid_for(B.dim.n, dev.sm_count), 256, 0, stream>>>(B);
+        ++T->launches;
+    }
     if (ok && direct) {
+        T->launches += 2;
         direct_count_kernel<<<grid_for(L.slots, dev.sm_count), 256, 0, stream>>>(B);
         const bool promises_every_key = L.code_bits > 0 && L.code_bits < 8 && L.entries == L.slots;
         direct_verify_kernel<<<1, 32, 0, stream>>>(B.header, status_dev, promises_every_key ? (long long)L.entries : -1);
@@ -691,6 +696,11 @@ extern "C" sjq_status sjq_table_info(const sjq_table *table, sjq_dim_layout *lay
     if (!table || table->magic != kTableMagic || !layout) return SJQ_ERR_INVALID_ARG;
     *layout = table->layout;
     return SJQ_OK;
+}
+
+extern "C" int32_t sjq_table_kernel_launches(const sjq_table *table)
+{
+    return (table && table->magic == kTableMagic) ? table->launches : 0;
 }
 
 extern "C" void sjq_table_destroy(sjq_table *table)

@@ -35,7 +35,8 @@ __global__ void __launch_bounds__(256) clear_kernel(const ClearParams C)
 
 struct CompactParams {
     const int64_t *gkeys, *gsums, *gcounts;
-    int64_t dense_base; // >= 0: the table is indexed by key + dense_base and has no key array
+    int64_t dense_base; // indexed: cell number = key + dense_base
+    int32_t indexed;    // the table is indexed by the key itself and has no key array
     int64_t gslots; // regular slots; the side slot follows (direct-indexed: cells - 1)
     int64_t *keys, *sums, *counts;
     int64_t capacity;
@@ -48,7 +49,7 @@ __global__ void __launch_bounds__(256) compact_kernel(const CompactParams C)
 {
     const int64_t stride = (int64_t)blockDim.x * gridDim.x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i <= C.gslots; i += stride) {
-        const bool direct = C.dense_base >= 0;
+        const bool direct = C.indexed != 0;
         const bool side = !direct && i == C.gslots;
         const int64_t k = direct ? i - C.dense_base : side ? kEmptyKey64 : C.gkeys[i];
         const bool used = (direct || side) ? (C.gcounts[i] != 0) : (k != kEmptyKey64);
@@ -146,11 +147,25 @@ fused_fn pick_kernel(int agg, bool mul, bool hash)
 
 // Shared-memory opt-in and occupancy of a kernel variant; both answers are remembered per device, so a
 // repeated query costs two map look-ups instead of two runtime calls.
+namespace {
+std::mutex g_occ_mutex;
+std::unordered_map<uint64_t, int> g_occupancy; // (device, variant, block, smem) -> blocks per SM
+std::unordered_map<uint32_t, int> g_opted;     // (device, variant) -> largest smem opted in for
+} // namespace
+
+int fused_cache_clear()
+{
+    std::lock_guard<std::mutex> lock(g_occ_mutex);
+    const int n = (int)g_occupancy.size();
+    g_occupancy.clear(); // the shared-memory opt-in of a kernel is a property of the function: kept
+    return n;
+}
+
 sjq_status fused_occupancy(int agg, bool mul, bool hash, int block, size_t smem, int *ctas_per_sm)
 {
-    static std::mutex mutex;
-    static std::unordered_map<uint64_t, int> occupancy; // (device, variant, block, smem) -> blocks per SM
-    static std::unordered_map<uint32_t, int> opted;     // (device, variant) -> largest smem opted in for
+    std::mutex &mutex = g_occ_mutex;
+    std::unordered_map<uint64_t, int> &occupancy = g_occupancy;
+    std::unordered_map<uint32_t, int> &opted = g_opted;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return SJQ_ERR_CUDA;
     const uint32_t variant = (uint32_t)(agg * 4 + (mul ? 2 : 0) + (hash ? 1 : 0));
@@ -236,10 +251,11 @@ sjq_status merge_launch(const int64_t *keys, const int64_t *sums, const int64_t 
 }
 
 sjq_status compact_launch(const int64_t *gkeys, const int64_t *gsums, const int64_t *gcounts, int64_t gslots,
-                          int64_t dense_base, int64_t *keys, int64_t *sums, int64_t *counts, int64_t capacity,
-                          int64_t *n_groups, int32_t *status, int sm_count, cudaStream_t stream)
+                          bool indexed, int64_t dense_base, int64_t *keys, int64_t *sums, int64_t *counts,
+                          int64_t capacity, int64_t *n_groups, int32_t *status, int sm_count, cudaStream_t stream)
 {
-    CompactParams C{gkeys, gsums, gcounts, dense_base, gslots, keys, sums, counts, capacity, n_groups, status};
+    CompactParams C{gkeys, gsums, gcounts, dense_base, indexed ? 1 : 0, gslots, keys, sums, counts, capacity, n_groups,
+                    status};
     int64_t blocks = (gslots + 256) / 256;
     if (blocks > (int64_t)sm_count * 8) blocks = (int64_t)sm_count * 8;
     compact_kernel<<<(int)blocks, 256, 0, stream>>>(C);

@@ -17,7 +17,6 @@
 // run that asks for specialisation fails with SJQ_ERR_JIT; it never falls back
 // silently.
 #include <dlfcn.h>
-#include <unistd.h>
 
 #include <cstdio>
 #include <cstdlib>
@@ -46,7 +45,6 @@ struct Nvrtc {
     int (*GetProgramLogSize)(nvrtcProgram, size_t *);
     int (*GetProgramLog)(nvrtcProgram, char *);
     int (*DestroyProgram)(nvrtcProgram *);
-    int (*Version)(int *, int *) = nullptr;
     bool ok = false;
 };
 
@@ -74,7 +72,6 @@ Nvrtc &nvrtc()
         N.GetProgramLog = reinterpret_cast<decltype(N.GetProgramLog)>(sym("nvrtcGetProgramLog"));
         N.DestroyProgram = reinterpret_cast<decltype(N.DestroyProgram)>(sym("nvrtcDestroyProgram"));
         N.ok = all;
-        N.Version = reinterpret_cast<decltype(N.Version)>(dlsym(N.handle, "nvrtcVersion"));
     });
     return N;
 }
@@ -160,7 +157,6 @@ std::string jit_shape_header(const RunParams &P, int agg, bool mul, bool hash, i
       << "\n#define SJQ_JIT_has_key " << P.has_key << "\n#define SJQ_JIT_mod32 " << P.mod32
       << "\n#define SJQ_JIT_warp_agg " << P.warp_agg << "\n";
     put(o, "modulo", P.modulo);
-    put(o, "post_offset", P.post_offset);
     o << "#define SJQ_JIT_modmask " << P.modmask << "ULL\n";
     o << "namespace sjq {\nnamespace {\n"
          "__device__ __forceinline__ DStage jit_stage(const RunParams &P, int s)\n{\n"
@@ -198,7 +194,6 @@ std::string shape_key(const RunParams &P, int agg, bool mul, bool hash, int lb_t
                             P.rows, P.want_count, P.eager, P.has_key, P.mod32, (int32_t)P.qfold, P.slots, P.warp_agg};
     put_raw(head, sizeof(head));
     put_raw(&P.modulo, sizeof(P.modulo));
-    put_raw(&P.post_offset, sizeof(P.post_offset));
     put_raw(&P.modmask, sizeof(P.modmask));
     for (int s = 0; s < P.nstages; ++s) {
         const DStage &S = P.st[s];
@@ -227,32 +222,6 @@ std::mutex g_mutex;
 std::unordered_map<std::string, Module> g_modules;
 std::string g_last_log;
 
-// Optional cache of compiled modules on disk (SJQ_JIT_CACHE_DIR): a process that meets a shape some
-// earlier process compiled loads the cubin instead of compiling.  The file name is a hash of everything
-// the cubin depends on: the shape text, the device sources, the compiler's version and the options.
-uint64_t fnv1a(uint64_t h, const std::string &s)
-{
-    for (unsigned char c : s) h = (h ^ c) * 0x100000001B3ULL;
-    return h;
-}
-
-std::string cache_path(const std::string &shape, const Sources &S, int nvrtc_major, int nvrtc_minor)
-{
-    const char *dir = std::getenv("SJQ_JIT_CACHE_DIR");
-    if (!dir || !*dir) return std::string();
-    uint64_t h = 0xCBF29CE484222325ULL;
-    h = fnv1a(h, shape);
-    h = fnv1a(h, S.device);
-    h = fnv1a(h, S.run);
-    h = fnv1a(h, S.internal);
-    h = fnv1a(h, S.api);
-    if (const char *e = std::getenv("SJQ_JIT_EXTRA")) h = fnv1a(h, e);
-    char name[96];
-    std::snprintf(name, sizeof(name), "/sjq_%016llx_nvrtc%d.%d_sm100a.cubin", (unsigned long long)h, nvrtc_major,
-                  nvrtc_minor);
-    return std::string(dir) + name;
-}
-
 sjq_status compile(const std::string &shape, std::vector<char> *cubin, std::string *log)
 {
     Nvrtc &N = nvrtc();
@@ -264,17 +233,6 @@ sjq_status compile(const std::string &shape, std::vector<char> *cubin, std::stri
     if (!S.ok) {
         *log = S.error;
         return SJQ_ERR_JIT;
-    }
-    int vmaj = 0, vmin = 0;
-    if (N.Version) N.Version(&vmaj, &vmin);
-    const std::string cached = cache_path(shape, S, vmaj, vmin);
-    if (!cached.empty()) {
-        std::string bytes;
-        if (read_file(cached, &bytes) && bytes.size() > 64) {
-            cubin->assign(bytes.begin(), bytes.end());
-            *log = "loaded from " + cached;
-            return SJQ_OK;
-        }
     }
     // what precedes the //@body line of the shape text must be seen before any other header
     const size_t cut = shape.find("//@body\n");
@@ -315,15 +273,6 @@ sjq_status compile(const std::string &shape, std::vector<char> *cubin, std::stri
     } else {
         cubin->resize(cs);
         if (N.GetCUBIN(prog, cubin->data()) != 0) st = SJQ_ERR_JIT;
-        if (st == SJQ_OK && !cached.empty()) { // write beside, then rename: readers never see a partial file
-            const std::string tmp = cached + ".tmp" + std::to_string((long long)getpid());
-            std::ofstream f(tmp, std::ios::binary);
-            if (f && f.write(cubin->data(), (std::streamsize)cubin->size()) && (f.close(), true)) {
-                if (std::rename(tmp.c_str(), cached.c_str()) != 0) std::remove(tmp.c_str());
-            } else {
-                std::remove(tmp.c_str());
-            }
-        }
     }
     N.DestroyProgram(&prog);
     return st;

@@ -33,8 +33,8 @@ sjq_status fused_launch(int agg, bool mul, bool hash, int grid, int block, size_
 sjq_status clear_launch(int64_t *sums, int64_t *counts, int64_t cells, int64_t *gkeys, int64_t gslots,
                         int64_t *n_groups, int32_t *status, int sm_count, cudaStream_t stream);
 sjq_status compact_launch(const int64_t *gkeys, const int64_t *gsums, const int64_t *gcounts, int64_t gslots,
-                          int64_t dense_base, int64_t *keys, int64_t *sums, int64_t *counts, int64_t capacity,
-                          int64_t *n_groups, int32_t *status, int sm_count, cudaStream_t stream);
+                          bool indexed, int64_t dense_base, int64_t *keys, int64_t *sums, int64_t *counts,
+                          int64_t capacity, int64_t *n_groups, int32_t *status, int sm_count, cudaStream_t stream);
 
 size_t unfused_scratch_bytes(int64_t n, int gathering_joins);
 sjq_status unfused_launch(const RunParams &P, int nfilter, int agg, bool mul, bool has_hash, void *scratch,
@@ -566,12 +566,39 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     // workspace arrays the group table is indexed directly by key + M - 1 (no key array, no hashing, no claim:
     // two atomics per row instead of a look-up and two atomics; every dense aggregation path applies) and the
     // compaction recovers the keys from the cell numbers (config 4, G = 10^6 at 10 %: 3.2 -> 1.6 ms).
+    // The same holds for a key without a modulo whose every term is a gathered payload: the tables know the
+    // range of each payload among the rows they hold, so the key's range is known before the run (the
+    // paper's city x city and city x brand keys, Section 3.3, are of this kind).  Whenever the range fits, the
+    // indexed table is chosen: its clear and its compaction touch no more cells than the hash table's (whose
+    // size follows the capacity, not the survivors), and a row costs less.
     const uint64_t gslots_all = spec->mode == SJQ_HASHED ? hashed_slots(spec->capacity) : 0;
-    const bool direct_groups = spec->mode == SJQ_HASHED && key && key->modulo > 0 && !opts.group_hash_always &&
-                               (uint64_t)key->modulo <= (gslots_all + 1) / 2;
-    const int64_t table_groups = direct_groups ? 2 * key->modulo - 1 : spec->num_groups;
+    bool key_bounded = spec->mode == SJQ_HASHED && key != nullptr;
+    __int128 key_lo = key ? key->offset : 0, key_hi = key_lo;
+    for (int t = 0; key_bounded && t < key->nterms; ++t) {
+        const sjq_term &T = key->t[t];
+        if (T.src != SJQ_SRC_PAYLOAD) {
+            key_bounded = false;
+            break;
+        }
+        const sjq_dim_layout &L = joins[T.a].table->layout;
+        const __int128 a = (__int128)T.mult * L.pay_min[T.b], b = (__int128)T.mult * L.pay_max[T.b];
+        key_lo += a < b ? a : b;
+        key_hi += a < b ? b : a;
+    }
+    if (key && key->modulo > 0) {
+        // C remainder: the sign follows the dividend, the magnitude stays below the modulus
+        const __int128 m1 = (__int128)key->modulo - 1;
+        const bool nonneg = key_bounded && key_lo >= 0, nonpos = key_bounded && key_hi <= 0;
+        key_lo = nonneg ? 0 : -m1;
+        key_hi = nonpos ? 0 : m1;
+        key_bounded = spec->mode == SJQ_HASHED;
+    }
+    const __int128 key_cells = key_hi - key_lo + 1;
+    const bool direct_groups = key_bounded && !opts.group_hash_always && key_cells >= 1 &&
+                               key_cells <= (__int128)gslots_all + 1 && key_lo > INT64_MIN && key_hi < INT64_MAX;
+    const int64_t table_groups = direct_groups ? (int64_t)key_cells : spec->num_groups;
     if (direct_groups) {
-        P.post_offset = key->modulo - 1;
+        P.post_offset = (int64_t)-key_lo;
         P.want_count = 1; // the counts tell which cells hold a group
     }
     // ------------------------------------------------------------ aggregation path
@@ -754,7 +781,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         return SJQ_ERR_CUDA;
     if (spec->mode == SJQ_HASHED) {
         st = compact_launch(gkeys, gsums, gcounts, direct_groups ? table_groups - 1 : (int64_t)gslots,
-                            direct_groups ? P.post_offset : -1, out->keys, out->sums, out->counts, spec->capacity,
+                            direct_groups, P.post_offset, out->keys, out->sums, out->counts, spec->capacity,
                             out->n_groups, out->status, dev.sm_count, stream);
         if (st != SJQ_OK) return st;
         ++launches;
@@ -812,7 +839,7 @@ extern "C" sjq_status sjq_merge_groups(const int64_t *keys, const int64_t *sums,
     if ((st = merge_launch(keys, sums, counts, n, gkeys, gsums, gcounts, gslots - 1, out->status, dev.sm_count,
                            stream)) != SJQ_OK)
         return st;
-    return compact_launch(gkeys, gsums, gcounts, (int64_t)gslots, -1, out->keys, out->sums, out->counts, capacity,
+    return compact_launch(gkeys, gsums, gcounts, (int64_t)gslots, false, 0, out->keys, out->sums, out->counts, capacity,
                           out->n_groups, out->status, dev.sm_count, stream);
 }
 
@@ -826,9 +853,11 @@ struct HostPipe {
     bool ok = false;
 };
 
+thread_local HostPipe g_pipes[64];
+
 HostPipe *host_pipe()
 {
-    static thread_local HostPipe pipes[64];
+    HostPipe *pipes = g_pipes;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
     HostPipe &p = pipes[dev];
@@ -1047,6 +1076,33 @@ extern "C" sjq_status sjq_run_host(const sjq_col *fact_host, int nfact, const sj
     return ok ? SJQ_OK : SJQ_ERR_CUDA;
 }
 
+
+namespace sjq {
+int fused_cache_clear();
+}
+
+extern "C" int32_t sjq_release(void)
+{
+    int32_t released = 0;
+    int current = 0;
+    const bool have_device = cudaGetDevice(&current) == cudaSuccess;
+    for (int d = 0; d < 64; ++d) {
+        HostPipe &p = g_pipes[d];
+        if (!p.ok) continue;
+        if (have_device && cudaSetDevice(d) == cudaSuccess) {
+            for (cudaStream_t &st : p.s)
+                if (st && cudaStreamDestroy(st) == cudaSuccess) ++released;
+            for (cudaEvent_t ev : {p.start, p.done[0], p.done[1]})
+                if (ev && cudaEventDestroy(ev) == cudaSuccess) ++released;
+        }
+        p = HostPipe();
+    }
+    if (have_device) (void)cudaSetDevice(current);
+    (void)cudaGetLastError();
+    released += sjq_jit_cache_clear();
+    released += sjq::fused_cache_clear();
+    return released;
+}
 
 // ---------------------------------------------------------------------------
 // Hashed group-by with the group table in the library's own device image, for

@@ -732,10 +732,19 @@ def jit_log() -> str:
 
 
 def build_launches(table: "Table") -> int:
-    """Kernels enqueued by sjq_dim_plan + sjq_build_dim for this table (cudaMemset calls not counted)."""
-    direct = table.layout.kind not in HASH_KINDS
-    rows = table.layout.dim_rows > 0
-    return 1 + (1 if rows else 0) + (1 if rows else 0) + (2 if direct else 1)
+    """Kernels enqueued by sjq_dim_plan + sjq_build_dim for this table (cudaMemset calls not counted): the
+    plan's two (counter initialisation, and the scan unless the dimension is empty) and what the build reports."""
+    L = lib()
+    L.sjq_table_kernel_launches.restype = ctypes.c_int32
+    L.sjq_table_kernel_launches.argtypes = [ctypes.c_void_p]
+    return 1 + (1 if table.layout.dim_rows > 0 else 0) + int(L.sjq_table_kernel_launches(table.handle))
+
+
+def release() -> int:
+    """sjq_release: drop the library's per-thread streams and events, compiled modules and cached answers."""
+    L = lib()
+    L.sjq_release.restype = ctypes.c_int32
+    return int(L.sjq_release())
 
 
 def build_workload_tables(w, dims: dict) -> dict:

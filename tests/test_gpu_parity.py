@@ -395,6 +395,33 @@ def test_city_pair_shape_many_groups_few_survivors():
     compare(wh, res, exp)
 
 
+def test_city_brand_shape_and_the_library_chosen_group_table():
+    """The paper's city x brand shape (Section 3.3): year, supplier city and part brand as group key, 1.75 M
+    possible groups, about one row in eleven thousand survives.  Asked for as a hashed list, the library picks
+    the form of its group table: every term of the key is a gathered payload, so the tables' payload ranges
+    bound the key (260,000 cells here); with room for that many cells the table is indexed by the key itself,
+    otherwise it is the hash table.  As a dense array of all possible groups it takes global atomics.  All
+    three give the oracle's groups bit for bit, with both kernels."""
+    w = W.city_brand(6_000_011)
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    dev_fact = to_dev(fact)
+    tables = None
+    for variant, want in ((w, "hash"), (replace(w, capacity=200_000), "global"),
+                          (W.city_brand(w.n_rows, hashed=False), "global")):
+        for specialise in (False, True):
+            res, exp, tables = run_both(variant, fact, hd, opts=sjq.RunOpts(specialise=specialise), dev_fact=dev_fact,
+                                        tables=tables)
+            assert res.status() == 0 and res.info.describe()["agg_path"] == want
+            compare(variant, res, exp)
+    assert 300 < exp["counts"].sum() < 900 and tables["supplier"].layout.pay_min[0] == 70
+    # the caller can still insist on the hash table
+    res, exp, _ = run_both(replace(w, capacity=200_000), fact, hd, opts=sjq.RunOpts(group_hash_always=True),
+                           dev_fact=dev_fact, tables=tables)
+    assert res.info.describe()["agg_path"] == "hash"
+    compare(w, res, exp)
+
+
 def test_host_path_reads_sparse_columns_in_place_and_matches_copies():
     """sjq_run_host leaves a column that few rows reach in page-locked host memory and lets the kernel read
     it there; copying everything (host_copy_all), pageable buffers (always copied) and the device-resident
@@ -561,7 +588,7 @@ def test_operator_at_a_time_ablation_matches_the_oracle(mk):
     res, exp, tables = run_both(w, fact, hd, opts=sjq.RunOpts(unfused_scratch=scratch))
     assert res.status() == 0
     compare(w, res, exp)
-    passes = len(w.preds) + sum(2 if (t.layout.kind >= 6 and t.layout.filter_bits) else 1 for t in tables.values())
+    passes = len(w.preds) + sum(2 if (t.layout.kind in (6, 7) and t.layout.filter_bits) else 1 for t in tables.values())
     assert res.info.kernel_launches == 1 + passes + 1 + (1 if w.mode == "HASHED" else 0)
     # too little scratch is refused on the host
     with pytest.raises(sjq.SjqError) as e:

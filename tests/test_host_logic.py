@@ -82,20 +82,11 @@ def test_device_source_compiles_for_builtin_query_shapes(libsjq):
     assert libsjq.sjq_jit_selftest(n, None, 0) == 1  # no such shape: invalid argument
 
 
-def test_compiled_modules_can_be_cached_on_disk(libsjq, tmp_path, monkeypatch):
-    """With SJQ_JIT_CACHE_DIR set a compilation leaves a cubin file behind and the next one loads it."""
-    monkeypatch.setenv("SJQ_JIT_CACHE_DIR", str(tmp_path))
-    libsjq.sjq_jit_selftest.restype = ctypes.c_int32
-    libsjq.sjq_jit_selftest.argtypes = [ctypes.c_int32, ctypes.c_char_p, ctypes.c_size_t]
-    log = ctypes.create_string_buffer(1 << 16)
-    assert libsjq.sjq_jit_selftest(0, log, len(log)) == 0
-    files = [f for f in os.listdir(tmp_path) if f.endswith(".cubin")]
-    assert len(files) == 1 and os.path.getsize(os.path.join(tmp_path, files[0])) > 1000
-    assert b"loaded from" not in log.value
-    assert libsjq.sjq_jit_selftest(0, log, len(log)) == 0
-    assert b"loaded from" in log.value
-    assert libsjq.sjq_jit_selftest(1, log, len(log)) == 0  # another shape: another file
-    assert len([f for f in os.listdir(tmp_path) if f.endswith(".cubin")]) == 2
+def test_release_without_a_device_is_harmless(libsjq):
+    libsjq.sjq_release.restype = ctypes.c_int32
+    assert libsjq.sjq_release() >= 0
+    assert libsjq.sjq_release() == 0  # nothing left to give back
+    assert libsjq.sjq_table_kernel_launches(None) == 0
 
 
 def test_build_rejects_inconsistent_layouts_on_the_host(libsjq):
@@ -146,7 +137,7 @@ def test_build_rejects_inconsistent_layouts_on_the_host(libsjq):
         L.dim_rows = n + 1  # planned for another dimension
         assert build(L) == 1
     L = hashed()
-    L.slots = 2044  # an open-addressing table is made of whole buckets
+    L.slots = 2046  # an open-addressing table is made of whole buckets
     with pytest.raises(b.SjqError):
         b.layout_bytes(L)
     L.table_bytes = hashed().table_bytes

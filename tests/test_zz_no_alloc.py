@@ -40,17 +40,21 @@ def _calls():
 
     many = W.config4(700_003, 0.5, 30_000, hashed=True, dim_rows=40_000)
     few = W.config4(300_001, 0.1, 700, hashed=True, dim_rows=40_000)
-    # keys without a modulo can only live in the hash table: the foreign key itself (tens of thousands of
-    # groups), then the gathered payload (four groups)
+    # a key built from a fact column without a modulo has no known range and can only live in the hash table:
+    # the foreign key itself (tens of thousands of groups), then the filtered column (a thousand groups)
     many_plain = replace(many, name="static_fk_groups", key=KeyExpr((Term("FACT", "fk"),), offset=-7),
                          capacity=40_000)
-    few_plain = replace(few, name="static_payload_groups", key=KeyExpr((Term("PAYLOAD", 0, 0, 5),), offset=-3),
-                        capacity=16)
+    few_plain = replace(few, name="static_p_groups", key=KeyExpr((Term("FACT", "p", 0, 3),), offset=-3),
+                        capacity=1024)
+    # a key made of gathered payloads only has a range the tables know: the indexed form again, four cells
+    payload_key = replace(few, name="static_payload_groups", key=KeyExpr((Term("PAYLOAD", 0, 0, 5),), offset=-3),
+                          capacity=16)
     always = sjq.RunOpts(group_hash_always=True)
     return [(many, None, "indexed"), (few, None, "indexed"),  # the table indexed by the key
             (many, always, "hash"), (few, always, "hash"),  # the same queries through the hash table
             (many_plain, None, "hash"), (few_plain, None, "hash"),
-            (many, None, "indexed")]  # and back: the indexed form over the hash table's leftovers
+            (many, None, "indexed"),  # and back: the indexed form over the hash table's leftovers
+            (payload_key, None, "indexed")]
 
 
 def test_static_group_table_matches_oracle_and_workspace_entry_point_call_after_call():
