@@ -138,7 +138,7 @@ enum {
 
 typedef struct sjq_build_opts {
     int32_t force_kind;       /* SJQ_TABLE_AUTO, SJQ_TABLE_FORCE_DIRECT or SJQ_TABLE_FORCE_HASH */
-    int32_t hash_load_pct;    /* 0 = default 50: slots >= entries * 100 / pct, in whole 32-byte buckets; <= 90 */
+    int32_t hash_load_pct;    /* 0 = default 40: slots >= entries * 100 / pct, in whole 32-byte buckets; <= 90 */
     int64_t max_direct_bytes; /* 0 = default 64 MiB: larger direct tables fall back to hashing */
     int32_t min_code_bits;    /* narrowest packed code of a direct table: 0 = default 2 (sub-byte codes where the
                                  payload range allows: a probed structure a quarter the size of Section 3.3's byte

@@ -537,7 +537,8 @@ extern "C" sjq_status sjq_dim_plan_end(const sjq_col *cols, int ncols, int key_c
     if (force != SJQ_TABLE_AUTO && force != SJQ_TABLE_FORCE_DIRECT && force != SJQ_TABLE_FORCE_HASH)
         return SJQ_ERR_INVALID_ARG;
     const int64_t max_direct = (opts && opts->max_direct_bytes > 0) ? opts->max_direct_bytes : (int64_t)64 << 20;
-    const int load_pct = (opts && opts->hash_load_pct > 0) ? opts->hash_load_pct : 50;
+    // (the skewed 64-bit-key workload: 1.61 / 1.65 / 1.71 / 1.91 ms at load 33 / 40 / 50 / 60 %)
+    const int load_pct = (opts && opts->hash_load_pct > 0) ? opts->hash_load_pct : 40;
     if (load_pct > 90) return SJQ_ERR_INVALID_ARG;
 
     const uint64_t span_m1 = (uint64_t)L.kmax - (uint64_t)L.kmin; // span - 1, no overflow
