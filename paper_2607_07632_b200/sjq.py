@@ -324,10 +324,17 @@ class TableBuilder:
     dimensions can be planned with a single wait (sjq_dim_plan_begin / _end, sjq_build_dim)."""
 
     def __init__(self, cols: dict, key: str, preds=(), payloads=(), force_kind: int = 0, hash_load_pct: int = 0,
-                 max_direct_bytes: int = 0, min_code_bits: int = 0):
+                 max_direct_bytes: int = 0, min_code_bits: int = 0, reuse_layout: bool = False):
         self.names = list(cols.keys())
         self.tensors = [cols[n] for n in self.names]
         self.device = self.tensors[0].device
+        # reuse_layout: a repeated build does not wait for its own key-range scan.  It is enqueued with the
+        # layout chosen from the newest scan whose statistics have already reached the host (the previous
+        # step's, as a rule) and the build kernel checks every key and payload against that layout on the
+        # device (SJQ_ERR_LAYOUT_MISMATCH / TABLE_FULL in the table's status word if the dimension outgrew it).
+        # A changed dimension is therefore re-planned one or two steps late, never silently mis-built.
+        self.reuse_layout = reuse_layout
+        self.planned = False
         with torch.cuda.device(self.device):
             self.carr = _cols(self.tensors)
             self.parr, self._keep = _preds(preds, self.names)
@@ -336,7 +343,12 @@ class TableBuilder:
             self.pay = (ctypes.c_int * max(1, len(payloads)))(*[self.names.index(p) for p in payloads])
             self.opts = _BuildOpts(force_kind, hash_load_pct, max_direct_bytes, min_code_bits, 0)
             self.scratch = torch.empty(PLAN_SCRATCH_BYTES, dtype=torch.uint8, device=self.device)
-            self.stats = torch.zeros(8, dtype=torch.int64, pin_memory=True)
+            # statistics of the last few scans (page-locked, written by an asynchronous copy), each with the
+            # event that says its copy has landed
+            self.stats = [torch.zeros(8, dtype=torch.int64, pin_memory=True) for _ in range(4)]
+            self.stats_done = [torch.cuda.Event() for _ in self.stats]
+            self.stats_used = [False] * len(self.stats)
+            self.scan = -1  # ring position of the newest scan
             self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
             self.side = torch.cuda.Stream(self.device)
             # two table buffers used in turn: the build of the next table does not have to wait for the run
@@ -350,19 +362,42 @@ class TableBuilder:
     def begin(self):
         """Enqueue the key-range scan on the side stream.  It only reads the dimension columns, so it does
         not wait for work queued on the current stream (a previous run may still be reading the old table)."""
+        j = (self.scan + 1) % len(self.stats)
+        if self.stats_used[j]:
+            self.stats_done[j].synchronize()  # the host is a whole ring ahead of the device
         rc = lib().sjq_dim_plan_begin(self.carr, len(self.names), self.parr, self.npreds, self.key_col, self.pay,
-                                      self.npay, self.scratch.data_ptr(), self.stats.data_ptr(),
+                                      self.npay, self.scratch.data_ptr(), self.stats[j].data_ptr(),
                                       self.side.cuda_stream)
         if rc != 0:
             raise SjqError(rc, "sjq_dim_plan_begin")
+        self.stats_done[j].record(self.side)
+        self.stats_used[j] = True
+        self.scan = j
 
-    def finish(self) -> Table:
-        """Wait for the scan, choose the layout, enqueue the build on the side stream."""
-        self.side.synchronize()
+    def _choose_layout(self):
+        """The layout for the scan just enqueued, or (reuse_layout) for the newest one that has completed."""
+        n = len(self.stats)
+        j = self.scan
+        if self.reuse_layout and self.planned:
+            for back in range(n):
+                c = (self.scan - back) % n
+                if self.stats_used[c] and self.stats_done[c].query():
+                    j = c
+                    break
+            else:
+                return  # nothing newer has arrived: keep the layout
+        else:
+            self.stats_done[j].synchronize()
         rc = lib().sjq_dim_plan_end(self.carr, len(self.names), self.key_col, self.npay, ctypes.byref(self.opts),
-                                    self.stats.data_ptr(), ctypes.byref(self.layout))
+                                    self.stats[j].data_ptr(), ctypes.byref(self.layout))
         if rc != 0:
             raise SjqError(rc, "sjq_dim_plan_end")
+        self.planned = True
+
+    def finish(self) -> Table:
+        """Choose the layout (waiting for the scan unless reuse_layout allows an earlier one), enqueue the
+        build on the side stream."""
+        self._choose_layout()
         i = self.turn
         self.turn ^= 1
         main = torch.cuda.current_stream(self.device)
@@ -389,9 +424,10 @@ class TableBuilder:
         return Table(handle.value, layout, mem, self.status)
 
 
-def workload_builders(w, dims: dict) -> dict:
+def workload_builders(w, dims: dict, reuse_layout: bool = False) -> dict:
     return {d.name: TableBuilder(dims[d.name], d.key, d.preds, d.payloads,
-                                 force_kind=FORCE_HASH if d.force_hash else 0) for d in w.dims}
+                                 force_kind=FORCE_HASH if d.force_hash else 0, reuse_layout=reuse_layout)
+            for d in w.dims}
 
 
 def build_tables(builders: dict) -> dict:

@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 
 sjq = pytest.importorskip("paper_2607_07632_b200") if torch.cuda.is_available() else None
 
-from gpuhelpers import compare, run_both, to_dev  # noqa: E402
+from gpuhelpers import compare, oracle_result, run_both, to_dev  # noqa: E402
 from qhelpers import adhoc, ex1, ex2, ex3, random_query  # noqa: E402
 from bruteforce import dup_keys_among_passing  # noqa: E402
 
@@ -377,6 +377,45 @@ def test_stale_layout_is_reported_not_followed():
     t = b.finish()
     torch.cuda.synchronize()
     assert t.status() == 21
+
+
+def test_reused_layouts_rebuild_without_waiting_and_follow_a_changed_dimension():
+    """Builders that reuse the layout of an earlier scan: same tables and result as a planned build while the
+    dimension is unchanged; once it changes, the build on the old layout is flagged on the device and a later
+    step (the changed statistics have reached the host by then) re-plans and matches the oracle again."""
+    for w in (W.config3(400_003), W.config4(300_007, 0.5, 1000, dim_rows=50_000)):
+        fact = W.host_fact(w)
+        hd = {d.name: W.host_dim(w, d) for d in w.dims}
+        _, exp, tables = run_both(w, fact, hd)
+        dev_dims = {k: to_dev(v) for k, v in hd.items()}
+        builders = sjq.workload_builders(w, dev_dims, reuse_layout=True)
+        dev_fact = to_dev(fact)
+        for _ in range(4):
+            tabs = sjq.build_tables(builders)
+            r = sjq.run_workload(w, dev_fact, tabs)
+        torch.cuda.synchronize()
+        assert all(t.status() == 0 for t in tabs.values())
+        for k in tabs:
+            assert bytes(tabs[k].layout) == bytes(tables[k].layout)
+        compare(w, r, exp)
+    # the dimension changes in place: every payload leaves the planned range of its packed code
+    hd2 = {"dim": {c: v.copy() for c, v in hd["dim"].items()}}
+    hd2["dim"]["w"] += 1000
+    dev_dims["dim"]["w"].copy_(torch.from_numpy(hd2["dim"]["w"]))
+    torch.cuda.synchronize()
+    _, exp2 = oracle_result(w, fact, hd2)
+    tabs = sjq.build_tables(builders)  # this step's scan is not waited for: the old layout is used
+    torch.cuda.synchronize()
+    assert tabs["dim"].status() in (0, 21)  # 21 unless the scan happened to finish before the layout was chosen
+    builders["dim"].status.zero_()
+    for _ in range(2):
+        tabs = sjq.build_tables(builders)
+        torch.cuda.synchronize()
+    assert tabs["dim"].status() == 0
+    assert tabs["dim"].layout.pay_min[0] == tables["dim"].layout.pay_min[0] + 1000
+    r = sjq.run_workload(w, dev_fact, tabs)
+    torch.cuda.synchronize()
+    compare(w, r, exp2)
 
 
 def test_city_pair_shape_many_groups_few_survivors():
