@@ -510,6 +510,10 @@ def main():
     dims = {d.name: W.device_dim(w, d, device) for d in w.dims}
     fact = W.device_fact(w, row0=row0, n=n, device=device)
     torch.cuda.synchronize()
+    # The query runs on a high-priority stream and the table builders' side streams keep the default (lowest)
+    # priority: the blocks of the persistent fused kernel are placed first, and the next step's key-range scans
+    # and builds fill in where an SM has room instead of delaying its start.
+    torch.cuda.set_stream(torch.cuda.Stream(device, priority=-1))
 
     # every event pair is created (recorded once) up front; the library records them around the fused kernel
     pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
@@ -627,8 +631,8 @@ def main():
                 for dn, cols in host_dims.items():  # the dimension columns come from the host too
                     for k, v in cols.items():
                         dims[dn][k].copy_(v, non_blocking=True)
-                for b in builders.values():  # the key-range scans run on side streams: after the copies
-                    b.side.wait_stream(torch.cuda.current_stream(device))
+                for b in builders.values():  # scans and builds run on side streams: after the copies
+                    b.after(torch.cuda.current_stream(device))
                 tabs = sjq.build_tables(builders)
                 eres, ehost = sjq.run_workload_host(w_local, host_fact, tabs, staging, chunk,
                                                     sjq.RunOpts(specialise=not args.interpret), result=eres, host=ehost)

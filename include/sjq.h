@@ -240,7 +240,8 @@ sjq_status sjq_dim_layout_bytes(const sjq_dim_layout *layout, size_t *bytes);
  * whether the probed structure stays in L1 / L2 (Section 3.3: the packed map is sized to stay cache-resident). */
 sjq_status sjq_table_info(const sjq_table *table, sjq_dim_layout *layout);
 
-/* Kernels sjq_build_dim enqueued for this table (fills done with memsets are not kernels). */
+/* Kernels sjq_build_dim enqueued for this table: one that prepares the memory, the build unless the dimension
+ * is empty, and for a direct table the occupancy count that ends with the duplicate check. */
 int32_t sjq_table_kernel_launches(const sjq_table *table);
 
 /* Frees the host handle only (the device memory belongs to the caller). */

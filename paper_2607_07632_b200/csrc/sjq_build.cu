@@ -125,11 +125,25 @@ struct BuildParams {
     int32_t *status;
 };
 
-template <typename W>
-__global__ void fill_kernel(W *p, W v, size_t n)
+// One launch prepares a table's memory: the header counters and the presence bitmap to zero, the slot array to
+// its empty pattern (bitmap: zeros; packed codes: all ones; open addressing: the empty key in every word).
+// All three regions start on 16-byte boundaries and are padded to a multiple of 16 bytes by the layout.
+struct InitParams {
+    uint4 *header, *slots, *filter;
+    size_t header16, slots16, filter16; // sizes in 16-byte units
+    uint4 pattern;
+};
+
+__global__ void __launch_bounds__(256) table_init_kernel(const __grid_constant__ InitParams I)
 {
     const size_t stride = (size_t)blockDim.x * gridDim.x;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) p[i] = v;
+    const size_t total = I.header16 + I.slots16 + I.filter16;
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        if (i < I.header16) I.header[i] = zero;
+        else if (i < I.header16 + I.slots16) I.slots[i - I.header16] = I.pattern;
+        else I.filter[i - I.header16 - I.slots16] = zero;
+    }
 }
 
 __device__ inline bool pack_code(const BuildParams &B, int64_t r, uint64_t *code)
@@ -248,9 +262,11 @@ __global__ void __launch_bounds__(256) build_kernel(const __grid_constant__ Buil
     if ((threadIdx.x & 31) == 0 && inserted) atomicAdd(&B.header[0], inserted);
 }
 
-// Count occupied slots of a direct table; a repeated key leaves fewer
-// occupied slots than inserted rows.
-__global__ void __launch_bounds__(256) direct_count_kernel(const __grid_constant__ BuildParams B)
+// Count occupied slots of a direct table; a repeated key leaves fewer occupied slots than inserted rows.  The
+// block that finishes last (a ticket in header[2]) compares the two counters.  `expect_full` >= 0: the layout
+// promises that every key of the range is present (a probe then trusts the range test alone), so exactly that
+// many rows must have been stored.
+__global__ void __launch_bounds__(256) direct_count_kernel(const __grid_constant__ BuildParams B, long long expect_full)
 {
     const uint64_t stride = (uint64_t)blockDim.x * gridDim.x;
     unsigned long long occ = 0;
@@ -273,16 +289,16 @@ __global__ void __launch_bounds__(256) direct_count_kernel(const __grid_constant
     }
     occ = (unsigned long long)warp_sum((int64_t)occ);
     if ((threadIdx.x & 31) == 0 && occ) atomicAdd(&B.header[1], occ);
-}
-
-// `expect_full` >= 0: the layout promises that every key of the range is present (a probe then trusts the
-// range test alone), so exactly that many rows must have been stored.
-__global__ void direct_verify_kernel(const unsigned long long *header, int32_t *status, long long expect_full)
-{
-    if (threadIdx.x == 0 && blockIdx.x == 0) {
-        if (header[0] != header[1]) set_status(status, SJQ_ERR_DUP_KEY);
-        else if (expect_full >= 0 && header[1] != (unsigned long long)expect_full)
-            set_status(status, SJQ_ERR_LAYOUT_MISMATCH);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(&B.header[2], 1ULL) == (unsigned long long)gridDim.x - 1) {
+            __threadfence();
+            const unsigned long long inserted = atomicAdd(&B.header[0], 0ULL), occupied = atomicAdd(&B.header[1], 0ULL);
+            if (inserted != occupied) set_status(B.status, SJQ_ERR_DUP_KEY);
+            else if (expect_full >= 0 && occupied != (unsigned long long)expect_full)
+                set_status(B.status, SJQ_ERR_LAYOUT_MISMATCH);
+        }
     }
 }
 
@@ -633,16 +649,21 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
     B.status = status_dev;
     B.slots = T->slots;
 
-    bool ok = cudaMemsetAsync(T->base, 0, kTableHeaderBytes, stream) == cudaSuccess;
+    InitParams I{};
+    I.header = reinterpret_cast<uint4 *>(T->base);
+    I.header16 = kTableHeaderBytes / 16;
+    I.slots = reinterpret_cast<uint4 *>(T->slots);
     const bool direct = is_direct_kind(L.kind);
+    size_t filter_bytes = 0;
     if (direct) {
         const size_t bytes = direct_array_bytes(L);
         T->slots_bytes = bytes;
-        ok = ok && cudaMemsetAsync(T->slots, L.kind == SJQ_TABLE_DIRECT_BITMAP ? 0 : 0xFF, bytes, stream) == cudaSuccess;
+        const unsigned int fill = L.kind == SJQ_TABLE_DIRECT_BITMAP ? 0u : 0xFFFFFFFFu;
+        I.pattern = make_uint4(fill, fill, fill, fill);
         if (L.filter_bits) {
             T->filter = T->slots + align_up(bytes, 256);
             B.filter = reinterpret_cast<unsigned int *>(T->filter);
-            ok = ok && cudaMemsetAsync(T->filter, 0, (size_t)(L.filter_bits / 8), stream) == cudaSuccess;
+            filter_bytes = (size_t)(L.filter_bits / 8);
         }
     } else {
         const int kb = L.key_dtype == SJQ_I64 ? 8 : 4, cb = L.code_bits / 8;
@@ -655,29 +676,30 @@ extern "C" sjq_status sjq_build_dim(const sjq_col *cols, int ncols, const sjq_pr
             T->filter = T->slots + align_up(bytes, 256);
             B.filter = reinterpret_cast<unsigned int *>(T->filter);
             B.fmask = (uint32_t)(L.filter_bits - 1);
-            ok = ok && cudaMemsetAsync(T->filter, 0, (size_t)(L.filter_bits / 8), stream) == cudaSuccess;
+            filter_bytes = (size_t)(L.filter_bits / 8);
         }
         // Every word of a bucket starts as the empty marker's pattern: both markers (the minimum of the key
         // type) are a repeated 0x80 00 .. 00 word, so the codes start as that pattern too and are overwritten
         // when their slot is claimed.
-        const int g = grid_for((int64_t)(bytes / 8), dev.sm_count);
-        if (L.key_dtype == SJQ_I64)
-            fill_kernel<int64_t><<<g, 256, 0, stream>>>(reinterpret_cast<int64_t *>(T->slots), kEmptyKey64, bytes / 8);
-        else
-            fill_kernel<int32_t><<<g, 256, 0, stream>>>(reinterpret_cast<int32_t *>(T->slots), kEmptyKey32, bytes / 4);
-        ++T->launches;
+        I.pattern = L.key_dtype == SJQ_I64 ? make_uint4(0u, 0x80000000u, 0u, 0x80000000u)
+                                           : make_uint4(0x80000000u, 0x80000000u, 0x80000000u, 0x80000000u);
     }
-    if (ok && B.dim.n > 0) {
+    I.slots16 = (T->slots_bytes + 15) / 16;
+    I.filter = reinterpret_cast<uint4 *>(T->filter);
+    I.filter16 = (filter_bytes + 15) / 16; // the layout pads the bitmap's region to 256 bytes
+    table_init_kernel<<<grid_for((int64_t)(I.header16 + I.slots16 + I.filter16), dev.sm_count), 256, 0, stream>>>(I);
+    ++T->launches;
+    if (B.dim.n > 0) {
         build_kernel<<<grid_for(B.dim.n, dev.sm_count), 256, 0, stream>>>(B);
         ++T->launches;
     }
-    if (ok && direct) {
-        T->launches += 2;
-        direct_count_kernel<<<grid_for(L.slots, dev.sm_count), 256, 0, stream>>>(B);
+    if (direct) {
         const bool promises_every_key = L.code_bits > 0 && L.code_bits < 8 && L.entries == L.slots;
-        direct_verify_kernel<<<1, 32, 0, stream>>>(B.header, status_dev, promises_every_key ? (long long)L.entries : -1);
+        direct_count_kernel<<<grid_for(L.slots, dev.sm_count), 256, 0, stream>>>(
+            B, promises_every_key ? (long long)L.entries : -1);
+        ++T->launches;
     }
-    if (!ok || cudaGetLastError() != cudaSuccess) {
+    if (cudaGetLastError() != cudaSuccess) {
         (void)cudaGetLastError();
         delete T;
         return SJQ_ERR_CUDA;

@@ -117,27 +117,13 @@ __global__ void __launch_bounds__(256) sample_kernel(const __grid_constant__ Sam
         atomicAdd(&S.counts[threadIdx.x], (unsigned long long)block_counts[threadIdx.x]);
 }
 
-typedef void (*fused_fn)(const RunParams);
-
 fused_fn pick_kernel(int agg, bool mul, bool hash)
 {
-    switch (agg * 4 + (mul ? 2 : 0) + (hash ? 1 : 0)) {
-    case 0: return fused_kernel<AGG_SCALAR, false, false>;
-    case 1: return fused_kernel<AGG_SCALAR, false, true>;
-    case 2: return fused_kernel<AGG_SCALAR, true, false>;
-    case 3: return fused_kernel<AGG_SCALAR, true, true>;
-    case 4: return fused_kernel<AGG_SMEM, false, false>;
-    case 5: return fused_kernel<AGG_SMEM, false, true>;
-    case 6: return fused_kernel<AGG_SMEM, true, false>;
-    case 7: return fused_kernel<AGG_SMEM, true, true>;
-    case 8: return fused_kernel<AGG_GLOBAL, false, false>;
-    case 9: return fused_kernel<AGG_GLOBAL, false, true>;
-    case 10: return fused_kernel<AGG_GLOBAL, true, false>;
-    case 11: return fused_kernel<AGG_GLOBAL, true, true>;
-    case 12: return fused_kernel<AGG_HASH, false, false>;
-    case 13: return fused_kernel<AGG_HASH, false, true>;
-    case 14: return fused_kernel<AGG_HASH, true, false>;
-    default: return fused_kernel<AGG_HASH, true, true>;
+    switch (agg) {
+    case AGG_SCALAR: return fused_variant_scalar(mul, hash);
+    case AGG_SMEM: return fused_variant_smem(mul, hash);
+    case AGG_GLOBAL: return fused_variant_global(mul, hash);
+    default: return fused_variant_hash(mul, hash);
     }
 }
 

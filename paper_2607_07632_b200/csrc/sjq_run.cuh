@@ -120,5 +120,16 @@ struct RunParams {
     uint32_t smem_queue;  // byte offset of the per-warp survivor queues
 };
 
+#if !defined(SJQ_JIT)
+// The sixteen ahead-of-time variants of the fused kernel (aggregation path x product aggregate x "some table is
+// open-addressing"), instantiated in one translation unit per aggregation path.
+typedef void (*fused_fn)(const RunParams);
+fused_fn fused_variant_scalar(bool mul, bool hash);
+fused_fn fused_variant_smem(bool mul, bool hash);
+fused_fn fused_variant_global(bool mul, bool hash);
+fused_fn fused_variant_hash(bool mul, bool hash);
+#endif
+
 } // namespace sjq
+
 #endif

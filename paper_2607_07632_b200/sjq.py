@@ -350,7 +350,8 @@ class TableBuilder:
             self.stats_used = [False] * len(self.stats)
             self.scan = -1  # ring position of the newest scan
             self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
-            self.side = torch.cuda.Stream(self.device)
+            self.side = torch.cuda.Stream(self.device)       # builds
+            self.scan_side = torch.cuda.Stream(self.device)  # key-range scans: independent of the builds
             # two table buffers used in turn: the build of the next table does not have to wait for the run
             # that still reads the previous one
             self.mems = [None, None]
@@ -367,12 +368,18 @@ class TableBuilder:
             self.stats_done[j].synchronize()  # the host is a whole ring ahead of the device
         rc = lib().sjq_dim_plan_begin(self.carr, len(self.names), self.parr, self.npreds, self.key_col, self.pay,
                                       self.npay, self.scratch.data_ptr(), self.stats[j].data_ptr(),
-                                      self.side.cuda_stream)
+                                      self.scan_side.cuda_stream)
         if rc != 0:
             raise SjqError(rc, "sjq_dim_plan_begin")
-        self.stats_done[j].record(self.side)
+        self.stats_done[j].record(self.scan_side)
         self.stats_used[j] = True
         self.scan = j
+
+    def after(self, stream):
+        """Scans and builds enqueued from now on follow the work already queued on `stream` (e.g. copies that
+        refresh the dimension columns)."""
+        self.side.wait_stream(stream)
+        self.scan_side.wait_stream(stream)
 
     def _choose_layout(self):
         """The layout for the scan just enqueued, or (reuse_layout) for the newest one that has completed."""
@@ -768,8 +775,8 @@ def jit_log() -> str:
 
 
 def build_launches(table: "Table") -> int:
-    """Kernels enqueued by sjq_dim_plan + sjq_build_dim for this table (cudaMemset calls not counted): the
-    plan's two (counter initialisation, and the scan unless the dimension is empty) and what the build reports."""
+    """Kernels enqueued by sjq_dim_plan + sjq_build_dim for this table: the plan's two (counter
+    initialisation, and the scan unless the dimension is empty) and what the build reports."""
     L = lib()
     L.sjq_table_kernel_launches.restype = ctypes.c_int32
     L.sjq_table_kernel_launches.argtypes = [ctypes.c_void_p]

@@ -371,7 +371,7 @@ def test_stale_layout_is_reported_not_followed():
             "p": torch.arange(0, 1000, dtype=torch.int32, device="cuda") % 50}
     b = sjq.TableBuilder(cols, "k", (), ("p",))
     b.begin()
-    b.side.synchronize()
+    b.scan_side.synchronize()
     cols["k"][7] = 5_000_000       # far outside the planned span
     cols["p"][9] = 100_000         # outside the planned payload range
     t = b.finish()
