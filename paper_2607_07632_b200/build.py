@@ -47,7 +47,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
     with ThreadPoolExecutor(max_workers=max(1, min(len(todo), os.cpu_count() or 1))) as pool:
         list(pool.map(compile_one, todo))
-    subprocess.check_call(["nvcc", "-shared", "-o", LIB, *[_object(s) for s in sources()]], cwd=HERE)
+    subprocess.check_call(["nvcc", "-shared", *NVCC_FLAGS[:2], "-o", LIB, *[_object(s) for s in sources()]], cwd=HERE)
     return LIB
 
 

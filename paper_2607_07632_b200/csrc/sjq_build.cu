@@ -61,6 +61,19 @@ __device__ inline int64_t warp_sum(int64_t v)
     return v;
 }
 
+// Sum over a block of at most 256 threads; the total is valid in thread 0.
+__device__ inline unsigned long long block_sum(unsigned long long v)
+{
+    __shared__ unsigned long long part[8];
+    v = (unsigned long long)warp_sum((int64_t)v);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = v;
+    __syncthreads();
+    unsigned long long t = 0;
+    if (threadIdx.x == 0)
+        for (int w = 0; w < (int)((blockDim.x + 31) >> 5); ++w) t += part[w];
+    return t;
+}
+
 // scratch: [0] kmin [1] kmax [2] count [3] p0min [4] p0max [5] p1min [6] p1max
 __global__ void plan_init_kernel(int64_t *s)
 {
@@ -96,13 +109,33 @@ __global__ void __launch_bounds__(256) plan_scan_kernel(const __grid_constant__ 
         pmin[i] = warp_min(pmin[i]);
         pmax[i] = warp_max(pmax[i]);
     }
-    if ((threadIdx.x & 31) == 0 && cnt > 0) {
-        atomicMin((long long *)&scratch[0], (long long)kmin);
-        atomicMax((long long *)&scratch[1], (long long)kmax);
-        atomicAdd((unsigned long long *)&scratch[2], (unsigned long long)cnt);
-        for (int i = 0; i < P.npayload; ++i) {
-            atomicMin((long long *)&scratch[3 + 2 * i], (long long)pmin[i]);
-            atomicMax((long long *)&scratch[4 + 2 * i], (long long)pmax[i]);
+    // one set of atomics per block, not per warp: they all land on the same seven words
+    __shared__ int64_t part[8][3 + 2 * SJQ_MAX_PAYLOADS];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) {
+        part[warp][0] = kmin;
+        part[warp][1] = kmax;
+        part[warp][2] = cnt;
+        for (int i = 0; i < SJQ_MAX_PAYLOADS; ++i) {
+            part[warp][3 + 2 * i] = pmin[i];
+            part[warp][4 + 2 * i] = pmax[i];
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < 3 + 2 * SJQ_MAX_PAYLOADS) {
+        const int f = threadIdx.x; // 0 kmin, 1 kmax, 2 count, then (min, max) per payload
+        const bool is_min = f == 0 || (f >= 3 && ((f - 3) & 1) == 0), is_sum = f == 2;
+        int64_t v = part[0][f];
+        for (int w = 1; w < (int)(blockDim.x >> 5); ++w) {
+            const int64_t t = part[w][f];
+            v = is_sum ? v + t : is_min ? (t < v ? t : v) : (t > v ? t : v);
+        }
+        int64_t block_cnt = 0;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) block_cnt += part[w][2];
+        if (block_cnt > 0 && f < 3 + 2 * P.npayload) {
+            if (is_sum) atomicAdd((unsigned long long *)&scratch[f], (unsigned long long)v);
+            else if (is_min) atomicMin((long long *)&scratch[f], (long long)v);
+            else atomicMax((long long *)&scratch[f], (long long)v);
         }
     }
 }
@@ -258,8 +291,8 @@ __global__ void __launch_bounds__(256) build_kernel(const __grid_constant__ Buil
             hash_insert<unsigned int>(B, (unsigned int)k32, (unsigned int)kEmptyKey32, (uint64_t)(int64_t)k32, code);
         }
     }
-    inserted = (unsigned long long)warp_sum((int64_t)inserted);
-    if ((threadIdx.x & 31) == 0 && inserted) atomicAdd(&B.header[0], inserted);
+    inserted = block_sum(inserted);
+    if (threadIdx.x == 0 && inserted) atomicAdd(&B.header[0], inserted);
 }
 
 // Count occupied slots of a direct table; a repeated key leaves fewer occupied slots than inserted rows.  The
@@ -287,10 +320,9 @@ __global__ void __launch_bounds__(256) direct_count_kernel(const __grid_constant
             occ += set;
         }
     }
-    occ = (unsigned long long)warp_sum((int64_t)occ);
-    if ((threadIdx.x & 31) == 0 && occ) atomicAdd(&B.header[1], occ);
-    __syncthreads();
+    occ = block_sum(occ);
     if (threadIdx.x == 0) {
+        if (occ) atomicAdd(&B.header[1], occ);
         __threadfence();
         if (atomicAdd(&B.header[2], 1ULL) == (unsigned long long)gridDim.x - 1) {
             __threadfence();
