@@ -131,7 +131,7 @@ class RunOpts:
     host_copy_all: bool = False  # run_host: copy every referenced column instead of reading sparse ones in place
     dense_slots: int = 0  # level 0: 0 auto, 2, or 4 groups of four rows per thread (4 needs specialise)
     group_hash_always: bool = False  # HASHED: keep the group hash table even when the key domain is small
-    warp_agg: int = 0  # group-by terminal: 0 auto, 1 add equal keys inside the warp before the atomics, 2 never
+    warp_agg: int = 0  # group-by terminal: 1 = add equal keys inside the warp before the atomics; 0 / 2 = off
     unfused_scratch: Optional[torch.Tensor] = None  # ablation: run operator at a time with this CUDA uint8 scratch
     pass_ppm: Sequence[int] = ()  # measured pass fractions (parts per million): predicates, then joins; 0 = unknown
 
