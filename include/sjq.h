@@ -337,7 +337,23 @@ typedef struct sjq_run_opts {
                                   estimates order the stages, split them into levels, pick the aggregation path
                                   and decide copy versus in-place reads in sjq_run_host: they change the run time,
                                   never the result. */
+    int32_t hot_keys; /* open-addressing joins: 0 = library chooses (a hot-key table is used when `hot_scratch` is
+                         given, the table sits behind its presence bitmap, its codes are at most 32 bits wide, the
+                         kernel is compiled for the query (`specialise`) and the fact table has at least 2^26
+                         rows), 1 = whenever the scratch is given, 2 = never.
+                         Section 3.3 keeps the probed structure small enough to stay in cache; an open-addressing
+                         table over millions of keys cannot, but with skewed foreign keys the answers for the few
+                         keys that carry most rows can: before the fused pass three small kernels sample the
+                         foreign-key column (2^18 evenly spaced rows), pick the keys seen most often and look each
+                         up in the dimension table once; the fused kernel holds the 2048 answers (present with
+                         this code / absent) in shared memory and consults them before the bitmap and before the
+                         exact probe.  When the keys held cover less than a tenth of the sample the table is left
+                         empty and the kernel skips the look-ups.  Same result either way; no host wait. */
+    void *hot_scratch;        /* device scratch of at least SJQ_HOT_SCRATCH_BYTES bytes (16-byte aligned), used by */
+    size_t hot_scratch_bytes; /* this run only; NULL = no hot-key table */
 } sjq_run_opts;
+
+#define SJQ_HOT_SCRATCH_BYTES ((size_t)3 * 1048576 + 65536)
 
 /* What the planner decided for a run (for reports and tests). */
 typedef struct sjq_run_info {

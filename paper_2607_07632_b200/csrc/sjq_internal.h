@@ -115,6 +115,20 @@ __host__ __device__ inline uint32_t filter_hash(uint64_t k)
     return (uint32_t)(k >> 32);
 }
 
+// Hot-key table of an open-addressing join (built per run from a sample of the foreign keys, held in shared
+// memory by the fused kernel): direct-mapped, 16-byte entries {key low word, key high word, payload code,
+// state}; state 0 = free, 1 = the key is in the dimension table (code valid), 2 = the key is absent.  Entry
+// kHotSlots is a header whose first word counts the keys stored.
+constexpr int kHotSlots = 2048;            // 32 KB of shared memory
+constexpr int kHotCountSlots = 1 << 18;    // sample count table (global scratch)
+constexpr int kHotSamples = 1 << 18;       // foreign keys sampled per run
+__host__ __device__ inline uint32_t hot_hash(uint64_t k)
+{
+    k ^= k >> 31;
+    k *= 0xBF58476D1CE4E5B9ULL;
+    return (uint32_t)(k >> 37);
+}
+
 // first-error-wins store into the status word
 __device__ inline void set_status(int32_t *status, int32_t code) { atomicCAS(status, 0, code); }
 

@@ -167,7 +167,8 @@ std::string jit_shape_header(const RunParams &P, int agg, bool mul, bool hash, i
           << "; S.never = " << (int)S.never << "; S.nset = " << (int)S.nset << "; S.set_idx = " << (int)S.set_idx
           << "; S.in_smem = " << (int)S.in_smem << "; S.kind = " << (int)S.kind << "; S.simple = " << (int)S.simple
           << "; S.acc = " << (int)S.acc << "; S.acc32 = " << S.acc32 << "; S.code_bits = " << (int)S.code_bits
-          << "; S.issue_after = " << (int)S.issue_after << "; S.full = " << (int)S.full << ";\n";
+          << "; S.issue_after = " << (int)S.issue_after << "; S.full = " << (int)S.full << "; S.hot = " << (int)S.hot
+          << ";\n";
         for (int i = 0; i < 9; ++i) {
             // INT64_MIN cannot be written as a literal
             if (S.mult[i] == INT64_MIN) o << "        S.mult[" << i << "] = (-9223372036854775807LL - 1);";
@@ -198,7 +199,7 @@ std::string shape_key(const RunParams &P, int agg, bool mul, bool hash, int lb_t
     for (int s = 0; s < P.nstages; ++s) {
         const DStage &S = P.st[s];
         const uint8_t b[] = {S.op, S.is64, S.neg, S.never, S.nset, S.set_idx, S.in_smem, S.kind, S.simple, S.code_bits,
-                             (uint8_t)S.issue_after, S.full};
+                             (uint8_t)S.issue_after, S.full, S.hot};
         put_raw(b, sizeof(b));
         put_raw(&S.acc, sizeof(S.acc));
         put_raw(&S.acc32, sizeof(S.acc32));

@@ -84,7 +84,10 @@ struct DStage {
     int8_t issue_after; // final level of a compiled kernel: the column is requested once this stage's mask is known
                         // (a stage before the level's first one = on entry)
     uint8_t full;   // sub-byte direct table holding every key of its range: a probe hits iff its key is in range
-    uint8_t pad[1];
+    uint8_t hot;    // open-addressing join (its bitmap stage and its exact probe): consult the hot-key table first
+    const void *hot_tab; // hot-key table in global memory (kHotSlots + 1 entries), copied to shared memory per block
+    uint32_t hot_off;    // byte offset of that copy in dynamic shared memory
+    uint32_t hot_pad;
 };
 static_assert(sizeof(DStage) % 8 == 0, "stage descriptors are copied as 64-bit words");
 

@@ -97,7 +97,8 @@ class _RunOpts(ctypes.Structure):
                 ("host_copy_all", ctypes.c_int32), ("dense_slots", ctypes.c_int32),
                 ("group_hash_always", ctypes.c_int32), ("warp_agg", ctypes.c_int32), ("unfused", ctypes.c_int32),
                 ("unfused_scratch", ctypes.c_void_p), ("unfused_scratch_bytes", ctypes.c_size_t),
-                ("pass_ppm", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS))]
+                ("pass_ppm", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS)), ("hot_keys", ctypes.c_int32),
+                ("hot_scratch", ctypes.c_void_p), ("hot_scratch_bytes", ctypes.c_size_t)]
 
 
 class RunInfo(ctypes.Structure):
@@ -134,6 +135,8 @@ class RunOpts:
     warp_agg: int = 0  # group-by terminal: 1 = add equal keys inside the warp before the atomics; 0 / 2 = off
     unfused_scratch: Optional[torch.Tensor] = None  # ablation: run operator at a time with this CUDA uint8 scratch
     pass_ppm: Sequence[int] = ()  # measured pass fractions (parts per million): predicates, then joins; 0 = unknown
+    hot_keys: int = 0  # open-addressing joins: 0 auto, 1 hot-key table whenever possible, 2 never
+    hot_scratch: Optional[torch.Tensor] = None  # CUDA uint8 scratch of HOT_SCRATCH_BYTES; run() supplies one if None
 
     def to_c(self) -> _RunOpts:
         o = _RunOpts()
@@ -146,6 +149,10 @@ class RunOpts:
         for i, v in enumerate(self.pass_ppm):
             o.pass_ppm[i] = int(v)
         o.warp_agg = self.warp_agg
+        o.hot_keys = self.hot_keys
+        if self.hot_scratch is not None:
+            o.hot_scratch = self.hot_scratch.data_ptr()
+            o.hot_scratch_bytes = self.hot_scratch.numel()
         if self.unfused_scratch is not None:
             o.unfused = 1
             o.unfused_scratch = self.unfused_scratch.data_ptr()
@@ -634,6 +641,9 @@ def run(fact: dict, preds=(), joins=(), key=None, agg=None, mode: str = "SCALAR"
         res = result if result is not None else alloc_result(mode, num_groups, capacity, agg.want_count, device)
         cres = _result_struct(res)
         copts = (opts or RunOpts()).to_c()
+        if not copts.hot_scratch and copts.hot_keys != 2 and any(t.layout.kind_name.startswith("HASH") for _, t in joins):
+            scratch = _hot_scratch(device)  # one per device, reused by every run (runs on one stream are ordered)
+            copts.hot_scratch, copts.hot_scratch_bytes = scratch.data_ptr(), scratch.numel()
         rc = lib().sjq_run(carr, len(names), parr, len(preds), jarr, len(joins),
                            ctypes.byref(kexpr) if kexpr is not None else None, ctypes.byref(aexpr),
                            ctypes.byref(spec), ctypes.byref(cres), ctypes.byref(copts), _stream_ptr(device),
@@ -644,6 +654,18 @@ def run(fact: dict, preds=(), joins=(), key=None, agg=None, mode: str = "SCALAR"
 
 
 STATIC_MAX_GROUPS = 65536
+HOT_SCRATCH_BYTES = 3 * 1048576 + 65536  # SJQ_HOT_SCRATCH_BYTES
+_hot_scratch_by_device: dict = {}
+
+
+def _hot_scratch(device) -> torch.Tensor:
+    """Scratch for the hot-key table of open-addressing joins (sjq_run_opts.hot_scratch).  The library
+    allocates nothing; this binding keeps one buffer per device.  Runs that may overlap on different streams
+    need a buffer each: pass RunOpts.hot_scratch."""
+    key = torch.device(device).index if torch.device(device).index is not None else torch.cuda.current_device()
+    if key not in _hot_scratch_by_device:
+        _hot_scratch_by_device[key] = torch.empty(HOT_SCRATCH_BYTES, dtype=torch.uint8, device=device)
+    return _hot_scratch_by_device[key]
 
 
 def run_hashed_static(fact: dict, preds=(), joins=(), key=None, agg=None, capacity: int = 0,

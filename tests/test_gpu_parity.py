@@ -633,3 +633,72 @@ def test_operator_at_a_time_ablation_matches_the_oracle(mk):
     with pytest.raises(sjq.SjqError) as e:
         sjq.run_workload(w, to_dev(fact), tables, sjq.RunOpts(unfused_scratch=scratch[: w.n_rows // 2]))
     assert e.value.status == 5
+
+
+def _hot_variants():
+    return [sjq.RunOpts(hot_keys=1), sjq.RunOpts(hot_keys=1, specialise=True), sjq.RunOpts(hot_keys=2),
+            sjq.RunOpts(hot_keys=1, compaction=1), sjq.RunOpts(hot_keys=1, specialise=True, compaction=2),
+            sjq.RunOpts(hot_keys=1, eager_loads=True)]
+
+
+def test_hot_key_table_skewed_keys_against_the_oracle():
+    """The hot-key table of an open-addressing join (heaviest foreign keys answered from shared memory): the
+    Zipf-skewed 64-bit-key shape, where three quarters of the heavy keys are absent from the filtered dimension,
+    bit for bit against the oracle with the table forced on, off, and in every kernel form."""
+    w = W.config5(1_300_007, 300_000)
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    dev_fact = to_dev(fact)
+    tables = None
+    for opts in _hot_variants():
+        res, exp, tables = run_both(w, fact, hd, opts=opts, dev_fact=dev_fact, tables=tables)
+        assert res.status() == 0
+        compare(w, res, exp)
+    assert int(res.counts.sum().item()) > 100_000
+    # the table really was in use: its header (after the count table, the claims and 2048 entries) counts the keys
+    # held, and together they cover a good part of the sampled rows
+    scratch = torch.empty(sjq.sjq.HOT_SCRATCH_BYTES, dtype=torch.uint8, device="cuda")
+    res, exp, _ = run_both(w, fact, hd, opts=sjq.RunOpts(hot_keys=1, hot_scratch=scratch), dev_fact=dev_fact,
+                           tables=tables)
+    compare(w, res, exp)
+    held, _, covered, _ = scratch[(1 << 18) * 12 + 2048 * 4 + 2048 * 16:][:16].view(torch.int32).tolist()
+    assert held > 500 and covered > 0.3 * min(w.n_rows, 1 << 18)
+
+
+def test_hot_key_table_uniform_keys_and_32_bit_keys():
+    # four open-addressing joins on 32-bit keys with payload codes (the first one gets the hot table); the keys
+    # are uniform, so the table stays empty or thin: either way the result is the oracle's
+    w = W.config3(1_200_007)
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    dev = {k: to_dev(v) for k, v in hd.items()}
+    tables = {d.name: sjq.build_dim(dev[d.name], d.key, d.preds, d.payloads, force_kind=sjq.sjq.FORCE_HASH)
+              for d in w.dims}
+    dev_fact = to_dev(fact)
+    for opts in _hot_variants():
+        res, exp, _ = run_both(w, fact, hd, opts=opts, dev_fact=dev_fact, tables=tables)
+        assert res.status() == 0
+        compare(w, res, exp)
+
+
+def test_hot_key_table_heavy_keys_with_special_values():
+    """A few keys carry nearly all rows, among them -1 (the count table's free-slot pattern), the table's empty
+    marker (never a key: always a miss) and keys the dimension does not hold."""
+    rng = np.random.default_rng(7)
+    n = 400_003
+    dim_keys = np.concatenate([np.array([-1, 5, 7_000_000_000, -9_000_000_000], dtype=np.int64),
+                               rng.integers(-2**62, 2**62, 5000, dtype=np.int64)])
+    dim = {"key": dim_keys, "pay": rng.integers(0, 1000, len(dim_keys)).astype(np.int32),
+           "attr": rng.integers(0, 4, len(dim_keys)).astype(np.int32)}
+    dim["attr"][:4] = [0, 0, 3, 0]  # 7_000_000_000 is filtered out: a heavy absent key
+    heavy = np.array([-1, 5, 7_000_000_000, -9_000_000_000, np.iinfo(np.int64).min, 123456789], dtype=np.int64)
+    pick = rng.integers(0, 100, n)
+    fk = np.where(pick < 90, heavy[pick % len(heavy)], dim_keys[rng.integers(0, len(dim_keys), n)])
+    fact = {"fk": fk.astype(np.int64), "m": rng.integers(0, 1_000_000, n).astype(np.int32)}
+    w = adhoc("hot_special", fact, [("dim", dim, "key", [Pred("attr", "LT", 3)], ["pay"], True)], [("fk", "dim")], [],
+              KeyExpr((Term("PAYLOAD", 0, 0),), modulo=64), AggExpr("COL", Term("FACT", "m")), "DENSE", num_groups=64)
+    tables = None
+    for opts in _hot_variants():
+        res, exp, tables = run_both(w, fact, {"dim": dim}, opts=opts, tables=tables)
+        assert res.status() == 0
+        compare(w, res, exp)
