@@ -702,3 +702,18 @@ def test_hot_key_table_heavy_keys_with_special_values():
         res, exp, tables = run_both(w, fact, {"dim": dim}, opts=opts, tables=tables)
         assert res.status() == 0
         compare(w, res, exp)
+
+
+def test_wrapping_product_matches_the_oracle():
+    # products beyond 63 bits wrap modulo 2^64 the same way on both sides (scalar and grouped)
+    rng = np.random.default_rng(11)
+    n = 10_007
+    fact = {"x": rng.integers(-2**62, 2**62, n, dtype=np.int64), "y": rng.integers(-2**62, 2**62, n, dtype=np.int64),
+            "g": rng.integers(0, 50, n).astype(np.int32)}
+    agg = AggExpr("MUL", Term("FACT", "x", 0, 3), Term("FACT", "y", 0, -5))
+    for w in (adhoc("wrapmul", fact, [], [], [], None, agg, "SCALAR"),
+              adhoc("wrapmul_g", fact, [], [], [], KeyExpr((Term("FACT", "g"),)), agg, "DENSE", num_groups=50)):
+        for opts in (sjq.RunOpts(), sjq.RunOpts(specialise=True)):
+            res, exp, _ = run_both(w, fact, {}, opts=opts)
+            assert res.status() == 0
+            compare(w, res, exp)

@@ -237,3 +237,19 @@ def test_sum_wraps_modulo_2_64():
     fact = {"v": np.array([2**62, 2**62, 2**62, 2**62, 5], np.int64)}
     w = adhoc("wrap", fact, [], [], [], None, AggExpr("COL", Term("FACT", "v")), "SCALAR")
     assert _run(w, fact, {})["sum"] == 5
+
+
+def _wrap64(x: int) -> int:
+    x &= (1 << 64) - 1
+    return x - (1 << 64) if x >= (1 << 63) else x
+
+
+def test_product_wraps_modulo_2_64():
+    # x * y beyond 63 bits, scaled terms included: the sum is the exact integer result reduced modulo 2^64
+    x = np.array([2**40, -(2**45), 3037000500, 2**62, -7], np.int64)
+    y = np.array([2**30, 2**33, 3037000500, 6, 2**61], np.int64)
+    fact = {"x": x, "y": y}
+    w = adhoc("wrapmul", fact, [], [], [], None, AggExpr("MUL", Term("FACT", "x", 0, 3), Term("FACT", "y", 0, -5)), "SCALAR")
+    exact = sum(int(a) * 3 * int(b) * -5 for a, b in zip(x, y))
+    assert exact.bit_length() > 64
+    assert _run(w, fact, {})["sum"] == _wrap64(exact)
