@@ -429,6 +429,25 @@ sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *preds, int np
                    const sjq_result *out, const sjq_run_opts *opts, void *stream, sjq_run_info *info);
 
 /*
+ * Put a HASHED result into its canonical order: ascending (signed) key.
+ * Section 3.3's global table returns its groups in table order, which depends
+ * on the hash function and the capacity; the paper compares results through an
+ * order-free checksum (Section 2.2), this library gives the list itself an
+ * order instead.  A radix sort of (key, position) pairs on the device, then
+ * one gather of the three arrays.
+ *   keys/sums/counts  device arrays of `capacity` entries (8-byte aligned), of
+ *                     which the first *n_groups hold the result; sorted in place
+ *   n_groups          device pointer, read by the kernels (no host wait)
+ *   scratch           device scratch of sjq_result_sort_scratch_bytes(capacity)
+ *                     bytes, 16-byte aligned (about 40 bytes per entry)
+ * capacity <= 2^31.  Enqueues 27 small kernels on `stream`; does not
+ * synchronise.  Errors: INVALID_ARG, ALIGN, BUFFER_SMALL, CUDA.
+ */
+sjq_status sjq_result_sort_scratch_bytes(int64_t capacity, size_t *bytes);
+sjq_status sjq_result_sort(int64_t *keys, int64_t *sums, int64_t *counts, const int64_t *n_groups, int64_t capacity,
+                           void *scratch, size_t scratch_bytes, void *stream);
+
+/*
  * Merge lists of (key, sum, count) triples into one list with one entry per
  * distinct key, sums and counts added (int64, wrapping).  This is the exchange
  * step of a row-sharded run over several GPUs (the paper's second scale point,

@@ -542,11 +542,35 @@ class Result:
             raise SjqError(st, "sjq_run")
         return self
 
+    def sort(self) -> "Result":
+        """sjq_result_sort: put a HASHED result into ascending key order, in place, on the current stream."""
+        capacity = self.keys.numel()
+        L = lib()
+        L.sjq_result_sort_scratch_bytes.restype = ctypes.c_int32
+        L.sjq_result_sort_scratch_bytes.argtypes = [ctypes.c_int64, ctypes.POINTER(ctypes.c_size_t)]
+        L.sjq_result_sort.restype = ctypes.c_int32
+        L.sjq_result_sort.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                      ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        need = ctypes.c_size_t(0)
+        rc = L.sjq_result_sort_scratch_bytes(capacity, ctypes.byref(need))
+        if rc != 0:
+            raise SjqError(rc, "sjq_result_sort_scratch_bytes")
+        device = self.keys.device
+        with torch.cuda.device(device):
+            scratch = torch.empty(need.value, dtype=torch.uint8, device=device)
+            rc = L.sjq_result_sort(self.keys.data_ptr(), self.sums.data_ptr(), self.counts.data_ptr(),
+                                   self.n_groups.data_ptr(), capacity, scratch.data_ptr(), scratch.numel(),
+                                   _stream_ptr(device))
+        if rc != 0:
+            raise SjqError(rc, "sjq_result_sort")
+        return self
+
     def hashed_sorted(self):
-        """(keys, sums, counts) of a HASHED result in ascending key order."""
+        """(keys, sums, counts) of a HASHED result in ascending key order (copies; the result is left as it is)."""
+        tmp = Result("HASHED", self.sums.clone(), self.counts.clone(), self.keys.clone(), self.n_groups,
+                     self.status_dev, None).sort()
         n = int(self.n_groups.item())
-        k, idx = torch.sort(self.keys[:n])
-        return k, self.sums[:n][idx], self.counts[:n][idx]
+        return tmp.keys[:n], tmp.sums[:n], tmp.counts[:n]
 
 
 def _term(t, names) -> _Term:

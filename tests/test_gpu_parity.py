@@ -717,3 +717,30 @@ def test_wrapping_product_matches_the_oracle():
             res, exp, _ = run_both(w, fact, {}, opts=opts)
             assert res.status() == 0
             compare(w, res, exp)
+
+
+@pytest.mark.parametrize("n,capacity", [(0, 8), (1, 1), (5, 64), (1023, 1024), (1025, 4096), (100_003, 131_072),
+                                        (300_000, 300_000)])
+def test_result_sort_orders_triples_by_signed_key(n, capacity):
+    # distinct keys over the whole signed range, special values included; entries past n_groups stay untouched
+    rng = np.random.default_rng(n + 1)
+    keys = np.unique(np.concatenate([rng.integers(-2**63, 2**63 - 1, n + 16, dtype=np.int64),
+                                     np.array([0, -1, 1, np.iinfo(np.int64).min, np.iinfo(np.int64).max, 255, 256,
+                                               -256, 2**32, -2**32], dtype=np.int64)]))
+    keys = rng.permutation(keys)[:n]
+    sums = rng.integers(-2**62, 2**62, capacity, dtype=np.int64)
+    counts = rng.integers(0, 2**40, capacity, dtype=np.int64)
+    allk = np.full(capacity, 77, dtype=np.int64)
+    allk[:n] = keys
+    res = sjq.Result("HASHED", torch.from_numpy(sums.copy()).cuda(), torch.from_numpy(counts.copy()).cuda(),
+                     torch.from_numpy(allk.copy()).cuda(), torch.tensor([n], dtype=torch.int64, device="cuda"),
+                     torch.zeros(1, dtype=torch.int32, device="cuda"), None)
+    res.sort()
+    torch.cuda.synchronize()
+    order = np.argsort(keys, kind="stable")
+    assert np.array_equal(res.keys.cpu().numpy()[:n], keys[order])
+    assert np.array_equal(res.sums.cpu().numpy()[:n], sums[:n][order])
+    assert np.array_equal(res.counts.cpu().numpy()[:n], counts[:n][order])
+    assert np.array_equal(res.keys.cpu().numpy()[n:], allk[n:])
+    assert np.array_equal(res.sums.cpu().numpy()[n:], sums[n:])
+    assert np.array_equal(res.counts.cpu().numpy()[n:], counts[n:])
