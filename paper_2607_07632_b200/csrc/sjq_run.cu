@@ -762,7 +762,8 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     }
 
     bool has_hash = false; // kernels without the hash probe are leaner; pick by what the stages need
-    for (int s2 = 0; s2 < ns; ++s2) has_hash |= P.st[s2].op == OP_HASH32 || P.st[s2].op == OP_HASH64;
+    for (int s2 = 0; s2 < ns; ++s2)
+        has_hash |= P.st[s2].op == OP_HASH32 || P.st[s2].op == OP_HASH64 || P.st[s2].op == OP_HASHBITS;
 
     // ------------------------------------------------------------ launch shape
     int per_sm = 0;
