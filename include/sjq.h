@@ -61,7 +61,9 @@ enum {
     SJQ_ERR_GROUP_RANGE = 18,    /* dense mode: a group key fell outside [0, num_groups) */
     SJQ_ERR_GROUP_OVERFLOW = 19, /* hashed mode: more distinct groups than the capacity */
     SJQ_ERR_RESERVED_KEY = 20,   /* a dimension key equals the reserved empty marker (minimum of its type) */
-    SJQ_ERR_LAYOUT_MISMATCH = 21 /* build saw a key or payload outside the planned layout */
+    SJQ_ERR_LAYOUT_MISMATCH = 21, /* build saw a key or payload outside the planned layout */
+    SJQ_ERR_ASYNC_WAIT = 22       /* a bounded wait for a bulk-asynchronous copy ran out; the kernel went on with
+                                     plain loads, so the result is still exact, but the device needs a look */
 };
 
 enum { SJQ_I32 = 0, SJQ_I64 = 1 };
@@ -351,6 +353,15 @@ typedef struct sjq_run_opts {
                          empty and the kernel skips the look-ups.  Same result either way; no host wait. */
     void *hot_scratch;        /* device scratch of at least SJQ_HOT_SCRATCH_BYTES bytes (16-byte aligned), used by */
     size_t hot_scratch_bytes; /* this run only; NULL = no hot-key table */
+    int32_t l0_bulk; /* first column of a query with survivor queues, compiled kernels only: 1 = bring it into
+                        shared memory with bulk-asynchronous copies (`cp.async.bulk` global -> shared completing on
+                        an mbarrier; one copy per block tile of 12 to 64 KB, three in flight per block; no tensor
+                        map, no cluster multicast, this GPU's memory only) whenever the shared memory is there;
+                        0 or 2 = 128-bit loads with L2 prefetch, the default: Section 3.2's scan is bound by the
+                        bytes in flight, and in this kernel, whose warps run independently, the loads keep more
+                        of them in flight than the staged tiles do (measured slower at every point of the
+                        selectivity sweep).  Every wait on a copy is bounded; one that runs out sets
+                        SJQ_ERR_ASYNC_WAIT in *out->status and the kernel goes on with loads. */
 } sjq_run_opts;
 
 #define SJQ_HOT_SCRATCH_BYTES ((size_t)3 * 1048576 + 65536)

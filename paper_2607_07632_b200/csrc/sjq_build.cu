@@ -783,6 +783,7 @@ extern "C" const char *sjq_strerror(sjq_status s)
     case SJQ_ERR_GROUP_OVERFLOW: return "more distinct groups than the hashed capacity";
     case SJQ_ERR_RESERVED_KEY: return "dimension key equals the reserved empty marker";
     case SJQ_ERR_LAYOUT_MISMATCH: return "dimension data does not match the planned layout";
+    case SJQ_ERR_ASYNC_WAIT: return "a bounded wait for a bulk-asynchronous copy ran out (result still exact)";
     default: return "unknown status";
     }
 }

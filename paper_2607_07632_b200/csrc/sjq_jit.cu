@@ -155,7 +155,7 @@ std::string jit_shape_header(const RunParams &P, int agg, bool mul, bool hash, i
     o << "#define SJQ_JIT_qfold " << P.qfold << "u\n";
     o << "#define SJQ_JIT_want_count " << P.want_count << "\n#define SJQ_JIT_eager " << P.eager
       << "\n#define SJQ_JIT_has_key " << P.has_key << "\n#define SJQ_JIT_mod32 " << P.mod32
-      << "\n#define SJQ_JIT_warp_agg " << P.warp_agg << "\n";
+      << "\n#define SJQ_JIT_warp_agg " << P.warp_agg << "\n#define SJQ_JIT_l0_bulk " << P.l0_bulk << "\n";
     put(o, "modulo", P.modulo);
     o << "#define SJQ_JIT_modmask " << P.modmask << "ULL\n";
     o << "namespace sjq {\nnamespace {\n"
@@ -192,7 +192,8 @@ std::string shape_key(const RunParams &P, int agg, bool mul, bool hash, int lb_t
     k.reserve(64 + (size_t)P.nstages * 128);
     auto put_raw = [&](const void *p, size_t n) { k.append(static_cast<const char *>(p), n); };
     const int32_t head[] = {agg, mul ? 1 : 0, hash ? 1 : 0, lb_threads, lb_blocks, P.nstages, P.nd0, P.nq,
-                            P.rows, P.want_count, P.eager, P.has_key, P.mod32, (int32_t)P.qfold, P.slots, P.warp_agg};
+                            P.rows, P.want_count, P.eager, P.has_key, P.mod32, (int32_t)P.qfold, P.slots, P.warp_agg,
+                            P.l0_bulk};
     put_raw(head, sizeof(head));
     put_raw(&P.modulo, sizeof(P.modulo));
     put_raw(&P.modmask, sizeof(P.modmask));
@@ -462,6 +463,28 @@ int canned_shape(int id, RunParams *P, int *agg, bool *mul, bool *hash)
         P->nstages = 4, P->nd0 = 0, P->nq = 0;
         P->modulo = 1000, P->mod32 = 1, P->want_count = 1;
         *agg = AGG_HASH, *hash = true;
+        return 1;
+    case 4: // one predicate on an int32 first column staged by bulk-asynchronous copies, one join with a 2-bit
+            // payload, shared-memory group table
+        P->st[0] = canned(OP_PRED_RANGE, ST_PRED, false, 0, 0, false);
+        P->st[1] = canned(OP_DIRECT_U2, ST_PROBE, false, 16, 2, false);
+        P->st[2] = canned(OP_LOAD, ST_LOAD, false, 1, 0, false);
+        P->st[3] = canned(OP_LOAD, ST_LOAD, false, 2, 0, false);
+        P->nstages = 4, P->nd0 = 1, P->nq = 1;
+        P->modulo = 1000, P->mod32 = 1, P->want_count = 1;
+        P->l0_bulk = 1;
+        *agg = AGG_SMEM;
+        return 1;
+    case 5: // 64-bit first column staged by bulk-asynchronous copies, hot-key table in front of the presence bitmap
+            // and of the open-addressing probe
+        P->st[0] = canned(OP_HASHBITS, ST_PROBE, true, 0, 0, false);
+        P->st[1] = canned(OP_HASH64, ST_PROBE, true, 8, 32, false);
+        P->st[2] = canned(OP_LOAD, ST_LOAD, false, 2, 0, false);
+        P->st[0].hot = 1, P->st[1].hot = 2;
+        P->nstages = 3, P->nd0 = 1, P->nq = 1;
+        P->modulo = 4096, P->modmask = 4095, P->mod32 = 1, P->want_count = 1;
+        P->l0_bulk = 1;
+        *agg = AGG_SMEM, *hash = true;
         return 1;
     default: return 0;
     }

@@ -761,6 +761,27 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
         }
     }
 
+    // ------------------------------------------------------------ bulk-asynchronous staging of the first column
+    // A kernel compiled for a query with survivor queues can have its first column copied into shared memory by
+    // the copy engine, one tile (block size x 4 x slots values) per copy, three in flight per block.  Only when
+    // asked for: measured on the selectivity sweep (600 M rows) the staged kernel is slower than 128-bit loads
+    // with L2 prefetch at every point (0.01 %: 0.42 vs 0.37 ms; 1 %: 0.64 vs 0.53; 10 %, 1000 groups: 1.25 vs 1.21)
+    // and much slower where its buffers crowd the shared memory (city x city: 1.09 vs 0.73 ms), although a bare
+    // scan kernel built on the same copies moves 7.3 TB/s against 6.7 TB/s for loads: the warps of the fused
+    // kernel consume a tile at their own pace, so the refill of a buffer waits for the slowest of them.
+    const size_t smem_without_bulk = smem;
+    if (opts.l0_bulk < 0 || opts.l0_bulk > 2) return SJQ_ERR_INVALID_ARG;
+    if (opts.specialise && !opts.unfused && P.nq > 0 && n > 0 && opts.l0_bulk == 1) {
+        const size_t tile_bytes = (size_t)block * 4 * P.slots * (P.st[0].is64 ? 8 : 4);
+        const size_t at = align_up(smem, 128);
+        const size_t total = at + 3 * tile_bytes + 3 * 8 + 3 * 4 + 4;
+        if (total <= smem_cap) {
+            P.l0_bulk = 1;
+            P.smem_l0 = (uint32_t)at;
+            smem = total;
+        }
+    }
+
     bool has_hash = false; // kernels without the hash probe are leaner; pick by what the stages need
     for (int s2 = 0; s2 < ns; ++s2)
         has_hash |= P.st[s2].op == OP_HASH32 || P.st[s2].op == OP_HASH64 || P.st[s2].op == OP_HASHBITS;
@@ -774,7 +795,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     const int lb_blocks = single_block ? 1
                           : opts.ctas_per_sm > 0 ? opts.ctas_per_sm
                           : block > 512 ? 1
-                          : (block <= 384 && smem <= ((size_t)48 << 10)) ? 3
+                          : (block <= 384 && smem_without_bulk <= ((size_t)48 << 10)) ? 3
                                                                         : 2;
     st = jit ? jit_occupancy(P, aggp, mul, has_hash, block, lb_blocks, smem, &per_sm)
              : fused_occupancy(aggp, mul, has_hash, block, smem, &per_sm);

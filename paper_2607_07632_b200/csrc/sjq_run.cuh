@@ -121,6 +121,8 @@ struct RunParams {
     uint32_t smem_stages; // byte offset of the stage descriptors copied to shared memory
     uint32_t smem_groups; // byte offset of the shared group table
     uint32_t smem_queue;  // byte offset of the per-warp survivor queues
+    uint32_t smem_l0;     // byte offset of the per-warp staging buffers of the first column (then their mbarriers)
+    int32_t l0_bulk;      // compiled kernels: the first column arrives by bulk-asynchronous copies into shared memory
 };
 
 #if !defined(SJQ_JIT)

@@ -98,7 +98,7 @@ class _RunOpts(ctypes.Structure):
                 ("group_hash_always", ctypes.c_int32), ("warp_agg", ctypes.c_int32), ("unfused", ctypes.c_int32),
                 ("unfused_scratch", ctypes.c_void_p), ("unfused_scratch_bytes", ctypes.c_size_t),
                 ("pass_ppm", ctypes.c_int32 * (MAX_PREDS + MAX_JOINS)), ("hot_keys", ctypes.c_int32),
-                ("hot_scratch", ctypes.c_void_p), ("hot_scratch_bytes", ctypes.c_size_t)]
+                ("hot_scratch", ctypes.c_void_p), ("hot_scratch_bytes", ctypes.c_size_t), ("l0_bulk", ctypes.c_int32)]
 
 
 class RunInfo(ctypes.Structure):
@@ -137,6 +137,7 @@ class RunOpts:
     pass_ppm: Sequence[int] = ()  # measured pass fractions (parts per million): predicates, then joins; 0 = unknown
     hot_keys: int = 0  # open-addressing joins: 0 auto, 1 hot-key table whenever possible, 2 never
     hot_scratch: Optional[torch.Tensor] = None  # CUDA uint8 scratch of HOT_SCRATCH_BYTES; run() supplies one if None
+    l0_bulk: int = 0  # 1 = first column by bulk-asynchronous copies into shared memory when it fits; 0 / 2 = loads
 
     def to_c(self) -> _RunOpts:
         o = _RunOpts()
@@ -150,6 +151,7 @@ class RunOpts:
             o.pass_ppm[i] = int(v)
         o.warp_agg = self.warp_agg
         o.hot_keys = self.hot_keys
+        o.l0_bulk = self.l0_bulk
         if self.hot_scratch is not None:
             o.hot_scratch = self.hot_scratch.data_ptr()
             o.hot_scratch_bytes = self.hot_scratch.numel()

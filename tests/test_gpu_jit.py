@@ -193,3 +193,35 @@ def test_clearing_the_module_cache_recompiles_and_gives_the_same_bits():
     assert L.sjq_jit_cache_clear() == 0
     res2, _, _ = run_both(w, fact, hd, opts=spec(), tables=tables)
     compare(w, res2, exp)
+
+
+BULK_SHAPES = [dict(), dict(block_threads=1024, ctas_per_sm=1), dict(dense_slots=4),
+               dict(block_threads=128, ctas_per_sm=2, compaction=2), dict(rows_per_lane=8)]
+
+
+@pytest.mark.parametrize("n", [0, 1, 255, 3071, 3072, 3073, 6145, 100003, 1_200_011])
+@pytest.mark.parametrize("cfg", ["c1", "c3", "c4d", "c4h", "c5"])
+def test_first_column_staged_by_bulk_copies(cfg, n):
+    """The first column brought into shared memory by bulk-asynchronous copies (one slice per warp and tile,
+    completion on an mbarrier with a bounded wait): int32 and int64 first columns, whole tiles, ragged tails
+    and tables smaller than one tile, several block shapes; bit for bit against the oracle, and the bounded
+    waits never ran out (status 0)."""
+    w = {"c1": lambda: W.config1(n), "c3": lambda: W.config3(n),
+         "c4d": lambda: W.config4(n, 0.1, 1000, dim_rows=50000), "c4h": lambda: W.config4(n, 0.01, 100000, dim_rows=50000),
+         "c5": lambda: W.config5(n, 20000)}[cfg]()
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    dev_fact = to_dev(fact)
+    tables = None
+    for shape in BULK_SHAPES if n > 3000 else BULK_SHAPES[:2]:
+        res, exp, tables = run_both(w, fact, hd, opts=spec(l0_bulk=1, **shape), dev_fact=dev_fact, tables=tables)
+        assert res.status() == 0
+        compare(w, res, exp)
+
+
+@pytest.mark.parametrize("seed", range(360, 372))
+def test_random_queries_with_bulk_staging(seed):
+    w, fact, hd = random_query(seed, n_fact=9000, allow_dup=False, wide_keys=True)
+    res, exp, _ = run_both(w, fact, hd, opts=spec(l0_bulk=1, block_threads=128, ctas_per_sm=1), check=False)
+    assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)
+    compare(w, res, exp)
