@@ -586,7 +586,8 @@ int32_t sjq_release(void);
  * kernel is compiled for the query's shape with NVRTC when sjq_run_opts.specialise is set).
  * Compiled modules are cached per process, keyed by the query's shape.  The compiler needs the device sources:
  * they are looked for in csrc/ beside the library and ../include (the environment variables SJQ_SOURCE_DIR and
- * SJQ_INCLUDE_DIR name other places); SJQ_JIT_VERBOSE=1 prints the compiler's output to stderr.
+ * SJQ_INCLUDE_DIR name other places); SJQ_JIT_VERBOSE=1 prints the compiler's output to stderr.  SJQ_JIT_EXTRA
+ * (extra compiler options, part of the cache key) is a development hook, not a supported interface.
  * sjq_jit_log copies the compiler output of the most recent compilation into `buf` (NUL-terminated, truncated
  * to `bytes`) and returns its full length.  sjq_jit_selftest compiles one of a few built-in query shapes
  * (shape_id 0 .. sjq_jit_selftest(-1, ...) - 1) without touching a device: SJQ_OK if the device code
