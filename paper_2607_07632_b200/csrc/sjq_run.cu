@@ -549,6 +549,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     }
     P.nstages = ns;
     P.eager = opts.eager_loads ? 1 : 0;
+    P.count32 = n < ((int64_t)1 << 32) ? 1 : 0;
     // Load schedule of the final level (used by kernels compiled for the query): a column is requested
     // once the last stage before it that is expected to drop rows has produced its mask, and at most
     // three columns ahead of the stage being processed.
