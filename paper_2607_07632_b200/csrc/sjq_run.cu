@@ -680,6 +680,12 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     // ------------------------------------------------------------ shared memory layout
     // [stage descriptors][staged tables][hot-key table][group table][per-warp survivor queues]
     int block = opts.block_threads ? opts.block_threads : SJQ_LB_THREADS;
+    // A compiled kernel without queues whose rows all meet in a shared group table runs as two blocks of 640
+    // threads per SM: two copies of the table instead of three and 40 warps instead of 36 (selectivity sweep at
+    // 100 %, a thousand groups: 2.73 -> 2.52 ms; 64 groups 2.57 -> 2.39; 4000 groups 3.25 -> 2.56).
+    const bool two_wide_blocks = opts.specialise && !opts.unfused && !opts.block_threads && !opts.ctas_per_sm &&
+                                 P.nq == 0 && aggp == AGG_SMEM;
+    if (two_wide_blocks) block = 640;
     const size_t smem_cap = (size_t)dev.max_smem_optin - 1024; // static reduce scratch + slack
     const size_t stage_bytes = align_up((size_t)ns * sizeof(DStage), 16);
     if (hot_bytes && stage_bytes + hot_bytes + group_bytes +
@@ -794,6 +800,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     // (three blocks of 384 threads when their shared memory leaves the L1 alone: 56 registers are enough for the
     // short pipelines that have so little state, and 36 warps hide more latency than 24)
     const int lb_blocks = single_block ? 1
+                          : two_wide_blocks ? 2
                           : opts.ctas_per_sm > 0 ? opts.ctas_per_sm
                           : block > 512 ? 1
                           : (block <= 384 && smem_without_bulk <= ((size_t)48 << 10)) ? 3
