@@ -133,10 +133,12 @@ def stage_pass_fractions(w, tables, survivors=None):
     return {k: (1.0 if v is None else v) for k, v in frac.items()}
 
 
-def algorithmic_bytes_per_row(w, order, frac):
+def algorithmic_bytes_per_row(w, order, frac, granule: int = 32):
     """Sector model: the first column is read whole; a later column is read for a 32-byte sector
     iff at least one of its rows survived everything evaluated before it.  `order`: the stage labels of
-    the plan that ran; `frac`: pass fraction per label."""
+    the plan that ran; `frac`: pass fraction per label.  granule = 64 gives the same model for 64-byte
+    pieces, the smallest unit DRAM delivered in the ncu captures (reported beside the 32-byte figure,
+    never instead of it)."""
     cols = [p.col for p in w.preds] + [fk for fk, _ in w.joins]
     reach, total, seen, applied = 1.0, 0.0, set(), set()
     for idx in order:
@@ -146,7 +148,7 @@ def algorithmic_bytes_per_row(w, order, frac):
         col = cols[idx]
         width = 8 if w.fact_col(col).is64 else 4
         if col not in seen:
-            total += width * (1.0 - (1.0 - reach) ** (32 // width))
+            total += width * (1.0 - (1.0 - reach) ** (granule // width))
             seen.add(col)
         reach *= frac.get(idx, 1.0)
     referenced = set(cols) | {t.a for t in ((w.key.terms if w.key and w.key.modulo != 1 else ()) + (w.agg.x,) +
@@ -154,7 +156,7 @@ def algorithmic_bytes_per_row(w, order, frac):
     for c in w.fact_cols:  # columns only the key or the aggregate reads
         if c.name not in seen and c.name in referenced:
             width = 8 if c.is64 else 4
-            total += width * (1.0 - (1.0 - reach) ** (32 // width))
+            total += width * (1.0 - (1.0 - reach) ** (granule // width))
     return total
 
 
@@ -388,6 +390,7 @@ def measure_point(sjq, torch, w, fact, tables, specialise, gpu_index, peak, extr
     out = {"workload": w.name, "rows": w.n_rows, "runs": runs, "ms_min": min(ms), "ms_mean": ms_mean,
            "kernel_ms_min": min(kms), "kernel_ms_mean": k_mean, "rows_per_s": w.n_rows / (ms_mean / 1000.0),
            "algorithmic_bytes_per_row": alg, "achieved_gbs": achieved, "frac": achieved / peak,
+           "bytes_per_row_64B_model": algorithmic_bytes_per_row(w, plan["order"], frac, 64),
            "referenced_bytes_per_row": ref_bytes, "effective_gbs_kernel": eff,
            "pct_of_8tbs": 100.0 * eff / CONTRACT_HBM_GBS, "survivors": survivors,
            "pass_fractions": {str(k): round(v, 6) for k, v in frac.items()},
@@ -609,6 +612,9 @@ def main():
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "traffic_source": traffic_note,
                 "algorithmic_bytes_per_row": alg_bpr, "kernel_ms": fused_ms,
+                "bytes_per_row_64B_model": algorithmic_bytes_per_row(w, list(info.order[: info.nstages]), pass_frac, 64),
+                "note": "achieved and frac use the 32-byte-sector model; DRAM delivers 64-byte pieces (ncu traffic), "
+                        "for which the same model gives bytes_per_row_64B_model",
                 "pass_fractions": {str(k): round(v, 6) for k, v in pass_frac.items()},
                 "effective_gbs_kernel": n * ref_bytes / (fused_ms / 1000.0) / 1e9}
 
