@@ -777,13 +777,13 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     // scan kernel built on the same copies moves 7.3 TB/s against 6.7 TB/s for loads: the warps of the fused
     // kernel consume a tile at their own pace, so the refill of a buffer waits for the slowest of them.
     const size_t smem_without_bulk = smem;
-    if (opts.l0_bulk < 0 || opts.l0_bulk > 2) return SJQ_ERR_INVALID_ARG;
-    if (opts.specialise && !opts.unfused && P.nq > 0 && n > 0 && opts.l0_bulk == 1) {
+    if (opts.l0_bulk < 0 || opts.l0_bulk > 3) return SJQ_ERR_INVALID_ARG;
+    if (opts.specialise && !opts.unfused && P.nq > 0 && n > 0 && (opts.l0_bulk == 1 || opts.l0_bulk == 3)) {
         const size_t tile_bytes = (size_t)block * 4 * P.slots * (P.st[0].is64 ? 8 : 4);
         const size_t at = align_up(smem, 128);
         const size_t total = at + 3 * tile_bytes + 3 * 8 + 3 * 4 + 4;
         if (total <= smem_cap) {
-            P.l0_bulk = 1;
+            P.l0_bulk = opts.l0_bulk == 3 ? 2 : 1; // 2: the kernel waits for copies nobody issues (failure-path test)
             P.smem_l0 = (uint32_t)at;
             smem = total;
         }

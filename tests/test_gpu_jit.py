@@ -225,3 +225,19 @@ def test_random_queries_with_bulk_staging(seed):
     res, exp, _ = run_both(w, fact, hd, opts=spec(l0_bulk=1, block_threads=128, ctas_per_sm=1), check=False)
     assert (res.status() == 18) == (exp["status"] == oracle.GROUP_RANGE)
     compare(w, res, exp)
+
+
+def test_bulk_copy_wait_that_runs_out_is_reported_and_survived():
+    """The failure path of the bulk-asynchronous staging, reached without faulting anything: the kernel waits
+    for copies that are never issued, every bounded wait runs out, the status word says so and the kernel
+    finishes the query with plain loads: same bits as the oracle."""
+    w = W.config4(20_011, 0.5, 1000, dim_rows=50000)
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    res, exp, tables = run_both(w, fact, hd, opts=spec(l0_bulk=3, block_threads=128, ctas_per_sm=1, compaction=2))
+    assert res.status() == 22
+    compare(w, res, exp)
+    # the context is still usable and the same query without the switch is clean
+    res, exp, _ = run_both(w, fact, hd, opts=spec(l0_bulk=1, block_threads=128, ctas_per_sm=1, compaction=2), tables=tables)
+    assert res.status() == 0
+    compare(w, res, exp)
