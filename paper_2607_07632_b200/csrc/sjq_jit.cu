@@ -18,6 +18,7 @@
 // silently.
 #include <dlfcn.h>
 
+#include <cstddef>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -145,13 +146,12 @@ std::string jit_shape_header(const RunParams &P, int agg, bool mul, bool hash, i
 {
     std::ostringstream o;
     o << "// generated: the shape of one query\n#define SJQ_ROWS " << (P.rows == 8 ? 8 : 4) << "\n#define SJQ_SLOTS "
-      << (P.slots == 4 ? 4 : 2) << "\n//@body\n";
+      << (P.slots == 4 ? 4 : 2) << "\n#define SJQ_JIT_nstages " << P.nstages << "\n//@body\n";
     o << "#define SJQ_JIT_AGG " << agg << "\n#define SJQ_JIT_MUL " << (mul ? 1 : 0) << "\n#define SJQ_JIT_HASH "
       << (hash ? 1 : 0) << "\n";
     o << "#define SJQ_LB_THREADS " << lb_threads << "\n#define SJQ_LB_BLOCKS " << lb_blocks << "\n";
     if (const char *extra = std::getenv("SJQ_JIT_EXTRA")) o << "// options: " << extra << "\n";
-    o << "#define SJQ_JIT_nstages " << P.nstages << "\n#define SJQ_JIT_nd0 " << P.nd0 << "\n#define SJQ_JIT_nq " << P.nq
-      << "\n";
+    o << "#define SJQ_JIT_nd0 " << P.nd0 << "\n#define SJQ_JIT_nq " << P.nq << "\n";
     o << "#define SJQ_JIT_qfold " << P.qfold << "u\n";
     o << "#define SJQ_JIT_want_count " << P.want_count << "\n#define SJQ_JIT_eager " << P.eager
       << "\n#define SJQ_JIT_has_key " << P.has_key << "\n#define SJQ_JIT_mod32 " << P.mod32
@@ -353,7 +353,16 @@ sjq_status jit_launch(const RunParams &P, int agg, bool mul, bool hash, int grid
         if (st != SJQ_OK) return st;
         kernel = M->kernel;
     }
-    void *args[] = {const_cast<RunParams *>(&P)};
+    // the compiled kernel's parameter struct holds P.nstages stage descriptors (at least one), then the same
+    // fields as RunParams: pack exactly that
+    const size_t nst = (size_t)(P.nstages > 0 ? P.nstages : 1);
+    const size_t tail_from = offsetof(RunParams, sets), tail_bytes = sizeof(RunParams) - tail_from;
+    static_assert(offsetof(RunParams, st) == 0 && offsetof(RunParams, sets) == sizeof(DStage) * (size_t)kMaxStages,
+                  "the stage descriptors lead the parameter block and the rest follows without padding");
+    alignas(16) unsigned char packed[sizeof(RunParams)];
+    std::memcpy(packed, P.st, nst * sizeof(DStage));
+    std::memcpy(packed + nst * sizeof(DStage), reinterpret_cast<const unsigned char *>(&P) + tail_from, tail_bytes);
+    void *args[] = {packed};
     if (cudaLaunchKernel(reinterpret_cast<const void *>(kernel), dim3(grid), dim3(block), args, smem, stream) !=
         cudaSuccess) {
         (void)cudaGetLastError();
