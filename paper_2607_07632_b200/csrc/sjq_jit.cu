@@ -54,10 +54,25 @@ Nvrtc &nvrtc()
     static Nvrtc N;
     static std::once_flag once;
     std::call_once(once, [] {
-        const char *names[] = {"libnvrtc.so.12", "libnvrtc.so", "/usr/local/cuda/lib64/libnvrtc.so.12",
-                               "/usr/local/cuda/lib64/libnvrtc.so"};
-        for (const char *nm : names)
-            if ((N.handle = dlopen(nm, RTLD_NOW | RTLD_LOCAL)) != nullptr) break;
+        // several copies may be around (the toolkit's, one bundled with a Python package): take the newest, since
+        // newer ones know more of the instruction set (256-bit loads need 12.9)
+        const char *names[] = {"/usr/local/cuda/lib64/libnvrtc.so.12", "/usr/local/cuda/lib64/libnvrtc.so",
+                               "libnvrtc.so.12", "libnvrtc.so"};
+        int best = -1;
+        for (const char *nm : names) {
+            void *h = dlopen(nm, RTLD_NOW | RTLD_LOCAL);
+            if (!h) continue;
+            int major = 0, minor = 0;
+            auto version = reinterpret_cast<int (*)(int *, int *)>(dlsym(h, "nvrtcVersion"));
+            const int v = (version && version(&major, &minor) == 0) ? major * 100 + minor : 0;
+            if (v > best) {
+                if (N.handle) dlclose(N.handle);
+                N.handle = h;
+                best = v;
+            } else {
+                dlclose(h);
+            }
+        }
         if (!N.handle) return;
         bool all = true;
         auto sym = [&](const char *s) {
@@ -169,7 +184,7 @@ std::string jit_shape_header(const RunParams &P, int agg, bool mul, bool hash, i
           << "; S.in_smem = " << (int)S.in_smem << "; S.kind = " << (int)S.kind << "; S.simple = " << (int)S.simple
           << "; S.acc = " << (int)S.acc << "; S.acc32 = " << S.acc32 << "; S.code_bits = " << (int)S.code_bits
           << "; S.issue_after = " << (int)S.issue_after << "; S.full = " << (int)S.full << "; S.hot = " << (int)S.hot
-          << ";\n";
+          << "; S.wide = " << (int)S.wide << ";\n";
         for (int i = 0; i < 9; ++i) {
             // INT64_MIN cannot be written as a literal
             if (S.mult[i] == INT64_MIN) o << "        S.mult[" << i << "] = (-9223372036854775807LL - 1);";
@@ -201,7 +216,7 @@ std::string shape_key(const RunParams &P, int agg, bool mul, bool hash, int lb_t
     for (int s = 0; s < P.nstages; ++s) {
         const DStage &S = P.st[s];
         const uint8_t b[] = {S.op, S.is64, S.neg, S.never, S.nset, S.set_idx, S.in_smem, S.kind, S.simple, S.code_bits,
-                             (uint8_t)S.issue_after, S.full, S.hot};
+                             (uint8_t)S.issue_after, S.full, S.hot, S.wide};
         put_raw(b, sizeof(b));
         put_raw(&S.acc, sizeof(S.acc));
         put_raw(&S.acc32, sizeof(S.acc32));
@@ -490,7 +505,7 @@ int canned_shape(int id, RunParams *P, int *agg, bool *mul, bool *hash)
         P->st[0] = canned(OP_HASHBITS, ST_PROBE, true, 0, 0, false);
         P->st[1] = canned(OP_HASH64, ST_PROBE, true, 8, 32, false);
         P->st[2] = canned(OP_LOAD, ST_LOAD, false, 2, 0, false);
-        P->st[0].hot = 1, P->st[1].hot = 2;
+        P->st[0].hot = 1, P->st[1].hot = 2, P->st[1].wide = 1;
         P->nstages = 3, P->nd0 = 1, P->nq = 1;
         P->modulo = 4096, P->modmask = 4095, P->mod32 = 1, P->want_count = 1;
         P->l0_bulk = 1;

@@ -383,6 +383,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
             S.full = (uint8_t)(L.code_bits > 0 && L.code_bits < 8 && L.entries == L.slots);
             if (is_hash_kind(L.kind)) {
                 S.last = (uint64_t)(T->slots_bytes / kBucketBytes); // bucket count
+                S.wide = (uint8_t)((reinterpret_cast<uintptr_t>(T->slots) & 31u) == 0);
                 if (sp.prefilter == 1) {
                     S.op = OP_HASHBITS;
                     S.tab = T->filter;

@@ -92,6 +92,7 @@ struct DStage {
                         // (a stage before the level's first one = on entry)
     uint8_t full;   // sub-byte direct table holding every key of its range: a probe hits iff its key is in range
     uint8_t hot;    // open-addressing join (its bitmap stage and its exact probe): consult the hot-key table first
+    uint8_t wide;   // open-addressing probe: the bucket array starts on a 32-byte boundary, so a bucket is one 256-bit load
     const void *hot_tab; // hot-key table in global memory (kHotSlots + 1 entries), copied to shared memory per block
     uint32_t hot_off;    // byte offset of that copy in dynamic shared memory
     uint32_t hot_pad;
