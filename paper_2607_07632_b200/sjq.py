@@ -294,10 +294,12 @@ class Table:
 
 
 def build_dim(cols: dict, key: str, preds=(), payloads=(), force_kind: int = 0, hash_load_pct: int = 0,
-              max_direct_bytes: int = 0, edit_layout=None, min_code_bits: int = 0) -> Table:
+              max_direct_bytes: int = 0, edit_layout=None, min_code_bits: int = 0, mem_offset: int = 0) -> Table:
     """sjq_dim_plan + sjq_build_dim over a dict of CUDA tensors (dimension columns).  `edit_layout`, if
     given, is called with the planned DimLayout and may change it before the build (sjq_build_dim takes
-    the layout from its caller: tests use this to hand it an undersized or inconsistent one)."""
+    the layout from its caller: tests use this to hand it an undersized or inconsistent one).  `mem_offset`
+    (a multiple of 16) places the table that many bytes into its allocation: table memory only has to be
+    16-byte aligned, and tests use this to get exactly that."""
     names = list(cols.keys())
     tensors = [cols[n] for n in names]
     device = tensors[0].device
@@ -316,7 +318,7 @@ def build_dim(cols: dict, key: str, preds=(), payloads=(), force_kind: int = 0, 
         planned_bytes = layout.table_bytes
         if edit_layout is not None:
             edit_layout(layout)
-        mem = torch.empty(max(planned_bytes, layout.table_bytes), dtype=torch.uint8, device=device)
+        mem = torch.empty(max(planned_bytes, layout.table_bytes) + mem_offset, dtype=torch.uint8, device=device)[mem_offset:]
         status = torch.zeros(1, dtype=torch.int32, device=device)
         handle = ctypes.c_void_p()
         rc = lib().sjq_build_dim(carr, len(names), parr, len(preds), names.index(key), pay, len(payloads),

@@ -744,3 +744,20 @@ def test_result_sort_orders_triples_by_signed_key(n, capacity):
     assert np.array_equal(res.keys.cpu().numpy()[n:], allk[n:])
     assert np.array_equal(res.sums.cpu().numpy()[n:], sums[n:])
     assert np.array_equal(res.counts.cpu().numpy()[n:], counts[n:])
+
+
+def test_open_addressing_table_at_a_16_byte_aligned_address():
+    """Table memory only has to be 16-byte aligned; a bucket array that does not start on a 32-byte boundary is
+    probed with two 128-bit loads instead of one 256-bit load.  Same result either way."""
+    w = W.config5(700_001, 100_000)
+    fact = W.host_fact(w)
+    hd = {d.name: W.host_dim(w, d) for d in w.dims}
+    d = w.dims[0]
+    dev = to_dev(hd[d.name])
+    for off in (0, 16):
+        t = sjq.build_dim(dev, d.key, d.preds, d.payloads, force_kind=sjq.sjq.FORCE_HASH, mem_offset=off).check()
+        assert t.mem.data_ptr() % 32 == off
+        for opts in (sjq.RunOpts(), sjq.RunOpts(specialise=True), sjq.RunOpts(specialise=True, hot_keys=1)):
+            res, exp, _ = run_both(w, fact, hd, opts=opts, tables={d.name: t})
+            assert res.status() == 0
+            compare(w, res, exp)
