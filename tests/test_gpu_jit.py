@@ -49,6 +49,7 @@ def test_random_queries_option_matrix_specialised(seed):
                  spec(agg_path=2), spec(compaction=1), spec(rows_per_lane=8), spec(rows_per_lane=8, compaction=2),
                  spec(no_filter_bitmap=True), spec(group_hash_always=True), spec(dense_slots=4), spec(dense_slots=4, block_threads=768, ctas_per_sm=1),
                  spec(warp_agg=1), spec(warp_agg=1, agg_path=2), spec(warp_agg=2, compaction=1),
+                 spec(hot_keys=1), spec(hot_keys=1, l0_bulk=1, block_threads=256, ctas_per_sm=2), spec(l0_bulk=1, compaction=2),
                  spec(pass_ppm=(900_000,) * (len(w.preds) + len(w.joins))),  # "most rows survive": the queue-free plan
                  spec(order=tuple(reversed(range(len(w.preds) + len(w.joins)))))):
         res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)

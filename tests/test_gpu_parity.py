@@ -51,6 +51,7 @@ def test_random_queries_option_matrix(seed):
                  sjq.RunOpts(block_threads=128, ctas_per_sm=1), sjq.RunOpts(block_threads=256, compaction=2, smem_tables=1), sjq.RunOpts(agg_path=2),
                  sjq.RunOpts(compaction=2), sjq.RunOpts(compaction=1), sjq.RunOpts(no_filter_bitmap=True),
                  sjq.RunOpts(group_hash_always=True), sjq.RunOpts(warp_agg=1), sjq.RunOpts(warp_agg=1, agg_path=2),
+                 sjq.RunOpts(hot_keys=1), sjq.RunOpts(hot_keys=1, compaction=1),
                  sjq.RunOpts(unfused_scratch=sjq.unfused_scratch(w.n_rows, len(w.joins))),
                  sjq.RunOpts(order=tuple(reversed(range(len(w.preds) + len(w.joins)))))):
         res, exp, tables = run_both(w, fact, hd, opts=opts, check=False, dev_fact=dev_fact, tables=tables)
