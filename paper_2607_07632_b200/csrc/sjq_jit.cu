@@ -170,7 +170,7 @@ std::string jit_shape_header(const RunParams &P, int agg, bool mul, bool hash, i
     o << "#define SJQ_JIT_qfold " << P.qfold << "u\n";
     o << "#define SJQ_JIT_want_count " << P.want_count << "\n#define SJQ_JIT_eager " << P.eager
       << "\n#define SJQ_JIT_has_key " << P.has_key << "\n#define SJQ_JIT_mod32 " << P.mod32
-      << "\n#define SJQ_JIT_warp_agg " << P.warp_agg << "\n#define SJQ_JIT_l0_bulk " << P.l0_bulk << "\n#define SJQ_JIT_count32 " << P.count32
+      << "\n#define SJQ_JIT_warp_agg " << P.warp_agg << "\n#define SJQ_JIT_l0_bulk " << P.l0_bulk << "\n#define SJQ_JIT_count32 " << P.count32 << "\n#define SJQ_JIT_sparse_push " << P.sparse_push
       << "\n";
     put(o, "modulo", P.modulo);
     o << "#define SJQ_JIT_modmask " << P.modmask << "ULL\n";
@@ -209,7 +209,7 @@ std::string shape_key(const RunParams &P, int agg, bool mul, bool hash, int lb_t
     auto put_raw = [&](const void *p, size_t n) { k.append(static_cast<const char *>(p), n); };
     const int32_t head[] = {agg, mul ? 1 : 0, hash ? 1 : 0, lb_threads, lb_blocks, P.nstages, P.nd0, P.nq,
                             P.rows, P.want_count, P.eager, P.has_key, P.mod32, (int32_t)P.qfold, P.slots, P.warp_agg,
-                            P.l0_bulk, P.count32};
+                            P.l0_bulk, P.count32, P.sparse_push};
     put_raw(head, sizeof(head));
     put_raw(&P.modulo, sizeof(P.modulo));
     put_raw(&P.modmask, sizeof(P.modmask));

@@ -130,6 +130,7 @@ struct RunParams {
     uint32_t smem_groups; // byte offset of the shared group table
     uint32_t smem_queue;  // byte offset of the per-warp survivor queues
     uint32_t smem_l0;     // byte offset of the per-warp staging buffers of the first column (then their mbarriers)
+    int32_t sparse_push;  // few rows survive level 0: the push into the first queue walks the set bits of the mask
     int32_t count32;      // fewer than 2^32 fact rows: a block's count of a group fits 32 bits (no carry into the high word)
     int32_t l0_bulk;      // compiled kernels: the first column arrives by bulk-asynchronous copies into shared memory
 };
