@@ -289,7 +289,7 @@ typedef struct sjq_result {
 
 /* Tuning and ablation switches; a zeroed struct (or NULL) means defaults. */
 typedef struct sjq_run_opts {
-    int32_t block_threads; /* 0 = library chooses (384; a kernel compiled for the query may run 1024); else a
+    int32_t block_threads; /* 0 = library chooses (384; a kernel compiled for the query may run 640 or 1024); else a
                               multiple of 32 in 128..384, or up to 1024 together with `specialise` */
     int32_t ctas_per_sm;   /* 0 = as many as fit */
     int32_t eager_loads;   /* 1 = load every column for every row (ablation of lazy loading) */
