@@ -464,6 +464,7 @@ def main():
     ap.add_argument("--sel", type=float, default=0.1, help="c4: fact predicate selectivity")
     ap.add_argument("--groups", type=int, default=1000, help="c4: number of groups")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-chunk-rows", type=int, default=16 << 20, help="rows per chunk of the host-buffer pipeline")
     ap.add_argument("--cpu-sample-rows", type=int, default=100_000_000)
     ap.add_argument("--interpret", action="store_true",
                     help="interpret the query descriptor instead of compiling the fused kernel for the query's shape")
@@ -628,7 +629,7 @@ def main():
                          for dn, cols in dims.items()}
             dim_bytes = sum(v.numel() * v.element_size() for cols in host_dims.values() for v in cols.values())
             torch.cuda.synchronize()
-            chunk = min(n, 32 << 20) // 4 * 4 or 4
+            chunk = min(n, args.e2e_chunk_rows) // 4 * 4 or 4
             staging = torch.empty(sjq.staging_bytes(host_fact, chunk), dtype=torch.uint8, device=device)
             eres, ehost = None, None
 
