@@ -36,6 +36,11 @@ def _run(w):
     variants = [sjq.RunOpts(specialise=True), sjq.RunOpts(specialise=False)]
     if w.mode == "HASHED":  # the group hash table as well as the direct-indexed table a modulo key allows
         variants.append(sjq.RunOpts(specialise=True, group_hash_always=True))
+    if any(t.layout.kind_name.startswith("HASH") for t in tables.values()):
+        # open-addressing joins: with the hot-key table switched off and forced on (the default decides by size)
+        variants += [sjq.RunOpts(specialise=True, hot_keys=2), sjq.RunOpts(specialise=True, hot_keys=1)]
+    # the first column staged by bulk-asynchronous copies where the shared memory is there (else plain loads)
+    variants.append(sjq.RunOpts(specialise=True, l0_bulk=1))
     for opts in variants:
         res = sjq.run_workload(w, fact, tables, opts)
         torch.cuda.synchronize()
