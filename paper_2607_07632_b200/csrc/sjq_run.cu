@@ -744,7 +744,24 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     // would crowd out the L1 (config 3: 1.43 -> 1.32 ms, config 5: 2.8 -> 1.8 ms), given enough tiles per
     // block to even out the tail.
     bool single_block = false;
-    if (opts.specialise && !opts.block_threads && !opts.ctas_per_sm && P.nq) {
+    // Between the two: a kernel with queues whose shared memory is moderate (more than three 384-thread blocks
+    // could share, at most 100 KB as a 640-thread block) runs as two 640-thread blocks: 40 warps instead of 24 or
+    // 32 and the L1 keeps half of the SM's memory (two-join workload 0.101 -> 0.094 ms, city x brand 0.681 ->
+    // 0.667, city x city 0.700 -> 0.691).
+    bool two_wide_queue_blocks = false;
+    if (opts.specialise && !opts.block_threads && !opts.ctas_per_sm && P.nq && !opts.unfused &&
+        stage_bytes + tables + hot_bytes + group_bytes + queue_bytes(block) > ((size_t)48 << 10)) {
+        size_t tables640 = 0;
+        if (stage_tables(640, &tables640) &&
+            stage_bytes + tables640 + hot_bytes + group_bytes + queue_bytes(640) <= ((size_t)100 << 10)) {
+            block = 640;
+            tables = tables640;
+            two_wide_queue_blocks = true;
+        } else if (!stage_tables(block, &tables)) {
+            return SJQ_ERR_UNSUPPORTED;
+        }
+    }
+    if (opts.specialise && !opts.block_threads && !opts.ctas_per_sm && P.nq && !two_wide_queue_blocks) {
         const size_t copies = tables + hot_bytes + group_bytes;
         const int64_t tiles_per_block = n / ((int64_t)1024 * 4 * P.slots) / dev.sm_count;
         size_t tables1024 = 0;
@@ -805,7 +822,7 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     // (three blocks of 384 threads when their shared memory leaves the L1 alone: 56 registers are enough for the
     // short pipelines that have so little state, and 36 warps hide more latency than 24)
     const int lb_blocks = single_block ? 1
-                          : two_wide_blocks ? 2
+                          : (two_wide_blocks || two_wide_queue_blocks) ? 2
                           : opts.ctas_per_sm > 0 ? opts.ctas_per_sm
                           : block > 512 ? 1
                           : (block <= 384 && smem_without_bulk <= ((size_t)48 << 10)) ? 3
