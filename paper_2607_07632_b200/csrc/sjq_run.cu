@@ -688,9 +688,11 @@ extern "C" sjq_status sjq_run(const sjq_col *fact, int nfact, const sjq_pred *pr
     // A compiled kernel without queues whose rows all meet in a shared group table runs as two blocks of 640
     // threads per SM: two copies of the table instead of three and 40 warps instead of 36 (selectivity sweep at
     // 100 %, a thousand groups: 2.73 -> 2.52 ms; 64 groups 2.57 -> 2.39; 4000 groups 3.25 -> 2.56).
+    // With register accumulators two blocks of 768 threads (48 warps at 42 registers) help while some rows still
+    // drop (the sweep at 50 %, one group: 1.48 -> 1.41 ms) and cost a little when none does (100 %: 2.18 -> 2.22).
     const bool two_wide_blocks = opts.specialise && !opts.unfused && !opts.block_threads && !opts.ctas_per_sm &&
-                                 P.nq == 0 && aggp == AGG_SMEM;
-    if (two_wide_blocks) block = 640;
+                                 P.nq == 0 && (aggp == AGG_SMEM || (aggp == AGG_SCALAR && reach[nfilter] < 0.8));
+    if (two_wide_blocks) block = aggp == AGG_SMEM ? 640 : 768;
     const size_t smem_cap = (size_t)dev.max_smem_optin - 1024; // static reduce scratch + slack
     const size_t stage_bytes = align_up((size_t)ns * sizeof(DStage), 16);
     if (hot_bytes && stage_bytes + hot_bytes + group_bytes +
